@@ -1,0 +1,137 @@
+"""ctypes front end of the CPU oracle (``csr_oracle.c``) plus the storage-format step.
+
+TEST INFRASTRUCTURE ONLY: tests, the smoke check and the benchmark's CPU legs call this.
+Nothing here is shared with, or imported by, the CUDA path.
+
+Paper passages: Eq. 2-4 (matching pursuit), Eq. 12 (de-sparse), and the "Analysis for
+CSR" paragraph (each kept entry is stored as an INT16 index and an fp16 coefficient, so a
+vector of d_h channels costs 32*s*s_n bits).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "csr_oracle.c")
+_LIB = os.path.join(_HERE, "libcsr_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP, no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-ffp-contract=off", "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i64, i32, p = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p
+        lib.csr_oracle_encode.argtypes = [p, p, i64, i32, i32, i32, p, p, p, p, p]
+        lib.csr_oracle_encode.restype = None
+        lib.csr_oracle_reconstruct.argtypes = [p, p, p, i64, i32, i32, i32, p]
+        lib.csr_oracle_reconstruct.restype = None
+        lib.csr_oracle_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().csr_oracle_num_threads())
+
+
+@dataclass
+class MPResult:
+    idx: np.ndarray       # [M][s] int32, selection order
+    coef: np.ndarray      # [M][s] float64, signed
+    gap: np.ndarray       # [M][s] relative gap between the two largest |correlations|
+    resnorm: np.ndarray   # [M][s] ||R_{g+1}|| after iteration g
+    residual: np.ndarray  # [M][d] R_s
+
+
+def _f32c(a: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.float32:
+        raise TypeError("the oracle takes fp32 bit patterns (widen bf16 to fp32 first)")
+    return a
+
+
+def mp_encode(D: np.ndarray, X: np.ndarray, s: int) -> MPResult:
+    """Matching pursuit, Eq. 2-4.  D [N][d] fp32 (one atom per row), X [M][d] fp32."""
+    D = _f32c(D)
+    X = _f32c(X)
+    N, d = D.shape
+    M = X.shape[0]
+    if X.ndim != 2 or X.shape[1] != d or s < 1:
+        raise ValueError("shape mismatch")
+    idx = np.empty((M, s), np.int32)
+    coef = np.empty((M, s), np.float64)
+    gap = np.empty((M, s), np.float64)
+    resnorm = np.empty((M, s), np.float64)
+    residual = np.empty((M, d), np.float64)
+    if M:
+        _load().csr_oracle_encode(D.ctypes.data, X.ctypes.data, M, d, N, s, idx.ctypes.data,
+                                  coef.ctypes.data, gap.ctypes.data, resnorm.ctypes.data,
+                                  residual.ctypes.data)
+    return MPResult(idx, coef, gap, resnorm, residual)
+
+
+def reconstruct(D: np.ndarray, idx: np.ndarray, coef: np.ndarray) -> np.ndarray:
+    """De-sparse, Eq. 12: X_hat = sum over the stored entries of coef * atom (fp64)."""
+    D = _f32c(D)
+    N, d = D.shape
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    coef = np.ascontiguousarray(coef, dtype=np.float64)
+    M, s = idx.shape
+    if coef.shape != (M, s):
+        raise ValueError("shape mismatch")
+    if M and (idx.min() < 0 or idx.max() >= N):
+        raise ValueError("index out of range")
+    out = np.empty((M, d), np.float64)
+    if M:
+        _load().csr_oracle_reconstruct(D.ctypes.data, idx.ctypes.data, coef.ctypes.data, M, d, N, s,
+                                       out.ctypes.data)
+    return out
+
+
+# --- storage format ("Analysis for CSR") -------------------------------------------------
+
+def pack_codes(idx: np.ndarray, coef: np.ndarray):
+    """Stored form of r: 16-bit index and fp16 coefficient per kept entry.
+
+    The coefficient goes fp64 -> fp32 -> fp16, round-to-nearest-even each time (the
+    kernel's coefficient leaves its arithmetic as fp32).  Indices are kept unsigned so
+    that dictionaries of up to 65536 atoms fit.
+    """
+    if idx.size and (idx.min() < 0 or idx.max() > 0xFFFF):
+        raise ValueError("index does not fit 16 bits")
+    return idx.astype(np.uint16), coef.astype(np.float32).astype(np.float16)
+
+
+def unpack_codes(idx16: np.ndarray, coef16: np.ndarray):
+    return idx16.astype(np.int32), coef16.astype(np.float64)
+
+
+def code_bits_per_channel(d_h: int, s: int, s_n: int = 1) -> float:
+    """Equivalent quantisation bits per channel: (16 + 16) * s * s_n / d_h."""
+    return 32.0 * s * s_n / d_h
+
+
+def code_bytes_per_vector(s: int, s_n: int = 1) -> int:
+    return 4 * s * s_n
+
+
+def relative_error(X: np.ndarray, X_hat: np.ndarray) -> np.ndarray:
+    """Per-vector ||x - x_hat|| / ||x|| in fp64 (0 for a zero vector)."""
+    X = np.asarray(X, np.float64)
+    num = np.linalg.norm(X - np.asarray(X_hat, np.float64), axis=1)
+    den = np.linalg.norm(X, axis=1)
+    return np.where(den > 0, num / np.where(den > 0, den, 1.0), 0.0)

@@ -1,0 +1,284 @@
+"""Pins for the CPU oracle: each test checks it against something the paper or the
+mathematics fixes, not against its own formula.
+
+Matching pursuit: paper Eq. 2-4; de-sparse: Eq. 12; storage format: "Analysis for CSR".
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+from oracle import csr_oracle as orc
+from paper_2412_11741_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand_dict(rng, N, d):
+    return wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+
+
+# --- brute force on tiny inputs (pins Eq. 2-3 and the order of Eq. 4) --------------------
+
+def _brute_force_mp(D, x, s):
+    """Independent restatement: stable descending sort of |D R| picks the atom."""
+    D = D.astype(np.float64)
+    R = x.astype(np.float64).copy()
+    idx, coef = [], []
+    for _ in range(s):
+        c = np.array([float(np.dot(R, D[n])) for n in range(D.shape[0])])
+        order = sorted(range(len(c)), key=lambda n: (-abs(c[n]), n))
+        i = order[0]
+        idx.append(i)
+        coef.append(c[i])
+        R = R - c[i] * D[i]
+    return np.array(idx), np.array(coef), R
+
+
+@pytest.mark.parametrize("d,N,s", [(2, 3, 2), (4, 7, 3), (8, 16, 4), (5, 16, 4), (8, 1, 2)])
+def test_brute_force_tiny(d, N, s):
+    rng = np.random.default_rng(100 + d * N)
+    D = _rand_dict(rng, N, d)
+    X = rng.standard_normal((37, d)).astype(np.float32)
+    res = orc.mp_encode(D, X, s)
+    for m in range(X.shape[0]):
+        bi, bc, bR = _brute_force_mp(D, X[m], s)
+        assert np.array_equal(res.idx[m], bi)
+        np.testing.assert_allclose(res.coef[m], bc, rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(res.residual[m], bR, rtol=0, atol=1e-13)
+
+
+def test_exhaustive_best_single_atom():
+    """For s = 1 the pick must minimise ||x - c d_n|| over every atom and every scalar c
+    (Eq. 1 restricted to one atom): the optimum is c = x.d_n / ||d_n||^2."""
+    rng = np.random.default_rng(7)
+    D = _rand_dict(rng, 12, 6)
+    X = rng.standard_normal((50, 6)).astype(np.float32)
+    res = orc.mp_encode(D, X, 1)
+    Dd = D.astype(np.float64)
+    for m in range(50):
+        errs = []
+        for n in range(12):
+            c = np.dot(X[m], Dd[n]) / np.dot(Dd[n], Dd[n])
+            errs.append(np.linalg.norm(X[m] - c * Dd[n]))
+        # unit-norm atoms (to ~1e-7): the arg-max of |x.d_n| is the arg-min of the error
+        assert res.idx[m, 0] == int(np.argmin(errs))
+
+
+# --- s = 1 reduces to a library matmul ---------------------------------------------------
+
+def test_s1_matches_matmul_argmax():
+    rng = np.random.default_rng(3)
+    D = _rand_dict(rng, 300, 64)
+    X = rng.standard_normal((500, 64)).astype(np.float32)
+    C = X.astype(np.float64) @ D.astype(np.float64).T
+    res = orc.mp_encode(D, X, 1)
+    assert np.array_equal(res.idx[:, 0], np.argmax(np.abs(C), axis=1))
+    np.testing.assert_allclose(res.coef[:, 0], C[np.arange(500), res.idx[:, 0]], rtol=1e-12)
+    srt = np.sort(np.abs(C), axis=1)
+    np.testing.assert_allclose(res.gap[:, 0], (srt[:, -1] - srt[:, -2]) / srt[:, -1], rtol=1e-9, atol=1e-13)
+
+
+# --- energy identity and monotone residual (pins the update and the signed coefficient) --
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_energy_identity_and_monotone(seed):
+    rng = np.random.default_rng(seed)
+    D = _rand_dict(rng, 256, 32)
+    X = (rng.standard_normal((200, 32)) * 3).astype(np.float32)
+    s = 12
+    res = orc.mp_encode(D, X, s)
+    x2 = (X.astype(np.float64) ** 2).sum(1)
+    dn2 = (D.astype(np.float64) ** 2).sum(1)
+    # exact identity for arbitrary atom norms: each step removes c^2 (2 - ||d||^2)
+    removed = (res.coef ** 2 * (2.0 - dn2[res.idx])).sum(1)
+    np.testing.assert_allclose(x2, (res.residual ** 2).sum(1) + removed, rtol=1e-12)
+    # unit-norm atoms: ||x||^2 = ||R_s||^2 + sum c^2 up to the 1e-7 normalisation error
+    np.testing.assert_allclose(x2, (res.residual ** 2).sum(1) + (res.coef ** 2).sum(1), rtol=5e-6)
+    norms = np.concatenate([np.sqrt(x2)[:, None], res.resnorm], axis=1)
+    assert np.all(np.diff(norms, axis=1) <= 1e-12)
+    np.testing.assert_allclose(res.resnorm[:, -1], np.linalg.norm(res.residual, axis=1), rtol=1e-12)
+    # |c_g| is non-increasing is NOT a property of MP; but |c_g| <= ||R_g|| always is
+    assert np.all(np.abs(res.coef) <= norms[:, :-1] * (1 + 1e-6))
+
+
+def test_sign_of_coefficient_is_kept():
+    D = np.eye(4, dtype=np.float32)
+    X = np.array([[0.5, -3.0, 1.0, 0.0]], np.float32)
+    res = orc.mp_encode(D, X, 2)
+    assert res.idx.tolist() == [[1, 2]]
+    assert res.coef.tolist() == [[-3.0, 1.0]]
+
+
+# --- orthonormal dictionary: textbook closed form ---------------------------------------
+
+def test_identity_dictionary_exact_recovery():
+    rng = np.random.default_rng(11)
+    d = 16
+    D = np.eye(d, dtype=np.float32)
+    X = rng.standard_normal((64, d)).astype(np.float32)
+    res = orc.mp_encode(D, X, d)
+    order = np.argsort(-np.abs(X), axis=1, kind="stable")
+    assert np.array_equal(res.idx, order)
+    assert np.array_equal(res.coef, np.take_along_axis(X.astype(np.float64), order, 1))
+    assert np.all(res.residual == 0.0)
+
+
+def test_orthogonal_dictionary_closed_form():
+    rng = np.random.default_rng(12)
+    d = 24
+    Q, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    D = Q.T.astype(np.float32)  # rows orthonormal to fp32 rounding
+    X = rng.standard_normal((40, d)).astype(np.float32)
+    res = orc.mp_encode(D, X, d)
+    proj = X.astype(np.float64) @ D.astype(np.float64).T
+    order = np.argsort(-np.abs(proj), axis=1, kind="stable")
+    assert np.array_equal(res.idx, order)
+    np.testing.assert_allclose(res.coef, np.take_along_axis(proj, order, 1), atol=1e-5)
+    assert np.abs(res.residual).max() < 1e-5
+
+
+# --- metamorphic relations ----------------------------------------------------------------
+
+def test_metamorphic():
+    rng = np.random.default_rng(21)
+    N, d, s = 128, 32, 6
+    D = _rand_dict(rng, N, d)
+    X = rng.standard_normal((100, d)).astype(np.float32)
+    base = orc.mp_encode(D, X, s)
+    # scaling the input by a power of two scales the coefficients, same atoms
+    sc = orc.mp_encode(D, (X * np.float32(4.0)), s)
+    assert np.array_equal(sc.idx, base.idx)
+    np.testing.assert_allclose(sc.coef, 4.0 * base.coef, rtol=1e-13)
+    # negating one atom negates its coefficients only
+    D2 = D.copy()
+    D2[5] = -D2[5]
+    ng = orc.mp_encode(D2, X, s)
+    assert np.array_equal(ng.idx, base.idx)
+    sign = np.where(base.idx == 5, -1.0, 1.0)
+    np.testing.assert_allclose(ng.coef, sign * base.coef, rtol=1e-13)
+    # permuting the atoms permutes the indices
+    perm = rng.permutation(N)
+    pm = orc.mp_encode(D[perm], X, s)
+    assert np.array_equal(perm[pm.idx], base.idx)
+    np.testing.assert_allclose(pm.coef, base.coef, rtol=1e-13)
+    # appended zero atoms are never picked
+    zp = orc.mp_encode(np.concatenate([D, np.zeros((16, d), np.float32)]), X, s)
+    assert np.array_equal(zp.idx, base.idx)
+
+
+def test_tie_break_lowest_index_and_zero_residual():
+    D = np.array([[1, 0], [0, 1], [1, 0], [-1, 0]], np.float32)
+    X = np.array([[2.0, 0.0], [0.0, 0.0]], np.float32)
+    res = orc.mp_encode(D, X, 3)
+    # atoms 0, 2, 3 tie in |correlation| at step 0: the lowest index wins; after that the
+    # residual is exactly zero and (0, 0) is emitted
+    assert res.idx[0].tolist() == [0, 0, 0]
+    assert res.coef[0].tolist() == [2.0, 0.0, 0.0]
+    assert res.idx[1].tolist() == [0, 0, 0] and res.coef[1].tolist() == [0.0, 0.0, 0.0]
+    assert res.gap[0, 0] == 0.0
+
+
+def test_repeated_atoms_accumulate_in_reconstruction():
+    # two coherent atoms: MP returns to the first one; Eq. 12 must add both entries
+    D = wl.normalise_rows(np.array([[1.0, 0.0], [1.0, 1.0]], np.float32))
+    X = np.array([[1.0, 0.45]], np.float32)
+    res = orc.mp_encode(D, X, 4)
+    assert len(set(res.idx[0].tolist())) < 4
+    xh = orc.reconstruct(D, res.idx, res.coef)
+    np.testing.assert_allclose(xh + res.residual, X.astype(np.float64), atol=1e-14)
+
+
+# --- de-sparse equals dense r times D (Eq. 12) -------------------------------------------
+
+def test_reconstruct_is_dense_product():
+    rng = np.random.default_rng(5)
+    N, d, s, M = 64, 16, 5, 80
+    D = _rand_dict(rng, N, d)
+    idx = rng.integers(0, N, size=(M, s)).astype(np.int32)
+    idx[:, 1] = idx[:, 0]  # force duplicates
+    coef = rng.standard_normal((M, s))
+    r = np.zeros((M, N))
+    for m in range(M):
+        for g in range(s):
+            r[m, idx[m, g]] += coef[m, g]
+    np.testing.assert_allclose(orc.reconstruct(D, idx, coef), r @ D.astype(np.float64), atol=1e-13)
+
+
+def test_codes_plus_residual_give_back_x():
+    w = wl.tiny(M=256)
+    res = orc.mp_encode(w.D, w.X, w.s)
+    xh = orc.reconstruct(w.D, res.idx, res.coef)
+    np.testing.assert_allclose(xh + res.residual, w.X.astype(np.float64), atol=1e-13)
+    np.testing.assert_allclose(orc.relative_error(w.X, xh),
+                               res.resnorm[:, -1] / np.linalg.norm(w.X.astype(np.float64), axis=1), rtol=1e-9)
+
+
+# --- exactly sparse inputs (config 1's extra rows) ---------------------------------------
+
+def test_sparse_rows_first_pick_in_support_and_decay():
+    w = wl.tiny(M=0)
+    lo, hi = w.meta["sparse_rows"]
+    X = w.X[lo:hi]
+    support = w.meta["support"]
+    errs = []
+    for s in (8, 16, 32):
+        res = orc.mp_encode(w.D, X, s)
+        if s == 8:
+            assert all(res.idx[m, 0] in support[m] for m in range(X.shape[0]))
+        errs.append((res.resnorm[:, -1] / np.linalg.norm(X, axis=1)).mean())
+    # MP (unlike OMP) does not recover a sparse combination of coherent atoms in s steps,
+    # but the residual must fall quickly
+    assert errs[0] < 0.3 and errs[1] < 0.25 * errs[0] and errs[2] < 0.1 * errs[1]
+
+
+def test_error_falls_with_s_and_N():
+    """Qualitative trend of the paper's MSE tables: more entries or more atoms, less error."""
+    rng = np.random.default_rng(9)
+    X = rng.standard_normal((300, 32)).astype(np.float32)
+    Dbig = _rand_dict(rng, 512, 32)
+
+    def err(D, s):
+        r = orc.mp_encode(D, X, s)
+        return orc.relative_error(X, orc.reconstruct(D, r.idx, r.coef)).mean()
+
+    assert err(Dbig, 2) > err(Dbig, 4) > err(Dbig, 8)
+    assert err(Dbig[:64], 4) > err(Dbig[:256], 4) > err(Dbig, 4)
+
+
+# --- storage format -------------------------------------------------------------------------
+
+def test_format_golden():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "code_format.txt")) if l.strip() and not l.startswith("#")]
+    for d_h, s, s_n, bits, ratio in rows:
+        d_h, s, s_n = int(d_h), int(s), int(s_n)
+        assert orc.code_bits_per_channel(d_h, s, s_n) == float(bits)
+        assert 2 * d_h / orc.code_bytes_per_vector(s, s_n) == float(ratio)
+    idx = np.array([[0, 65535, 7]], np.int32)
+    coef = np.array([[1.0, -0.333333333, 48.123]])
+    i16, c16 = orc.pack_codes(idx, coef)
+    assert i16.dtype == np.uint16 and c16.dtype == np.float16
+    assert i16.nbytes + c16.nbytes == orc.code_bytes_per_vector(3)
+    bi, bc = orc.unpack_codes(i16, c16)
+    assert np.array_equal(bi, idx)
+    np.testing.assert_allclose(bc, coef, rtol=2.0 ** -11)
+    with pytest.raises(ValueError):
+        orc.pack_codes(np.array([[70000]], np.int32), np.array([[1.0]]))
+
+
+# --- planted mistakes must be caught (the pins are not vacuous) -----------------------------
+
+def test_pins_detect_unsigned_coefficient():
+    rng = np.random.default_rng(0)
+    D = _rand_dict(rng, 64, 16)
+    x = rng.standard_normal(16)
+    R = x.copy()
+    e = 0.0
+    for _ in range(4):
+        c = D.astype(np.float64) @ R
+        i = int(np.argmax(np.abs(c)))
+        R = R - abs(c[i]) * D[i]          # the literal reading of Eq. 2
+        e += c[i] ** 2
+    # with an unsigned coefficient the energy identity breaks for this input
+    assert abs((x ** 2).sum() - (R ** 2).sum() - e) > 1e-3
