@@ -1,0 +1,162 @@
+/*
+ * libcsr — sparse codec of CSR ("Cache Sparse Representation") for NVIDIA B200 (sm_100a).
+ *
+ * The codec turns every dense key/value head vector x (d channels) into s
+ * (atom index, coefficient) pairs over a fixed dictionary D of N unit-norm atoms by
+ * greedy matching pursuit, and turns such pairs back into dense vectors.
+ *
+ * Conventions shared by every entry point
+ *   - All functions return an int status: CSR_OK (0) or a negative CSR_ERR_* code.
+ *     csr_last_error_string() returns the message of the calling thread's last failure.
+ *     No exception crosses this boundary and no argument error is undefined behaviour.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the
+ *     caller.  The library neither frees nor keeps caller pointers after a call's work
+ *     has finished on its stream.
+ *   - Calls are asynchronous with respect to the host: work is enqueued on the given
+ *     CUDA stream (the 8-argument forms use the legacy default stream, 0) and the
+ *     function returns without synchronising, except csr_encode_host and
+ *     csr_device_status, which synchronise.
+ *   - Layout.  D is [N][d] row-major fp32: one atom per row, the d channels contiguous
+ *     (the paper's d x N matrix of "Sparse representation", stored column by column).
+ *     Atoms are assumed unit l2-norm; this is not checked and the formulas are applied
+ *     as written if they are not.  X and X_hat are [M][d] row-major.  Codes are
+ *     idx [M][s] and coef [M][s] row-major, entry g of a row being iteration g of the
+ *     pursuit.
+ *   - Limits: d in {64, 128}; 1 <= N <= 65536 (indices are stored as uint16); 1 <= s <= 64;
+ *     M >= 0 (M == 0 succeeds and does nothing).  The fast mode additionally needs
+ *     N % 128 == 0.  Data pointers must be 16-byte aligned.
+ *   - NaN or Inf in X or D: results are unspecified; the call neither crashes nor hangs.
+ *   - Device-side waits are bounded.  If one expires the kernel stops early, the outputs
+ *     are unspecified and csr_device_status() reports CSR_ERR_TIMEOUT.
+ */
+#ifndef CSR_H_
+#define CSR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CSR_VERSION 100
+
+#define CSR_OK 0
+#define CSR_ERR_INVALID_ARG (-1)
+#define CSR_ERR_UNSUPPORTED (-2)
+#define CSR_ERR_ALIGNMENT (-3)
+#define CSR_ERR_CUDA (-4)
+#define CSR_ERR_TIMEOUT (-5)
+#define CSR_ERR_WORKSPACE (-6)
+
+/* element types of X, X_hat and coef */
+#define CSR_DTYPE_F32 0
+#define CSR_DTYPE_BF16 1
+#define CSR_DTYPE_F16 2
+
+/*
+ * Arithmetic mode of the encoder.
+ *   CSR_MODE_FP32_EXACT  correlations with fp32 operands and fp32 accumulation on the
+ *                        plain ALUs; whenever the two largest |correlations| of a row
+ *                        are closer than fp32 rounding can resolve, that row's step is
+ *                        re-scored in fp64.  The coefficient and the residual update
+ *                        are fp64.  Selects the same atoms as an fp64 evaluation of the
+ *                        pursuit except at exact-to-rounding ties.
+ *   CSR_MODE_BF16_FAST   correlations on the tcgen05 tensor cores with bf16 operands
+ *                        (residual and atoms rounded to bf16) and fp32 accumulation.
+ *                        Near-tied picks may differ from an fp64 evaluation; the mean
+ *                        reconstruction error does not.
+ */
+#define CSR_MODE_FP32_EXACT 0
+#define CSR_MODE_BF16_FAST 1
+
+typedef struct csr_encode_params {
+    uint32_t struct_size;   /* sizeof(csr_encode_params_t), for versioning */
+    int32_t mode;           /* CSR_MODE_* */
+    const void* D;          /* [N][d] fp32 */
+    const void* X;          /* [M][d], x_dtype (F32 or BF16) */
+    int32_t x_dtype;
+    int32_t coef_dtype;     /* F16 (the paper's stored form) or F32 */
+    int64_t M;
+    int32_t d, N, s;
+    int32_t reserved0;
+    uint16_t* out_idx;      /* [M][s] */
+    void* out_coef;         /* [M][s], coef_dtype */
+    void* stream;           /* cudaStream_t; NULL = legacy default stream */
+    void* workspace;        /* scratch of at least csr_encode_workspace_bytes(); NULL = the
+                               library keeps one grow-only allocation per device */
+    size_t workspace_bytes;
+} csr_encode_params_t;
+
+typedef struct csr_reconstruct_params {
+    uint32_t struct_size;
+    int32_t reserved0;
+    const void* D;          /* [N][d] fp32 */
+    const uint16_t* idx;    /* [M][s] */
+    const void* coef;       /* [M][s], coef_dtype */
+    int32_t coef_dtype;     /* F16 or F32 */
+    int32_t out_dtype;      /* BF16 or F32 */
+    int64_t M;
+    int32_t d, N, s;
+    int32_t reserved1;
+    void* X_hat;            /* [M][d], out_dtype */
+    void* stream;
+} csr_reconstruct_params_t;
+
+/*
+ * Matching-pursuit encode ("Sparse representation", Eq. 2-4; "KV Decomposition and
+ * Sparse Storage").  For every row x of X: R_0 = x; for g = 0 .. s-1: correlate R_g
+ * with all N atoms, i_g = argmax_n |R_g . d_n| (lowest n among equal values),
+ * c_g = R_g . d_{i_g} (signed), R_{g+1} = R_g - c_g d_{i_g}.  Atoms are never masked:
+ * an atom may be selected more than once.  A zero residual yields (0, 0).
+ * Writes out_idx[m][g] = i_g and out_coef[m][g] = c_g in the stored form of "Analysis
+ * for CSR": 16-bit index, fp16 coefficient (round to nearest even), 4*s bytes per row.
+ *
+ * 8-argument form: X is bf16, out_coef is fp16, mode is CSR_MODE_BF16_FAST, stream 0,
+ * library-owned workspace.
+ */
+int csr_encode(const void* D, const void* X, int64_t M, int d, int N, int s, uint16_t* out_idx,
+               void* out_coef);
+int csr_encode_ex(const csr_encode_params_t* p);
+
+/* Scratch bytes csr_encode_ex needs for the given mode and sizes (0 if none);
+ * negative CSR_ERR_* on invalid arguments. */
+int64_t csr_encode_workspace_bytes(int mode, int d, int N);
+
+/*
+ * De-sparse ("De-Sparse to restore", Eq. 12): X_hat[m,:] = sum_g coef[m][g] * D[idx[m][g]][:],
+ * accumulated in fp32 in the order g = 0 .. s-1; repeated indices accumulate.  Every idx
+ * must be < N (larger values are clamped to N-1 rather than read out of bounds).
+ *
+ * 8-argument form: coef is fp16, X_hat is bf16, stream 0.
+ */
+int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_t M, int d, int N,
+                    int s, void* X_hat);
+int csr_reconstruct_ex(const csr_reconstruct_params_t* p);
+
+/*
+ * Encode with HOST buffers (the same operation as csr_encode_ex; only X, out_idx and
+ * out_coef are host pointers, ideally page-locked).  X is copied to the device in
+ * chunks that overlap with the encoding of the previous chunk, the codes are copied
+ * back, and the function returns after everything has finished.  D stays a device
+ * pointer.  Uses library-owned device staging buffers (grow-only, per device).
+ */
+int csr_encode_host(const csr_encode_params_t* p);
+
+/*
+ * Synchronises the stream and reports whether a kernel of this library has given up on a
+ * bounded wait since the last call of this function on the current device: CSR_OK or
+ * CSR_ERR_TIMEOUT (or CSR_ERR_CUDA if the stream itself is in error).
+ */
+int csr_device_status(void* stream);
+
+/* Releases the library-owned device buffers of the current device. */
+int csr_release_workspace(void);
+
+const char* csr_last_error_string(void);
+int csr_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSR_H_ */

@@ -1,0 +1,247 @@
+"""ctypes binding of libcsr.so: argument marshalling only.
+
+Every function here has the name of the C entry point it forwards to (see include/csr.h).
+torch is used for device memory and the current stream; no arithmetic of the codec is
+done in Python.  If the shared library is missing or cannot be loaded the import of a
+function fails loudly: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libcsr.so")
+
+CSR_OK = 0
+CSR_ERR_INVALID_ARG = -1
+CSR_ERR_UNSUPPORTED = -2
+CSR_ERR_ALIGNMENT = -3
+CSR_ERR_CUDA = -4
+CSR_ERR_TIMEOUT = -5
+CSR_ERR_WORKSPACE = -6
+
+CSR_DTYPE_F32 = 0
+CSR_DTYPE_BF16 = 1
+CSR_DTYPE_F16 = 2
+
+CSR_MODE_FP32_EXACT = 0
+CSR_MODE_BF16_FAST = 1
+
+EXPORTS = (
+    "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
+    "csr_encode_host", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
+)
+
+
+class csr_encode_params_t(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("mode", ctypes.c_int32),
+        ("D", ctypes.c_void_p), ("X", ctypes.c_void_p),
+        ("x_dtype", ctypes.c_int32), ("coef_dtype", ctypes.c_int32),
+        ("M", ctypes.c_int64),
+        ("d", ctypes.c_int32), ("N", ctypes.c_int32), ("s", ctypes.c_int32), ("reserved0", ctypes.c_int32),
+        ("out_idx", ctypes.c_void_p), ("out_coef", ctypes.c_void_p),
+        ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+    ]
+
+
+class csr_reconstruct_params_t(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("reserved0", ctypes.c_int32),
+        ("D", ctypes.c_void_p), ("idx", ctypes.c_void_p), ("coef", ctypes.c_void_p),
+        ("coef_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+        ("M", ctypes.c_int64),
+        ("d", ctypes.c_int32), ("N", ctypes.c_int32), ("s", ctypes.c_int32), ("reserved1", ctypes.c_int32),
+        ("X_hat", ctypes.c_void_p), ("stream", ctypes.c_void_p),
+    ]
+
+
+class CsrError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"libcsr error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libcsr.so (built in-tree by paper_2412_11741_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2412_11741_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
+        L.csr_encode.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp]
+        L.csr_encode.restype = i32
+        L.csr_encode_ex.argtypes = [ctypes.POINTER(csr_encode_params_t)]
+        L.csr_encode_ex.restype = i32
+        L.csr_encode_host.argtypes = [ctypes.POINTER(csr_encode_params_t)]
+        L.csr_encode_host.restype = i32
+        L.csr_encode_workspace_bytes.argtypes = [i32, i32, i32]
+        L.csr_encode_workspace_bytes.restype = i64
+        L.csr_reconstruct.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp]
+        L.csr_reconstruct.restype = i32
+        L.csr_reconstruct_ex.argtypes = [ctypes.POINTER(csr_reconstruct_params_t)]
+        L.csr_reconstruct_ex.restype = i32
+        L.csr_device_status.argtypes = [vp]
+        L.csr_device_status.restype = i32
+        L.csr_release_workspace.argtypes = []
+        L.csr_release_workspace.restype = i32
+        L.csr_last_error_string.argtypes = []
+        L.csr_last_error_string.restype = ctypes.c_char_p
+        L.csr_version.argtypes = []
+        L.csr_version.restype = i32
+        _lib = L
+    return _lib
+
+
+def csr_last_error_string() -> str:
+    return lib().csr_last_error_string().decode()
+
+
+def csr_version() -> int:
+    return int(lib().csr_version())
+
+
+def _check(rc: int) -> None:
+    if rc != CSR_OK:
+        raise CsrError(rc, csr_last_error_string())
+
+
+_TORCH_DTYPE = {torch.float32: CSR_DTYPE_F32, torch.bfloat16: CSR_DTYPE_BF16, torch.float16: CSR_DTYPE_F16}
+
+
+def _stream_ptr(t: torch.Tensor) -> int:
+    return int(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+def csr_encode_workspace_bytes(mode: int, d: int, N: int) -> int:
+    n = int(lib().csr_encode_workspace_bytes(mode, d, N))
+    if n < 0:
+        raise CsrError(n, csr_last_error_string())
+    return n
+
+
+def _encode_params(D, X, s, out_idx, out_coef, mode, stream, workspace) -> csr_encode_params_t:
+    p = csr_encode_params_t()
+    p.struct_size = ctypes.sizeof(csr_encode_params_t)
+    p.mode = mode
+    p.D = D.data_ptr()
+    p.X = X.data_ptr()
+    p.x_dtype = _TORCH_DTYPE[X.dtype]
+    p.coef_dtype = _TORCH_DTYPE[out_coef.dtype]
+    p.M = X.shape[0]
+    p.d = D.shape[1]
+    p.N = D.shape[0]
+    p.s = s
+    p.out_idx = out_idx.data_ptr()
+    p.out_coef = out_coef.data_ptr()
+    p.stream = stream
+    if workspace is not None:
+        p.workspace = workspace.data_ptr()
+        p.workspace_bytes = workspace.numel() * workspace.element_size()
+    return p
+
+
+def csr_encode_ex(D: torch.Tensor, X: torch.Tensor, s: int, *, mode: int = CSR_MODE_BF16_FAST,
+                  coef_dtype: torch.dtype = torch.float16, out_idx: Optional[torch.Tensor] = None,
+                  out_coef: Optional[torch.Tensor] = None,
+                  workspace: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """csr_encode_ex on CUDA tensors: D [N][d] fp32, X [M][d] fp32 or bf16.
+    Returns (idx [M][s] uint16, coef [M][s] coef_dtype); runs on torch's current stream."""
+    assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.is_contiguous()
+    assert D.dtype == torch.float32 and X.dim() == 2 and D.dim() == 2 and X.shape[1] == D.shape[1]
+    M = X.shape[0]
+    if out_idx is None:
+        out_idx = torch.empty((M, s), dtype=torch.uint16, device=X.device)
+    if out_coef is None:
+        out_coef = torch.empty((M, s), dtype=coef_dtype, device=X.device)
+    p = _encode_params(D, X, s, out_idx, out_coef, mode, _stream_ptr(X), workspace)
+    with torch.cuda.device(X.device):
+        _check(lib().csr_encode_ex(ctypes.byref(p)))
+    return out_idx, out_coef
+
+
+def csr_encode(D: torch.Tensor, X: torch.Tensor, s: int, out_idx: Optional[torch.Tensor] = None,
+               out_coef: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """The 8-argument csr_encode: bf16 X, fp16 coefficients, fast mode, legacy default stream."""
+    assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.is_contiguous()
+    assert D.dtype == torch.float32 and X.dtype == torch.bfloat16
+    M, d = X.shape
+    N = D.shape[0]
+    if out_idx is None:
+        out_idx = torch.empty((M, s), dtype=torch.uint16, device=X.device)
+    if out_coef is None:
+        out_coef = torch.empty((M, s), dtype=torch.float16, device=X.device)
+    with torch.cuda.device(X.device):
+        _check(lib().csr_encode(D.data_ptr(), X.data_ptr(), M, d, N, s, out_idx.data_ptr(), out_coef.data_ptr()))
+    return out_idx, out_coef
+
+
+def csr_encode_host(D: torch.Tensor, X_host: torch.Tensor, s: int, out_idx_host: torch.Tensor,
+                    out_coef_host: torch.Tensor, *, mode: int = CSR_MODE_BF16_FAST) -> None:
+    """csr_encode_host: D on the device; X and the outputs are host tensors (pinned for speed).
+    Returns after the codes have arrived in the host tensors."""
+    assert D.is_cuda and not X_host.is_cuda and not out_idx_host.is_cuda and not out_coef_host.is_cuda
+    assert X_host.is_contiguous() and out_idx_host.is_contiguous() and out_coef_host.is_contiguous()
+    assert out_idx_host.dtype == torch.uint16 and tuple(out_idx_host.shape) == (X_host.shape[0], s)
+    p = _encode_params(D, X_host, s, out_idx_host, out_coef_host, mode, None, None)
+    with torch.cuda.device(D.device):
+        _check(lib().csr_encode_host(ctypes.byref(p)))
+
+
+def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *,
+                       out_dtype: torch.dtype = torch.bfloat16,
+                       X_hat: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """csr_reconstruct_ex on CUDA tensors; returns X_hat [M][d]."""
+    assert D.is_cuda and idx.is_cuda and coef.is_cuda
+    assert D.is_contiguous() and idx.is_contiguous() and coef.is_contiguous()
+    assert D.dtype == torch.float32 and idx.dtype == torch.uint16 and idx.shape == coef.shape
+    M, s = idx.shape
+    N, d = D.shape
+    if X_hat is None:
+        X_hat = torch.empty((M, d), dtype=out_dtype, device=D.device)
+    p = csr_reconstruct_params_t()
+    p.struct_size = ctypes.sizeof(csr_reconstruct_params_t)
+    p.D = D.data_ptr()
+    p.idx = idx.data_ptr()
+    p.coef = coef.data_ptr()
+    p.coef_dtype = _TORCH_DTYPE[coef.dtype]
+    p.out_dtype = _TORCH_DTYPE[X_hat.dtype]
+    p.M, p.d, p.N, p.s = M, d, N, s
+    p.X_hat = X_hat.data_ptr()
+    p.stream = _stream_ptr(D)
+    with torch.cuda.device(D.device):
+        _check(lib().csr_reconstruct_ex(ctypes.byref(p)))
+    return X_hat
+
+
+def csr_reconstruct(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor,
+                    X_hat: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The 8-argument csr_reconstruct: fp16 coefficients in, bf16 X_hat out, legacy default stream."""
+    assert D.is_cuda and D.dtype == torch.float32 and idx.dtype == torch.uint16 and coef.dtype == torch.float16
+    M, s = idx.shape
+    N, d = D.shape
+    if X_hat is None:
+        X_hat = torch.empty((M, d), dtype=torch.bfloat16, device=D.device)
+    with torch.cuda.device(D.device):
+        _check(lib().csr_reconstruct(D.data_ptr(), idx.data_ptr(), coef.data_ptr(), M, d, N, s, X_hat.data_ptr()))
+    return X_hat
+
+
+def csr_device_status(device=None) -> int:
+    """Synchronises torch's current stream and returns CSR_OK or CSR_ERR_TIMEOUT."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        return int(lib().csr_device_status(int(torch.cuda.current_stream(dev).cuda_stream)))
+
+
+def csr_release_workspace() -> None:
+    _check(lib().csr_release_workspace())

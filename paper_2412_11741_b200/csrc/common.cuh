@@ -1,0 +1,54 @@
+// Shared declarations of the libcsr translation units (host-side plumbing only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "csr.h"
+
+namespace csr {
+
+// Records the calling thread's last error message and returns `code`.
+int fail(int code, const char* fmt, ...);
+
+// Device status word written by kernels whose bounded waits expire.
+constexpr uint32_t kStatusTimeout = 1u;
+
+struct EncodeArgs {
+    const float* D;
+    const void* X;
+    int x_dtype;
+    int coef_dtype;
+    int64_t M;
+    int d, N, s;
+    uint16_t* out_idx;
+    void* out_coef;
+    cudaStream_t stream;
+};
+
+// fp32-operand matching pursuit with fp64 re-scoring of unresolved picks.
+int launch_encode_exact(const EncodeArgs& a);
+
+// tcgen05 bf16 matching pursuit.  `workspace` holds the bf16 copy of D (N*d*2 bytes,
+// 1024-byte aligned); `status` is a device word that receives kStatusTimeout.
+int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status);
+size_t encode_fast_workspace_bytes(int d, int N);
+
+struct ReconstructArgs {
+    const float* D;
+    const uint16_t* idx;
+    const void* coef;
+    int coef_dtype;
+    int out_dtype;
+    int64_t M;
+    int d, N, s;
+    void* X_hat;
+    cudaStream_t stream;
+};
+int launch_reconstruct(const ReconstructArgs& a);
+
+int sm_count();
+
+}  // namespace csr

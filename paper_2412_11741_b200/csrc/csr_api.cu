@@ -1,0 +1,370 @@
+// C boundary of libcsr: argument checks, workspace management, stream plumbing.
+// Every computation is done by the kernels in the other translation units.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace csr {
+
+static thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kStatusBytes = 256;
+
+// Library-owned, grow-only device buffers of one device.
+struct DeviceBuffers {
+    void* work = nullptr;      // [status word | encoder scratch]
+    size_t work_bytes = 0;
+    void* stage_x[2] = {nullptr, nullptr};   // host-entry staging: X chunks
+    void* stage_idx[2] = {nullptr, nullptr};
+    void* stage_coef[2] = {nullptr, nullptr};
+    size_t stage_rows = 0;
+    size_t stage_x_bytes = 0, stage_code_bytes = 0;
+    cudaStream_t copy_streams[2] = {nullptr, nullptr};
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
+};
+DeviceBuffers g_dev[kMaxDevices];
+std::mutex g_mu;
+
+int current_device(int* dev) {
+    cudaError_t e = cudaGetDevice(dev);
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (*dev < 0 || *dev >= kMaxDevices) return fail(CSR_ERR_UNSUPPORTED, "device ordinal %d not supported", *dev);
+    return CSR_OK;
+}
+
+// Returns the library's work buffer (status word first), grown to hold `scratch` bytes.
+int ensure_work(size_t scratch, void** base) {
+    int dev;
+    if (int rc = current_device(&dev)) return rc;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceBuffers& b = g_dev[dev];
+    const size_t need = kStatusBytes + 1024 + scratch;
+    if (b.work_bytes < need) {
+        if (b.work) {
+            cudaDeviceSynchronize();
+            cudaFree(b.work);
+            b.work = nullptr;
+            b.work_bytes = 0;
+        }
+        cudaError_t e = cudaMalloc(&b.work, need);
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMalloc(%zu): %s", need, cudaGetErrorString(e));
+        e = cudaMemset(b.work, 0, kStatusBytes);
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemset: %s", cudaGetErrorString(e));
+        b.work_bytes = need;
+    }
+    *base = b.work;
+    return CSR_OK;
+}
+
+inline void* align_up(void* p, size_t a) {
+    return reinterpret_cast<void*>((reinterpret_cast<uintptr_t>(p) + a - 1) / a * a);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_dims(int d, int N, int s, int64_t M) {
+    if (d != 64 && d != 128) return fail(CSR_ERR_UNSUPPORTED, "d = %d: only 64 and 128 are supported", d);
+    if (N < 1 || N > 65536) return fail(CSR_ERR_INVALID_ARG, "N = %d outside [1, 65536]", N);
+    if (s < 1 || s > 64) return fail(CSR_ERR_INVALID_ARG, "s = %d outside [1, 64]", s);
+    if (M < 0) return fail(CSR_ERR_INVALID_ARG, "M = %lld is negative", (long long)M);
+    return CSR_OK;
+}
+
+int check_encode(const csr_encode_params_t* p, bool host_io) {
+    if (!p) return fail(CSR_ERR_INVALID_ARG, "params is NULL");
+    if (p->struct_size != sizeof(csr_encode_params_t))
+        return fail(CSR_ERR_INVALID_ARG, "struct_size %u != %zu", p->struct_size, sizeof(csr_encode_params_t));
+    if (p->mode != CSR_MODE_FP32_EXACT && p->mode != CSR_MODE_BF16_FAST)
+        return fail(CSR_ERR_INVALID_ARG, "unknown mode %d", p->mode);
+    if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
+    if (p->x_dtype != CSR_DTYPE_F32 && p->x_dtype != CSR_DTYPE_BF16)
+        return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32 or BF16");
+    if (p->coef_dtype != CSR_DTYPE_F32 && p->coef_dtype != CSR_DTYPE_F16)
+        return fail(CSR_ERR_INVALID_ARG, "coef_dtype must be F32 or F16");
+    if (p->mode == CSR_MODE_BF16_FAST && (p->N % 128) != 0)
+        return fail(CSR_ERR_UNSUPPORTED, "fast mode needs N %% 128 == 0 (N = %d); pad D with zero atoms", p->N);
+    if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
+    if (p->M > 0 && (!p->X || !p->out_idx || !p->out_coef))
+        return fail(CSR_ERR_INVALID_ARG, "X, out_idx or out_coef is NULL");
+    if (!aligned16(p->D) || (!host_io && (!aligned16(p->X) || !aligned16(p->out_idx) || !aligned16(p->out_coef))))
+        return fail(CSR_ERR_ALIGNMENT, "D, X, out_idx and out_coef must be 16-byte aligned");
+    if (p->workspace && !aligned16(p->workspace)) return fail(CSR_ERR_ALIGNMENT, "workspace must be 16-byte aligned");
+    return CSR_OK;
+}
+
+int64_t workspace_bytes(int mode, int d, int N) {
+    if (mode == CSR_MODE_FP32_EXACT) return 0;
+    return (int64_t)(kStatusBytes + 1024 + encode_fast_workspace_bytes(d, N));
+}
+
+// Runs one encode on device pointers.
+int encode_device(const csr_encode_params_t* p) {
+    if (p->M == 0) return CSR_OK;
+    EncodeArgs a;
+    a.D = static_cast<const float*>(p->D);
+    a.X = p->X;
+    a.x_dtype = p->x_dtype;
+    a.coef_dtype = p->coef_dtype;
+    a.M = p->M;
+    a.d = p->d;
+    a.N = p->N;
+    a.s = p->s;
+    a.out_idx = p->out_idx;
+    a.out_coef = p->out_coef;
+    a.stream = static_cast<cudaStream_t>(p->stream);
+    if (p->mode == CSR_MODE_FP32_EXACT) return launch_encode_exact(a);
+
+    void* base = nullptr;
+    if (p->workspace) {
+        const int64_t need = workspace_bytes(p->mode, p->d, p->N);
+        if ((int64_t)p->workspace_bytes < need)
+            return fail(CSR_ERR_WORKSPACE, "workspace of %zu bytes given, %lld needed", p->workspace_bytes,
+                        (long long)need);
+        base = p->workspace;
+        cudaError_t e = cudaMemsetAsync(base, 0, kStatusBytes, a.stream);
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    } else {
+        if (int rc = ensure_work(encode_fast_workspace_bytes(p->d, p->N), &base)) return rc;
+    }
+    uint32_t* status = static_cast<uint32_t*>(base);
+    void* scratch = align_up(static_cast<char*>(base) + kStatusBytes, 1024);
+    return launch_encode_fast(a, scratch, status);
+}
+
+}  // namespace
+}  // namespace csr
+
+using namespace csr;
+
+extern "C" {
+
+int csr_version(void) { return CSR_VERSION; }
+
+const char* csr_last_error_string(void) { return g_err; }
+
+int64_t csr_encode_workspace_bytes(int mode, int d, int N) {
+    if (mode != CSR_MODE_FP32_EXACT && mode != CSR_MODE_BF16_FAST)
+        return fail(CSR_ERR_INVALID_ARG, "unknown mode %d", mode);
+    if (int rc = check_dims(d, N, 1, 0)) return rc;
+    return workspace_bytes(mode, d, N);
+}
+
+int csr_encode_ex(const csr_encode_params_t* p) {
+    if (int rc = check_encode(p, false)) return rc;
+    return encode_device(p);
+}
+
+int csr_encode(const void* D, const void* X, int64_t M, int d, int N, int s, uint16_t* out_idx, void* out_coef) {
+    csr_encode_params_t p;
+    memset(&p, 0, sizeof(p));
+    p.struct_size = sizeof(p);
+    p.mode = CSR_MODE_BF16_FAST;
+    p.D = D;
+    p.X = X;
+    p.x_dtype = CSR_DTYPE_BF16;
+    p.coef_dtype = CSR_DTYPE_F16;
+    p.M = M;
+    p.d = d;
+    p.N = N;
+    p.s = s;
+    p.out_idx = out_idx;
+    p.out_coef = out_coef;
+    return csr_encode_ex(&p);
+}
+
+int csr_reconstruct_ex(const csr_reconstruct_params_t* p) {
+    if (!p) return fail(CSR_ERR_INVALID_ARG, "params is NULL");
+    if (p->struct_size != sizeof(csr_reconstruct_params_t))
+        return fail(CSR_ERR_INVALID_ARG, "struct_size %u != %zu", p->struct_size, sizeof(csr_reconstruct_params_t));
+    if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
+    if (p->coef_dtype != CSR_DTYPE_F32 && p->coef_dtype != CSR_DTYPE_F16)
+        return fail(CSR_ERR_INVALID_ARG, "coef_dtype must be F32 or F16");
+    if (p->out_dtype != CSR_DTYPE_F32 && p->out_dtype != CSR_DTYPE_BF16)
+        return fail(CSR_ERR_INVALID_ARG, "out_dtype must be F32 or BF16");
+    if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
+    if (p->M > 0 && (!p->idx || !p->coef || !p->X_hat)) return fail(CSR_ERR_INVALID_ARG, "idx, coef or X_hat is NULL");
+    if (!aligned16(p->D) || !aligned16(p->idx) || !aligned16(p->coef) || !aligned16(p->X_hat))
+        return fail(CSR_ERR_ALIGNMENT, "D, idx, coef and X_hat must be 16-byte aligned");
+    ReconstructArgs a;
+    a.D = static_cast<const float*>(p->D);
+    a.idx = p->idx;
+    a.coef = p->coef;
+    a.coef_dtype = p->coef_dtype;
+    a.out_dtype = p->out_dtype;
+    a.M = p->M;
+    a.d = p->d;
+    a.N = p->N;
+    a.s = p->s;
+    a.X_hat = p->X_hat;
+    a.stream = static_cast<cudaStream_t>(p->stream);
+    return launch_reconstruct(a);
+}
+
+int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_t M, int d, int N, int s,
+                    void* X_hat) {
+    csr_reconstruct_params_t p;
+    memset(&p, 0, sizeof(p));
+    p.struct_size = sizeof(p);
+    p.D = D;
+    p.idx = idx;
+    p.coef = coef;
+    p.coef_dtype = CSR_DTYPE_F16;
+    p.out_dtype = CSR_DTYPE_BF16;
+    p.M = M;
+    p.d = d;
+    p.N = N;
+    p.s = s;
+    p.X_hat = X_hat;
+    return csr_reconstruct_ex(&p);
+}
+
+int csr_encode_host(const csr_encode_params_t* p) {
+    if (int rc = check_encode(p, true)) return rc;
+    if (p->M == 0) return CSR_OK;
+    int dev;
+    if (int rc = current_device(&dev)) return rc;
+    const size_t xb = (p->x_dtype == CSR_DTYPE_BF16 ? 2 : 4) * (size_t)p->d;
+    const size_t cb = (p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4) * (size_t)p->s;
+    const size_t ib = 2 * (size_t)p->s;
+    // chunk rows: a multiple of 256, about 1/8 of the job, at least 32768 rows
+    int64_t chunk = ((p->M / 8 + 255) / 256) * 256;
+    if (chunk < 32768) chunk = 32768;
+    if (chunk > p->M) chunk = ((p->M + 255) / 256) * 256;
+    DeviceBuffers& b = g_dev[dev];
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        cudaError_t e = cudaSuccess;
+        if (!b.copy_streams[0]) {
+            for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+                e = cudaStreamCreateWithFlags(&b.copy_streams[i], cudaStreamNonBlocking);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b.ev_in[i], cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b.ev_done[i], cudaEventDisableTiming);
+            }
+            if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "stream/event creation: %s", cudaGetErrorString(e));
+        }
+        const size_t need_x = (size_t)chunk * xb, need_c = (size_t)chunk * (cb > ib ? cb : ib);
+        if (b.stage_x_bytes < need_x || b.stage_code_bytes < need_c) {
+            cudaDeviceSynchronize();
+            for (int i = 0; i < 2; ++i) {
+                cudaFree(b.stage_x[i]);
+                cudaFree(b.stage_idx[i]);
+                cudaFree(b.stage_coef[i]);
+                b.stage_x[i] = b.stage_idx[i] = b.stage_coef[i] = nullptr;
+            }
+            b.stage_x_bytes = b.stage_code_bytes = 0;
+            for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+                e = cudaMalloc(&b.stage_x[i], need_x);
+                if (e == cudaSuccess) e = cudaMalloc(&b.stage_idx[i], need_c);
+                if (e == cudaSuccess) e = cudaMalloc(&b.stage_coef[i], need_c);
+            }
+            if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "staging cudaMalloc: %s", cudaGetErrorString(e));
+            b.stage_x_bytes = need_x;
+            b.stage_code_bytes = need_c;
+        }
+    }
+    // Chunk j uses slot j % 2 with its own stream for copy-in, encode and copy-out, so the
+    // copies of one chunk overlap the kernels of the other.
+    const int64_t n_chunks = (p->M + chunk - 1) / chunk;
+    int rc = CSR_OK;
+    for (int64_t j = 0; j < n_chunks && rc == CSR_OK; ++j) {
+        const int slot = (int)(j & 1);
+        const int64_t r0 = j * chunk;
+        const int64_t rows = (p->M - r0 < chunk) ? (p->M - r0) : chunk;
+        cudaStream_t st = b.copy_streams[slot];
+        cudaError_t e = cudaMemcpyAsync(b.stage_x[slot], static_cast<const char*>(p->X) + (size_t)r0 * xb,
+                                        (size_t)rows * xb, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) {
+            rc = fail(CSR_ERR_CUDA, "H2D copy: %s", cudaGetErrorString(e));
+            break;
+        }
+        csr_encode_params_t q = *p;
+        q.X = b.stage_x[slot];
+        q.M = rows;
+        q.out_idx = static_cast<uint16_t*>(b.stage_idx[slot]);
+        q.out_coef = b.stage_coef[slot];
+        q.stream = st;
+        q.workspace = nullptr;
+        q.workspace_bytes = 0;
+        rc = encode_device(&q);
+        if (rc != CSR_OK) break;
+        e = cudaMemcpyAsync(reinterpret_cast<char*>(p->out_idx) + (size_t)r0 * ib, b.stage_idx[slot],
+                            (size_t)rows * ib, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(static_cast<char*>(p->out_coef) + (size_t)r0 * cb, b.stage_coef[slot],
+                                (size_t)rows * cb, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) rc = fail(CSR_ERR_CUDA, "D2H copy: %s", cudaGetErrorString(e));
+    }
+    for (int i = 0; i < 2; ++i) {
+        cudaError_t e = cudaStreamSynchronize(b.copy_streams[i]);
+        if (e != cudaSuccess && rc == CSR_OK) rc = fail(CSR_ERR_CUDA, "stream sync: %s", cudaGetErrorString(e));
+    }
+    return rc;
+}
+
+int csr_device_status(void* stream) {
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "stream sync: %s", cudaGetErrorString(e));
+    int dev;
+    if (int rc = current_device(&dev)) return rc;
+    void* work;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        work = g_dev[dev].work;
+    }
+    if (!work) return CSR_OK;
+    uint32_t st = 0;
+    e = cudaMemcpy(&st, work, sizeof(st), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "status read: %s", cudaGetErrorString(e));
+    if (st != 0) {
+        cudaMemset(work, 0, kStatusBytes);
+        return fail(CSR_ERR_TIMEOUT, "a device-side wait expired (status word 0x%x)", st);
+    }
+    return CSR_OK;
+}
+
+int csr_release_workspace(void) {
+    int dev;
+    if (int rc = current_device(&dev)) return rc;
+    cudaDeviceSynchronize();
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceBuffers& b = g_dev[dev];
+    cudaFree(b.work);
+    b.work = nullptr;
+    b.work_bytes = 0;
+    for (int i = 0; i < 2; ++i) {
+        cudaFree(b.stage_x[i]);
+        cudaFree(b.stage_idx[i]);
+        cudaFree(b.stage_coef[i]);
+        b.stage_x[i] = b.stage_idx[i] = b.stage_coef[i] = nullptr;
+    }
+    b.stage_x_bytes = b.stage_code_bytes = 0;
+    return CSR_OK;
+}
+
+}  // extern "C"

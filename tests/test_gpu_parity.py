@@ -1,0 +1,292 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs (paper Eq. 2-4 for the encoder, Eq. 12 for the de-sparse)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import csr_oracle as orc
+from paper_2412_11741_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _np_idx(t):
+    """uint16 tensor -> numpy (through an int16 view: few torch ops take uint16)."""
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def _take_rows(t, rows):
+    return t.view(torch.int16)[rows].view(torch.uint16) if t.dtype == torch.uint16 else t[rows]
+
+
+@pytest.fixture(scope="module")
+def csr():
+    from paper_2412_11741_b200 import build
+    build.build()
+    import paper_2412_11741_b200 as pkg
+    return pkg
+
+
+def _dev_x(w, X=None):
+    X = w.X if X is None else X
+    t = torch.from_numpy(np.ascontiguousarray(X)).to(DEV)
+    return t.to(torch.bfloat16) if w.x_dtype == "bf16" else t
+
+
+def _encode(csr, w, X, mode, coef_dtype=torch.float32):
+    D = torch.from_numpy(w.D).to(DEV)
+    idx, coef = csr.csr_encode_ex(D, _dev_x(w, X), w.s, mode=mode, coef_dtype=coef_dtype)
+    assert csr.csr_device_status() == csr.CSR_OK
+    return _np_idx(idx), coef.float().cpu().numpy()
+
+
+# ---------------------------------------------------------------------------------------
+# exact mode
+# ---------------------------------------------------------------------------------------
+
+def test_exact_tiny_config_all_rows(csr):
+    w = wl.tiny()
+    idx, coef = _encode(csr, w, w.X, csr.CSR_MODE_FP32_EXACT)
+    rep = parity.compare_exact(w.D, w.X, w.s, idx, coef)
+    assert rep.ok, rep.detail
+    assert rep.unexplained_rows == 0 and rep.coef_max_rel < 1e-4
+    # the stored fp16 coefficient is the round-to-nearest-even of the fp32 one
+    idx16, coef16 = _encode(csr, w, w.X, csr.CSR_MODE_FP32_EXACT, torch.float16)
+    assert np.array_equal(idx16, idx)
+    assert np.array_equal(coef16, coef.astype(np.float16).astype(np.float32))
+    # exactly sparse rows: same picks as the oracle, first pick inside the true support
+    lo, hi = w.meta["sparse_rows"]
+    assert all(idx[m, 0] in w.meta["support"][m - lo] for m in range(lo, hi))
+
+
+@pytest.mark.parametrize("make,rows", [
+    (lambda: wl.llama2_layer(tokens=64), 2048),
+    (lambda: wl.gqa_long(tokens=32), 1536),
+    (lambda: wl.sparsity_sweep(32, tokens=64, N=8192), 768),
+    (lambda: wl.dict_sweep(2048, M=4096), 2048),
+    (lambda: wl.dict_sweep(4096, d=64, M=4096), 2048),
+])
+def test_exact_configs_subsample(csr, make, rows):
+    w = make()
+    sel = wl.stratified_rows(w.M, rows, seed=7)
+    X = w.X[sel]
+    idx, coef = _encode(csr, w, X, csr.CSR_MODE_FP32_EXACT)
+    rep = parity.compare_exact(w.D, X, w.s, idx, coef)
+    assert rep.ok, rep.detail
+
+
+@pytest.mark.parametrize("M", [0, 1, 2, 63, 64, 65, 127, 129, 200])
+def test_exact_ragged_rows(csr, M):
+    rng = np.random.default_rng(M)
+    D = wl.normalise_rows(rng.standard_normal((272, 128)).astype(np.float32))   # N not a tile multiple
+    X = rng.standard_normal((M, 128)).astype(np.float32)
+    w = wl.Workload("ragged", D, X, 5, "f32")
+    if M == 0:
+        Dd = torch.from_numpy(D).to(DEV)
+        i, c = csr.csr_encode_ex(Dd, torch.empty((0, 128), device=DEV), 5, mode=csr.CSR_MODE_FP32_EXACT,
+                                 coef_dtype=torch.float32)
+        assert i.shape == (0, 5)
+        return
+    idx, coef = _encode(csr, w, X, csr.CSR_MODE_FP32_EXACT)
+    rep = parity.compare_exact(D, X, 5, idx, coef)
+    assert rep.ok, rep.detail
+
+
+@pytest.mark.parametrize("N,s", [(1, 3), (16, 1), (130, 7), (1024, 64)])
+def test_exact_small_dictionaries(csr, N, s):
+    rng = np.random.default_rng(N * 100 + s)
+    D = wl.normalise_rows(rng.standard_normal((N, 64)).astype(np.float32))
+    X = rng.standard_normal((150, 64)).astype(np.float32)
+    idx, coef = _encode(csr, wl.Workload("small", D, X, s, "f32"), X, csr.CSR_MODE_FP32_EXACT)
+    rep = parity.compare_exact(D, X, s, idx, coef)
+    assert rep.ok, rep.detail
+
+
+def test_exact_degenerate_inputs(csr):
+    """Zero vectors, exact ties, an input that is itself an atom, a duplicated atom."""
+    rng = np.random.default_rng(5)
+    D = wl.normalise_rows(rng.standard_normal((256, 128)).astype(np.float32))
+    D[200] = D[3]                       # duplicate atom: the lower index must win
+    D[17] = -D[9]                       # sign-flipped duplicate
+    X = rng.standard_normal((64, 128)).astype(np.float32)
+    X[0] = 0.0
+    X[1] = D[42] * np.float32(2.0)      # exactly one atom: residual becomes (nearly) zero
+    X[2] = D[3] * np.float32(-1.5)
+    X[3] = D[9]
+    idx, coef = _encode(csr, wl.Workload("deg", D, X, 6, "f32"), X, csr.CSR_MODE_FP32_EXACT)
+    res = orc.mp_encode(D, X, 6)
+    assert idx[0].tolist() == [0] * 6 and np.all(coef[0] == 0)
+    assert idx[1, 0] == 42 and idx[2, 0] == 3 and idx[3, 0] == 9
+    assert np.array_equal(idx[:, 0], res.idx[:, 0])
+    rep = parity.compare_exact(D, X, 6, idx, coef, res)
+    assert rep.ok, rep.detail
+
+
+def test_exact_identity_dictionary_recovers_exactly(csr):
+    rng = np.random.default_rng(8)
+    D = np.eye(64, dtype=np.float32)
+    X = rng.standard_normal((130, 64)).astype(np.float32)
+    idx, coef = _encode(csr, wl.Workload("eye", D, X, 64, "f32"), X, csr.CSR_MODE_FP32_EXACT)
+    order = np.argsort(-np.abs(X), axis=1, kind="stable")
+    assert np.array_equal(idx, order)
+    assert np.array_equal(coef, np.take_along_axis(X, order, 1))
+
+
+# ---------------------------------------------------------------------------------------
+# fast mode
+# ---------------------------------------------------------------------------------------
+
+def test_fast_tiny_config(csr):
+    w = wl.tiny()
+    idx, coef = _encode(csr, w, w.X, csr.CSR_MODE_BF16_FAST)
+    rep = parity.compare_fast(w.D, w.X, w.s, idx, coef)
+    assert rep.ok, rep.detail
+    assert rep.same_rows > 0.8 * rep.rows
+
+
+@pytest.mark.parametrize("make,rows", [
+    (lambda: wl.llama2_layer(tokens=64), 2048),
+    (lambda: wl.gqa_long(tokens=32), 1536),
+    (lambda: wl.sparsity_sweep(4, tokens=64, N=8192), 1024),
+    (lambda: wl.sparsity_sweep(32, tokens=64, N=8192), 768),
+    (lambda: wl.dict_sweep(2048, M=4096), 2048),
+    (lambda: wl.dict_sweep(16384, M=4096), 768),
+    (lambda: wl.dict_sweep(4096, d=64, M=4096), 2048),
+])
+def test_fast_configs_subsample(csr, make, rows):
+    w = make()
+    sel = wl.stratified_rows(w.M, rows, seed=11)
+    X = w.X[sel]
+    idx, coef = _encode(csr, w, X, csr.CSR_MODE_BF16_FAST)
+    rep = parity.compare_fast(w.D, X, w.s, idx, coef)
+    assert rep.ok, rep.detail
+
+
+@pytest.mark.parametrize("M", [1, 127, 128, 129, 255, 256, 257, 300 * 256 + 5])
+def test_fast_ragged_rows_match_full_tiles(csr, M):
+    """Rows of a ragged tail get the same codes as the same rows inside full tiles, and
+    rows past M are not written."""
+    rng = np.random.default_rng(3)
+    D = wl.normalise_rows(rng.standard_normal((512, 128)).astype(np.float32))
+    Mfull = ((M + 255) // 256 + 1) * 256
+    X = wl.round_to_bf16(rng.standard_normal((Mfull, 128)).astype(np.float32))
+    Dd = torch.from_numpy(D).to(DEV)
+    Xd = torch.from_numpy(X).to(DEV).to(torch.bfloat16)
+    s = 8
+    i_full, c_full = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float32)
+    out_i = torch.full((Mfull, s), -1, dtype=torch.int16, device=DEV).view(torch.uint16)
+    out_c = torch.full((Mfull, s), -7.0, dtype=torch.float32, device=DEV)
+    csr.csr_encode_ex(Dd, Xd[:M].contiguous(), s, coef_dtype=torch.float32, out_idx=out_i[:M], out_coef=out_c[:M])
+    assert csr.csr_device_status() == csr.CSR_OK
+    assert np.array_equal(_np_idx(out_i)[:M], _np_idx(i_full)[:M])
+    assert torch.equal(out_c[:M].cpu(), c_full[:M].cpu())
+    assert np.all(_np_idx(out_i)[M:] == 0xFFFF) and bool((out_c[M:] == -7.0).all())
+    if M <= 300:
+        rep = parity.compare_fast(D, X[:M], s, _np_idx(out_i)[:M], out_c[:M].cpu().numpy())
+        assert rep.mean_ratio < 1.05 and rep.ratio_max < 1.5, rep
+
+
+def test_fast_fp32_input_and_odd_s(csr):
+    rng = np.random.default_rng(13)
+    D = wl.normalise_rows(rng.standard_normal((1024, 128)).astype(np.float32))
+    X = rng.standard_normal((1000, 128)).astype(np.float32)
+    for s in (1, 3, 11):
+        w = wl.Workload("f32in", D, X, s, "f32")
+        idx, coef = _encode(csr, w, X, csr.CSR_MODE_BF16_FAST)
+        rep = parity.compare_fast(D, X, s, idx, coef)
+        assert rep.ok, rep.detail
+        idx16, coef16 = _encode(csr, w, X, csr.CSR_MODE_BF16_FAST, torch.float16)
+        assert np.array_equal(idx16, idx)
+        assert np.array_equal(coef16, coef.astype(np.float16).astype(np.float32))
+
+
+def test_fast_zero_rows_and_eight_arg_form(csr):
+    w = wl.llama2_layer(tokens=8, N=1024)
+    X = w.X.copy()
+    X[5] = 0.0
+    D = torch.from_numpy(w.D).to(DEV)
+    Xd = torch.from_numpy(X).to(DEV).to(torch.bfloat16)
+    idx, coef = csr.csr_encode(D, Xd, w.s)
+    torch.cuda.synchronize()
+    assert csr.csr_device_status() == csr.CSR_OK
+    assert idx.dtype == torch.uint16 and coef.dtype == torch.float16
+    assert _np_idx(idx)[5].tolist() == [0] * w.s and bool((coef[5] == 0).all())
+    rep = parity.compare_fast(w.D, X, w.s, _np_idx(idx), coef.float().cpu().numpy())
+    assert rep.ok, rep.detail
+    # caller-provided workspace gives the same codes
+    nbytes = csr.csr_encode_workspace_bytes(csr.CSR_MODE_BF16_FAST, 128, 1024)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=DEV)
+    idx2, coef2 = csr.csr_encode_ex(D, Xd, w.s, workspace=ws)
+    assert np.array_equal(_np_idx(idx2), _np_idx(idx)) and torch.equal(coef2.cpu(), coef.cpu())
+    with pytest.raises(csr.CsrError):
+        csr.csr_encode_ex(D, Xd, w.s, workspace=ws[:1024])
+
+
+def test_fast_full_size_llama2_layer_sampled(csr):
+    """Config 2 at full size in the launch configuration the benchmark times; the oracle
+    checks a stratified sample of the outputs."""
+    w = wl.llama2_layer()
+    assert w.M == 262144 and w.N == 4096 and w.s == 8
+    D = torch.from_numpy(w.D).to(DEV)
+    Xd = torch.from_numpy(w.X).to(DEV).to(torch.bfloat16)
+    idx, coef = csr.csr_encode(D, Xd, w.s)
+    assert csr.csr_device_status() == csr.CSR_OK
+    sel = wl.stratified_rows(w.M, 2048, seed=21)
+    st = torch.from_numpy(sel).to(DEV)
+    rep = parity.compare_fast(w.D, w.X[sel], w.s, _np_idx(_take_rows(idx, st)), coef[st].float().cpu().numpy())
+    assert rep.ok, rep.detail
+    # every row got a valid code and the whole tensor reconstructs with the sample's error level
+    assert int(_np_idx(idx).max()) < w.N
+    xh = csr.csr_reconstruct(D, idx, coef)
+    err = ((xh.float() - Xd.float()).norm(dim=1) / Xd.float().norm(dim=1)).mean().item()
+    assert abs(err / rep.mean_err - 1) < 0.02
+
+
+# ---------------------------------------------------------------------------------------
+# de-sparse
+# ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("d,N,s,M", [(128, 1024, 8, 4096), (64, 300, 5, 1001), (128, 65536, 33, 517), (128, 16, 64, 64)])
+def test_reconstruct_matches_oracle(csr, d, N, s, M):
+    rng = np.random.default_rng(d + N + s)
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    idx = rng.integers(0, N, size=(M, s)).astype(np.int32)
+    idx[:, -1] = idx[:, 0]                     # repeated atoms accumulate
+    coef = (rng.standard_normal((M, s)) * 3).astype(np.float32)
+    idx16, coef16 = orc.pack_codes(idx, coef.astype(np.float64))
+    Dd = torch.from_numpy(D).to(DEV)
+    it = torch.from_numpy(idx16).to(DEV)
+    ref32 = orc.reconstruct(D, idx, coef.astype(np.float64))
+    scale = np.abs(coef).sum(1, keepdims=True) + 1e-30
+    out32 = csr.csr_reconstruct_ex(Dd, it, torch.from_numpy(coef).to(DEV), out_dtype=torch.float32).cpu().numpy()
+    assert np.abs(out32 - ref32).max() <= 1e-6 * scale.max()
+    assert np.all(np.abs(out32 - ref32) <= 2e-6 * scale)
+    # stored form: fp16 coefficients in, bf16 out
+    ref16 = orc.reconstruct(D, idx, coef16.astype(np.float64))
+    out16 = csr.csr_reconstruct(Dd, it, torch.from_numpy(coef16).to(DEV)).float().cpu().numpy()
+    assert np.all(np.abs(out16 - ref16) <= 2.0 ** -8 * np.abs(ref16) + 2e-6 * scale)
+
+
+def test_encode_then_reconstruct_round_trip(csr):
+    w = wl.gqa_long(tokens=16)
+    D = torch.from_numpy(w.D).to(DEV)
+    Xd = torch.from_numpy(w.X).to(DEV).to(torch.bfloat16)
+    idx, coef = csr.csr_encode(D, Xd, w.s)
+    xh = csr.csr_reconstruct(D, idx, coef).float().cpu().numpy()
+    ref = orc.reconstruct(w.D, _np_idx(idx).astype(np.int32), coef.float().cpu().numpy().astype(np.float64))
+    assert np.all(np.abs(xh - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-3)
+
+
+def test_host_entry_point(csr):
+    w = wl.llama2_layer(tokens=600, N=1024)         # 38400 rows: more than one chunk
+    D = torch.from_numpy(w.D).to(DEV)
+    Xh = torch.from_numpy(w.X).to(torch.bfloat16).pin_memory()
+    oi = torch.empty((w.M, w.s), dtype=torch.uint16).pin_memory()
+    oc = torch.empty((w.M, w.s), dtype=torch.float16).pin_memory()
+    csr.csr_encode_host(D, Xh, w.s, oi, oc)
+    idx, coef = csr.csr_encode(D, Xh.to(DEV), w.s)
+    torch.cuda.synchronize()
+    assert np.array_equal(_np_idx(oi), _np_idx(idx)) and torch.equal(oc, coef.cpu())
