@@ -144,6 +144,38 @@ int csr_reconstruct_ex(const csr_reconstruct_params_t* p);
 int csr_encode_host(const csr_encode_params_t* p);
 
 /*
+ * Fast encode without any allocation (the paper has no counterpart; this entry point
+ * exists for the deployment reasons below).  Same operation, layouts and results as the
+ * 8-argument csr_encode (bf16 X, fp16 coefficients, fast mode), on the given stream.
+ *
+ * For whom: callers that may not allocate or free device memory while they run, e.g. an
+ * inference server whose device memory is carved up once at start-up, a process whose
+ * free device memory is all owned by a framework's caching allocator, or a
+ * latency-critical loop that cannot afford the implicit device-wide synchronisation an
+ * allocation or a free may cause.  The other encode entry points keep their bf16 copy of
+ * the dictionary in a cudaMalloc'ed buffer (or take a caller workspace); this one keeps
+ * it in a fixed array inside the library image and calls no cudaMalloc, cudaFree or
+ * other allocating routine.
+ *
+ * Limits and rules
+ *   - N * d <= CSR_STATIC_MAX_DICT_ELEMS (8192 atoms of 128 channels, a 2 MiB bf16 copy);
+ *     larger dictionaries are rejected with CSR_ERR_UNSUPPORTED.  Every GPU on which the
+ *     library is loaded holds the array (2 MiB + 2 KiB) until the process exits.
+ *   - The first call on a device looks up the array's device address, once, with that
+ *     device current; make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, and it keeps what the last call wrote.
+ *     Each call rewrites the dictionary copy in full and zeroes its status word before
+ *     use, so stale contents never matter; but two calls whose work overlaps on the GPU
+ *     (different streams, no ordering between them) race on it.  Order them.
+ *   - dev_status: optional device word (4-byte aligned) that is zeroed by the call and
+ *     receives a non-zero value if a device-side wait expired; NULL keeps that word
+ *     inside the array, where csr_device_status does not look.
+ */
+#define CSR_STATIC_MAX_DICT_ELEMS (8192 * 128)
+int csr_encode_static(const void* D, const void* X, int64_t M, int d, int N, int s, uint16_t* out_idx,
+                      void* out_coef, void* stream, uint32_t* dev_status);
+
+/*
  * Synchronises the stream and reports whether a kernel of this library has given up on a
  * bounded wait since the last call of this function on the current device: CSR_OK or
  * CSR_ERR_TIMEOUT (or CSR_ERR_CUDA if the stream itself is in error).

@@ -33,7 +33,7 @@ CSR_MODE_BF16_FAST = 1
 
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
-    "csr_encode_host", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
+    "csr_encode_host", "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
 
@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.csr_encode_ex.restype = i32
         L.csr_encode_host.argtypes = [ctypes.POINTER(csr_encode_params_t)]
         L.csr_encode_host.restype = i32
+        L.csr_encode_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+        L.csr_encode_static.restype = i32
         L.csr_encode_workspace_bytes.argtypes = [i32, i32, i32]
         L.csr_encode_workspace_bytes.restype = i64
         L.csr_reconstruct.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp]
@@ -183,6 +185,21 @@ def csr_encode(D: torch.Tensor, X: torch.Tensor, s: int, out_idx: Optional[torch
     with torch.cuda.device(X.device):
         _check(lib().csr_encode(D.data_ptr(), X.data_ptr(), M, d, N, s, out_idx.data_ptr(), out_coef.data_ptr()))
     return out_idx, out_coef
+
+
+def csr_encode_static(D: torch.Tensor, X: torch.Tensor, s: int, out_idx: torch.Tensor, out_coef: torch.Tensor,
+                      dev_status: Optional[torch.Tensor] = None) -> None:
+    """csr_encode_static: the fast encode for callers that must not allocate.  Outputs are
+    passed in (this wrapper allocates nothing either); runs on torch's current stream."""
+    assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.is_contiguous()
+    assert D.dtype == torch.float32 and X.dtype == torch.bfloat16
+    assert out_idx.dtype == torch.uint16 and out_coef.dtype == torch.float16
+    M, d = X.shape
+    assert tuple(out_idx.shape) == (M, s) and tuple(out_coef.shape) == (M, s)
+    st = None if dev_status is None else dev_status.data_ptr()
+    with torch.cuda.device(X.device):
+        _check(lib().csr_encode_static(D.data_ptr(), X.data_ptr(), M, d, D.shape[0], s, out_idx.data_ptr(),
+                                       out_coef.data_ptr(), _stream_ptr(X), st))
 
 
 def csr_encode_host(D: torch.Tensor, X_host: torch.Tensor, s: int, out_idx_host: torch.Tensor,
