@@ -6,21 +6,34 @@
 //   - the residual tiles live in shared memory as bf16, in the K-major 128-byte-swizzled
 //     layout tcgen05.mma reads (operand A);
 //   - the bf16 copy of the dictionary (a few MB, L2 resident) streams through a ring of
-//     shared-memory stages, 128 atoms per stage, fetched by TMA (operand B); each stage
-//     is used by both row tiles, so every dictionary byte fetched feeds 256 rows;
-//   - tcgen05.mma (M=128, N=128, K=16, bf16 x bf16 -> fp32) writes the 128 x 128
-//     correlations of (row tile, atom tile) into one of four TMEM accumulators
-//     (2 row tiles x 2 buffers x 128 columns = all 512 columns);
+//     shared-memory stages fetched by TMA (operand B).  A stage holds 64 channels of 256
+//     atoms (32 KB); every stage feeds both row tiles, so each dictionary byte fetched
+//     from L2 serves 256 rows;
+//   - tcgen05.mma (M = 128, N = 256, K = 16, bf16 x bf16 -> fp32) writes the 128 x 256
+//     correlations of (row tile, atom tile) into that row tile's TMEM accumulator (2 row
+//     tiles x 256 columns = all 512 columns).  N = 256 per instruction is what keeps the
+//     tensor pipe fed: with N = 128 the operand reads from shared memory (A and B per
+//     instruction) need the whole shared-memory bandwidth and the pipe starves;
 //   - eight epilogue warps (four per row tile, one thread per row) pull the
 //     accumulators out with tcgen05.ld and keep a running arg-max of |correlation| per
-//     row: each value's sign bit is cleared and its low 7 mantissa bits are replaced by
-//     127 - column, so that one 3-input integer max per two values finds both the
-//     largest magnitude and where it was.  The M x N correlations never leave the SM;
-//   - at the end of a sweep every epilogue thread gathers its winning atom (bf16, from
-//     L2), recomputes the signed coefficient as an fp32 dot product with its residual
-//     row, subtracts coefficient * atom, writes the bf16 residual back into the operand
-//     tile and releases the MMA warp for the next iteration;
-//   - codes are collected per thread and written as 16-byte vectors (uint16 index,
+//     row.  The plain-ALU work per correlation value is what bounds the kernel next to
+//     the tensor pipe, so it is cut in two levels: groups of G adjacent atoms are first
+//     reduced to max |value| with 3-input floating-point maxima (absolute value is an
+//     operand modifier, half an instruction per value), then the group maximum's low
+//     mantissa bits are replaced by a group tag (one logic instruction per group) and a
+//     3-input integer max per two groups tracks the largest magnitude and where it was.
+//     The first half of an accumulator is processed while its second half is already on
+//     its way into registers, so the accumulator is handed back to the tensor core after
+//     half of the arithmetic; the two row tiles alternate on the tensor pipe.  The M x N
+//     correlations never leave the SM;
+//   - at the end of a sweep the four warps of a row tile resolve their rows' picks
+//     cooperatively: eight lanes per row gather the G atoms of the row's winning group
+//     (bf16, from L2, 128 contiguous bytes or more per request), recompute the G signed
+//     correlations as fp32 dot products with the residual row, take the largest in
+//     magnitude as (index, coefficient), subtract coefficient * atom and write the bf16
+//     residual back into the operand tile; then the MMA warp is released for the next
+//     iteration;
+//   - codes are collected in shared memory and written as 16-byte vectors (uint16 index,
 //     fp16 or fp32 coefficient).
 //
 // Warp roles: warps 0-3 epilogue of row tile 0, warps 4-7 epilogue of row tile 1 (warp w
@@ -30,14 +43,17 @@
 // its TMEM and exits.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace csr {
 namespace {
 
 constexpr int TILE_M = 128;
-constexpr int TILE_N = 128;
+constexpr int TILE_N = 256;                           // atoms per accumulator / per MMA instruction
 constexpr int UMMA_K = 16;
+constexpr int STAGE_CH = 64;                          // channels per dictionary stage (one 128-byte row)
 constexpr int STAGES = 4;
 constexpr int NT = 320;
 constexpr int PRODUCER_WARP = 8;
@@ -129,6 +145,15 @@ __device__ __forceinline__ void tmem_wait_ld(uint32_t (&v)[32]) {
                  : "memory");
 }
 
+// Orders later uses of the registers after the preceding tcgen05.wait::ld without emitting
+// an instruction (the asynchronous load that fills them is invisible to the compiler).
+__device__ __forceinline__ void reg_fence(uint32_t (&v)[32]) {
+    asm volatile(""
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+                 :
+                 : "memory");
+}
+
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
@@ -155,7 +180,7 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
     return desc;
 }
 
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = 128.
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = 256.
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((TILE_N >> 3) << 17) | ((TILE_M >> 4) << 24);
 
 // ---------------------------------------------------------------------------------------
@@ -163,15 +188,16 @@ constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((TILE_N >>
 // ---------------------------------------------------------------------------------------
 template <int D_>
 struct FastSmem {
-    static constexpr int kTileBytes = TILE_M * D_ * 2;   // one operand tile (A or B)
-    alignas(1024) uint8_t A[2][kTileBytes];
-    alignas(1024) uint8_t B[STAGES][kTileBytes];
+    static constexpr int kATileBytes = TILE_M * D_ * 2;          // residual tile: D_/64 blocks of 128 rows x 128 B
+    static constexpr int kStageBytes = TILE_N * STAGE_CH * 2;    // 256 atoms x 64 channels
+    alignas(1024) uint8_t A[2][kATileBytes];
+    alignas(1024) uint8_t B[STAGES][kStageBytes];
     alignas(16) uint16_t code_idx[2 * TILE_M][CODE_BLOCK];
     alignas(16) float code_coef[2 * TILE_M][CODE_BLOCK];
     uint64_t full_b[STAGES];
     uint64_t empty_b[STAGES];
-    uint64_t acc_full[2][2];
-    uint64_t acc_empty[2][2];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
     uint64_t res_ready[2];
     uint64_t drained;
     uint32_t tmem_base;
@@ -200,8 +226,7 @@ __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, con
     return false;
 }
 
-// Byte offset of 16-byte chunk `chunk` (8 channels) of row `r` inside an operand tile.
-template <int D_>
+// Byte offset of 16-byte chunk `chunk` (8 channels) of row `r` inside a residual tile.
 __device__ __forceinline__ uint32_t swz_off(int r, int chunk) {
     const int khalf = chunk >> 3, cc = chunk & 7;
     return khalf * (TILE_M * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
@@ -214,20 +239,149 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// max over 32 packed keys (|value| with the low 7 bits replaced by 127 - column)
-template <int COL0>
-__device__ __forceinline__ uint32_t chunk_key_max(const uint32_t (&v)[32], uint32_t m) {
-    uint32_t m0 = m, m1 = 0, m2 = 0, m3 = 0;
-#pragma unroll
-    for (int j = 0; j < 32; j += 8) {
-#define CSR_KEY(J) ((v[(J)] & 0x7FFFFF80u) | static_cast<uint32_t>(127 - (COL0 + (J))))
-        m0 = __vimax3_u32(m0, CSR_KEY(j + 0), CSR_KEY(j + 1));
-        m1 = __vimax3_u32(m1, CSR_KEY(j + 2), CSR_KEY(j + 3));
-        m2 = __vimax3_u32(m2, CSR_KEY(j + 4), CSR_KEY(j + 5));
-        m3 = __vimax3_u32(m3, CSR_KEY(j + 6), CSR_KEY(j + 7));
-#undef CSR_KEY
+// (a & mask) | TAG as one logic instruction: the mask is a kernel argument (so it sits in
+// a register) and the tag is the instruction's immediate.
+template <uint32_t TAG>
+__device__ __forceinline__ uint32_t mask_tag(uint32_t a, uint32_t mask) {
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "n"(TAG));
+    return r;
+}
+// max(|a|, |b|, |c|)
+__device__ __forceinline__ float absmax3(float a, float b, float c) {
+    float r;
+    asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// Key of the group of G values starting at v[J] (column COL0 + J of the accumulator):
+// max |value| with its low bits replaced by the tag of the group (higher tag = lower
+// column, so that the lowest column wins ties).
+template <int G, int COL0, int J>
+__device__ __forceinline__ uint32_t group_key(const uint32_t (&v)[32], uint32_t mask) {
+    constexpr uint32_t kTag = static_cast<uint32_t>(TILE_N / G - 1 - (COL0 + J) / G);
+    if constexpr (G == 1) {
+        return mask_tag<kTag>(v[J], mask);                // the mask also clears the sign
+    } else {
+        float gm;
+        if constexpr (G == 2) {
+            gm = fmaxf(fabsf(__uint_as_float(v[J])), fabsf(__uint_as_float(v[J + 1])));
+        } else if constexpr (G == 4) {
+            gm = fmaxf(absmax3(__uint_as_float(v[J]), __uint_as_float(v[J + 1]), __uint_as_float(v[J + 2])),
+                       fabsf(__uint_as_float(v[J + 3])));
+        } else {
+            const float t1 = absmax3(__uint_as_float(v[J]), __uint_as_float(v[J + 1]), __uint_as_float(v[J + 2]));
+            const float t2 = absmax3(__uint_as_float(v[J + 3]), __uint_as_float(v[J + 4]), __uint_as_float(v[J + 5]));
+            gm = fmaxf(t2, absmax3(__uint_as_float(v[J + 6]), __uint_as_float(v[J + 7]), t1));
+        }
+        return mask_tag<kTag>(__float_as_uint(gm), mask);
     }
-    return __vimax3_u32(__vimax3_u32(m0, m1, m2), m3, 0u);
+}
+
+// Running key maxima (two independent chains) over the 32 / G groups of a 32-column chunk.
+template <int G, int COL0, int J = 0>
+__device__ __forceinline__ void chunk_key_max(const uint32_t (&v)[32], uint32_t mask, uint32_t& m0, uint32_t& m1) {
+    if constexpr (J < 32) {
+        m0 = __vimax3_u32(m0, group_key<G, COL0, J>(v, mask), group_key<G, COL0, J + G>(v, mask));
+        m1 = __vimax3_u32(m1, group_key<G, COL0, J + 2 * G>(v, mask), group_key<G, COL0, J + 3 * G>(v, mask));
+        chunk_key_max<G, COL0, J + 4 * G>(v, mask, m0, m1);
+    }
+}
+
+// fp32 dot product of eight bf16 pairs (one 16-byte chunk of a residual row and of an atom)
+__device__ __forceinline__ void dot8(const uint4& rv, const uint4& av, float& even, float& odd) {
+    even = fmaf(bf_lo(rv.x), bf_lo(av.x), even);
+    odd = fmaf(bf_hi(rv.x), bf_hi(av.x), odd);
+    even = fmaf(bf_lo(rv.y), bf_lo(av.y), even);
+    odd = fmaf(bf_hi(rv.y), bf_hi(av.y), odd);
+    even = fmaf(bf_lo(rv.z), bf_lo(av.z), even);
+    odd = fmaf(bf_hi(rv.z), bf_hi(av.z), odd);
+    even = fmaf(bf_lo(rv.w), bf_lo(av.w), even);
+    odd = fmaf(bf_hi(rv.w), bf_hi(av.w), odd);
+}
+// r -= coef * a on one 16-byte chunk, rounded back to bf16
+__device__ __forceinline__ uint4 axpy8(const uint4& rv, const uint4& av, float coef) {
+    uint4 o;
+    o.x = pack_bf16(fmaf(-coef, bf_lo(av.x), bf_lo(rv.x)), fmaf(-coef, bf_hi(av.x), bf_hi(rv.x)));
+    o.y = pack_bf16(fmaf(-coef, bf_lo(av.y), bf_lo(rv.y)), fmaf(-coef, bf_hi(av.y), bf_hi(rv.y)));
+    o.z = pack_bf16(fmaf(-coef, bf_lo(av.z), bf_lo(rv.z)), fmaf(-coef, bf_hi(av.z), bf_hi(rv.z)));
+    o.w = pack_bf16(fmaf(-coef, bf_lo(av.w), bf_lo(rv.w)), fmaf(-coef, bf_hi(av.w), bf_hi(rv.w)));
+    return o;
+}
+
+// End of a sweep for the 32 rows of one epilogue warp (Eq. 2-4).  Lane i enters with the
+// first atom `n0` of the winning group of row q*32 + i.  Eight lanes work on one row (four
+// rows per pass, eight passes): each lane gathers its 1/8 of the G candidate atoms (one
+// contiguous run of G * 2 * D_ bytes per row), the G signed correlations with the row's
+// residual are rebuilt as fp32 dot products and summed over the eight lanes, the largest
+// in magnitude (lowest atom on ties) gives the index and the coefficient, and, unless
+// this was the last iteration, the residual row in the operand tile becomes
+// R - coef * atom.  The code goes to the row's slot in the shared-memory staging arrays.
+template <int D_, int G>
+__device__ __forceinline__ void pick_and_update(uint8_t* Atile, int q, int lane, const uint16_t* __restrict__ Db,
+                                                int n0, bool update, uint16_t (*code_idx)[CODE_BLOCK],
+                                                float (*code_coef)[CODE_BLOCK], int gi) {
+    constexpr int CH = D_ / 64;                           // 16-byte chunks per lane per atom
+    constexpr int APR = D_ / 8;                           // 16-byte chunks per atom row
+    constexpr int LPP = G * CH;                           // gathered chunks per lane per pass
+    constexpr int WAVE = (32 / LPP) < 8 ? (32 / LPP) : 8; // passes whose gathers are in flight together
+    const int sub = lane >> 3, l8 = lane & 7;
+#pragma unroll
+    for (int w0 = 0; w0 < 8; w0 += WAVE) {
+        uint4 atom[WAVE][G][CH];
+        int base[WAVE];
+#pragma unroll
+        for (int it = 0; it < WAVE; ++it) {
+            base[it] = __shfl_sync(0xffffffffu, n0, (w0 + it) * 4 + sub);
+            const uint4* src = reinterpret_cast<const uint4*>(Db + static_cast<size_t>(base[it]) * D_) + l8 * CH;
+#pragma unroll
+            for (int j = 0; j < G; ++j)
+#pragma unroll
+                for (int c = 0; c < CH; ++c) atom[it][j][c] = __ldg(src + j * APR + c);
+        }
+#pragma unroll
+        for (int it = 0; it < WAVE; ++it) {
+            const int i = (w0 + it) * 4 + sub;            // row inside the warp's 32
+            const int r = q * 32 + i;                     // row inside the tile
+            uint4 rv[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c) rv[c] = *reinterpret_cast<const uint4*>(Atile + swz_off(r, l8 * CH + c));
+            float dot[G];
+#pragma unroll
+            for (int j = 0; j < G; ++j) {
+                float ev = 0.f, od = 0.f;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) dot8(rv[c], atom[it][j][c], ev, od);
+                dot[j] = ev + od;
+            }
+#pragma unroll
+            for (int m = 1; m < 8; m <<= 1)
+#pragma unroll
+                for (int j = 0; j < G; ++j) dot[j] += __shfl_xor_sync(0xffffffffu, dot[j], m);
+            float coef = dot[0];
+            int jb = 0;
+#pragma unroll
+            for (int j = 1; j < G; ++j)
+                if (fabsf(dot[j]) > fabsf(coef)) {
+                    coef = dot[j];
+                    jb = j;
+                }
+            if (update) {
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    uint4 av = atom[it][0][c];
+#pragma unroll
+                    for (int j = 1; j < G; ++j)
+                        if (jb == j) av = atom[it][j][c];
+                    *reinterpret_cast<uint4*>(Atile + swz_off(r, l8 * CH + c)) = axpy8(rv[c], av, coef);
+                }
+            }
+            if (l8 == 0) {
+                code_idx[r][gi] = static_cast<uint16_t>(base[it] + jb);
+                code_coef[r][gi] = coef;
+            }
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -246,22 +400,23 @@ __global__ void dict_to_bf16_kernel(const float4* __restrict__ src, uint2* __res
 // ---------------------------------------------------------------------------------------
 // the encoder
 // ---------------------------------------------------------------------------------------
-template <int D_>
+template <int D_, int G>
 __global__ void __launch_bounds__(NT, 1)
 encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* __restrict__ Db,
                    const void* __restrict__ X, int x_dtype, int64_t M, int N, int s, uint16_t* __restrict__ out_idx,
-                   void* __restrict__ out_coef, int coef_dtype, uint32_t* status) {
+                   void* __restrict__ out_coef, int coef_dtype, uint32_t key_mask, uint32_t* status) {
     using S = FastSmem<D_>;
     extern __shared__ uint8_t smem_raw[];
     S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int T = N / TILE_N;                               // dictionary tiles per sweep
+    const int T = (N + TILE_N - 1) / TILE_N;                // dictionary tiles per sweep (the last may be half)
     const int64_t n_pairs = (M + 2 * TILE_M - 1) / (2 * TILE_M);
-    constexpr int KSTEPS = D_ / UMMA_K;
+    constexpr int KH = D_ / STAGE_CH;                       // stages per dictionary tile
+    constexpr int KSTEPS = STAGE_CH / UMMA_K;               // MMAs per stage
     constexpr int CHUNKS = D_ / 8;                          // 16-byte chunks per row
-    constexpr uint32_t kStageBytes = S::kTileBytes;
+    constexpr int NG = TILE_N / G;                          // arg-max groups per accumulator
     const WaitCtx wc{&sm.abort, status};
 
     if (threadIdx.x == 0) {
@@ -270,10 +425,8 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             mbar_init(&sm.empty_b[i], 1);
         }
         for (int t = 0; t < 2; ++t) {
-            for (int b = 0; b < 2; ++b) {
-                mbar_init(&sm.acc_full[t][b], 1);
-                mbar_init(&sm.acc_empty[t][b], 4);
-            }
+            mbar_init(&sm.acc_full[t], 1);
+            mbar_init(&sm.acc_empty[t], 4);
             mbar_init(&sm.res_ready[t], TILE_M);
         }
         mbar_init(&sm.drained, 1);
@@ -297,26 +450,26 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             bool ok = true;
             for (int64_t pair = blockIdx.x; pair < n_pairs && ok; pair += gridDim.x) {
                 for (int g = 0; g < s && ok; ++g) {
-                    for (int t = 0; t < T; ++t, ++p) {
-                        const int stage = p % STAGES;
-                        if (!wait_bounded(&sm.empty_b[stage], ((p / STAGES) & 1) ^ 1, wc)) {
-                            ok = false;
-                            break;
+                    for (int t = 0; t < T && ok; ++t) {
+                        for (int h = 0; h < KH; ++h, ++p) {
+                            const int stage = p % STAGES;
+                            if (!wait_bounded(&sm.empty_b[stage], ((p / STAGES) & 1) ^ 1, wc)) {
+                                ok = false;
+                                break;
+                            }
+                            // rows past N (a half tile at the end) arrive as zeros and count as bytes
+                            mbar_expect_tx(&sm.full_b[stage], S::kStageBytes);
+                            tma_load_2d(&sm.B[stage][0], &tmap_d, h * STAGE_CH, t * TILE_N, &sm.full_b[stage]);
                         }
-                        mbar_expect_tx(&sm.full_b[stage], kStageBytes);
-#pragma unroll
-                        for (int h = 0; h < D_ / 64; ++h)
-                            tma_load_2d(&sm.B[stage][h * (TILE_N * 128)], &tmap_d, h * 64, t * TILE_N,
-                                        &sm.full_b[stage]);
                     }
                 }
             }
             if (!ok) {
                 // let the copies already issued land before the CTA goes away
                 const uint32_t first = p > STAGES ? p - STAGES : 0;
-                for (uint32_t q = first; q < p; ++q) {
+                for (uint32_t qq = first; qq < p; ++qq) {
                     const unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(&sm.full_b[q % STAGES], (q / STAGES) & 1))
+                    while (!mbar_try_wait(&sm.full_b[qq % STAGES], (qq / STAGES) & 1))
                         if (globaltimer_ns() - t0 > 20000000ull) break;
                 }
             }
@@ -328,36 +481,39 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             bool ok = true;
             for (int64_t pair = blockIdx.x; pair < n_pairs && ok; pair += gridDim.x) {
                 for (int g = 0; g < s && ok; ++g, ++steps) {
-                    for (int t = 0; t < T && ok; ++t, ++p, ++accn) {
-                        const int stage = p % STAGES;
-                        const uint32_t buf = accn & 1;
-                        if (!wait_bounded(&sm.full_b[stage], (p / STAGES) & 1, wc)) {
-                            ok = false;
-                            break;
-                        }
-                        for (int tile = 0; tile < 2; ++tile) {
+                    for (int t = 0; t < T && ok; ++t, p += KH, ++accn) {
+                        for (int tile = 0; tile < 2 && ok; ++tile) {
                             if (t == 0 && !wait_bounded(&sm.res_ready[tile], steps & 1, wc)) {
                                 ok = false;
                                 break;
                             }
-                            if (!wait_bounded(&sm.acc_empty[tile][buf], ((accn >> 1) & 1) ^ 1, wc)) {
+                            if (!wait_bounded(&sm.acc_empty[tile], (accn & 1) ^ 1, wc)) {
                                 ok = false;
                                 break;
                             }
-                            tc_fence_after();
-                            const uint32_t d_tmem = tmem_base + (tile * 2 + buf) * TILE_N;
-                            const uint64_t a0 = make_smem_desc(smem_u32(&sm.A[tile][0]));
-                            const uint64_t b0 = make_smem_desc(smem_u32(&sm.B[stage][0]));
+                            const uint32_t d_tmem = tmem_base + tile * TILE_N;
 #pragma unroll
-                            for (int k = 0; k < KSTEPS; ++k) {
-                                // 16 channels = 32 bytes inside a 128-byte swizzled row; the
-                                // second 64-channel half is a separate block of TILE_M rows
-                                const uint64_t off = static_cast<uint64_t>(((k >> 2) * (TILE_M * 128) + (k & 3) * 32) >> 4);
-                                umma_bf16(d_tmem, a0 + off, b0 + off, kInstrDesc, k > 0 ? 1u : 0u);
+                            for (int h = 0; h < KH; ++h) {
+                                const uint32_t ps = p + h;
+                                const int stage = ps % STAGES;
+                                if (tile == 0 && !wait_bounded(&sm.full_b[stage], (ps / STAGES) & 1, wc)) {
+                                    ok = false;
+                                    break;
+                                }
+                                tc_fence_after();
+                                const uint64_t a0 = make_smem_desc(smem_u32(&sm.A[tile][h * (TILE_M * 128)]));
+                                const uint64_t b0 = make_smem_desc(smem_u32(&sm.B[stage][0]));
+#pragma unroll
+                                for (int k = 0; k < KSTEPS; ++k) {
+                                    // 16 channels = 32 bytes inside a 128-byte swizzled row
+                                    const uint64_t off = static_cast<uint64_t>((k * 32) >> 4);
+                                    umma_bf16(d_tmem, a0 + off, b0 + off, kInstrDesc, (h | k) ? 1u : 0u);
+                                }
+                                // the second row tile is the last reader of a stage
+                                if (tile == 1) umma_commit(&sm.empty_b[stage]);
                             }
-                            umma_commit(&sm.acc_full[tile][buf]);
+                            if (ok) umma_commit(&sm.acc_full[tile]);
                         }
-                        if (ok) umma_commit(&sm.empty_b[stage]);
                     }
                 }
             }
@@ -376,6 +532,9 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         const int r = q * 32 + lane;                      // row inside the tile == TMEM lane
         const int slot = tile * TILE_M + r;               // row inside the CTA's pair
         uint8_t* Atile = &sm.A[tile][0];
+        uint16_t (*code_idx)[CODE_BLOCK] = &sm.code_idx[tile * TILE_M];
+        float (*code_coef)[CODE_BLOCK] = &sm.code_coef[tile * TILE_M];
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + tile * TILE_N;
         uint32_t accn = 0;
         bool ok = true;
         for (int64_t pair = blockIdx.x; pair < n_pairs && ok; pair += gridDim.x) {
@@ -388,7 +547,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 for (int c = 0; c < CHUNKS; ++c) {
                     uint4 v = make_uint4(0u, 0u, 0u, 0u);
                     if (valid) v = __ldg(src + c);
-                    *reinterpret_cast<uint4*>(Atile + swz_off<D_>(r, c)) = v;
+                    *reinterpret_cast<uint4*>(Atile + swz_off(r, c)) = v;
                 }
             } else {
                 const float4* src = reinterpret_cast<const float4*>(X) + m * (CHUNKS * 2);
@@ -404,7 +563,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     v.y = pack_bf16(a.z, a.w);
                     v.z = pack_bf16(b.x, b.y);
                     v.w = pack_bf16(b.z, b.w);
-                    *reinterpret_cast<uint4*>(Atile + swz_off<D_>(r, c)) = v;
+                    *reinterpret_cast<uint4*>(Atile + swz_off(r, c)) = v;
                 }
             }
             fence_proxy_async_smem();
@@ -414,33 +573,44 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 // ---- sweep: running arg-max of |correlation| over all atom tiles ----
                 uint32_t best_key = 0, best_t = 0;
                 for (int t = 0; t < T; ++t, ++accn) {
-                    const uint32_t buf = accn & 1;
-                    bool got = wait_bounded(&sm.acc_full[tile][buf], (accn >> 1) & 1, wc);
+                    bool got = wait_bounded(&sm.acc_full[tile], accn & 1, wc);
                     got = __all_sync(0xffffffffu, got);
                     if (!got) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (tile * 2 + buf) * TILE_N;
-                    uint32_t va[32], vb[32];
-                    uint32_t key = 0;
-                    tmem_ld32(taddr + 0, va);
-                    tmem_wait_ld(va);
-                    tmem_ld32(taddr + 32, vb);
-                    key = chunk_key_max<0>(va, key);
-                    tmem_wait_ld(vb);
-                    tmem_ld32(taddr + 64, va);
-                    key = chunk_key_max<32>(vb, key);
-                    tmem_wait_ld(va);
-                    tmem_ld32(taddr + 96, vb);
-                    key = chunk_key_max<64>(va, key);
-                    tmem_wait_ld(vb);
+                    uint32_t v0[32], v1[32], v2[32], v3[32];
+                    uint32_t k0 = 0, k1 = 0;
+                    tmem_ld32(taddr + 0, v0);
+                    tmem_ld32(taddr + 32, v1);
+                    tmem_ld32(taddr + 64, v2);
+                    tmem_ld32(taddr + 96, v3);
+                    tmem_wait_ld(v0);
+                    reg_fence(v1);
+                    reg_fence(v2);
+                    reg_fence(v3);
+                    chunk_key_max<G, 0>(v0, key_mask, k0, k1);
+                    tmem_ld32(taddr + 128, v0);
+                    chunk_key_max<G, 32>(v1, key_mask, k0, k1);
+                    tmem_ld32(taddr + 160, v1);
+                    chunk_key_max<G, 64>(v2, key_mask, k0, k1);
+                    tmem_ld32(taddr + 192, v2);
+                    chunk_key_max<G, 96>(v3, key_mask, k0, k1);
+                    tmem_ld32(taddr + 224, v3);
+                    tmem_wait_ld(v0);
+                    reg_fence(v1);
+                    reg_fence(v2);
+                    reg_fence(v3);
                     // every column of this accumulator is in registers: hand it back
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.acc_empty[tile][buf]);
-                    key = chunk_key_max<96>(vb, key);
+                    if (lane == 0) mbar_arrive(&sm.acc_empty[tile]);
+                    chunk_key_max<G, 128>(v0, key_mask, k0, k1);
+                    chunk_key_max<G, 160>(v1, key_mask, k0, k1);
+                    chunk_key_max<G, 192>(v2, key_mask, k0, k1);
+                    chunk_key_max<G, 224>(v3, key_mask, k0, k1);
+                    const uint32_t key = k0 > k1 ? k0 : k1;
                     if (key > best_key) {
                         best_key = key;
                         best_t = t;
@@ -448,43 +618,16 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 }
                 if (!ok) break;
                 // ---- pick, signed coefficient, residual update ----
-                const int n = best_t * TILE_N + (127 - static_cast<int>(best_key & 127u));
-                const uint4* arow = reinterpret_cast<const uint4*>(Db + static_cast<size_t>(n) * D_);
-                uint4 atom[CHUNKS];
-#pragma unroll
-                for (int c = 0; c < CHUNKS; ++c) atom[c] = __ldg(arow + c);
-                float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
-#pragma unroll
-                for (int c = 0; c < CHUNKS; ++c) {
-                    const uint4 rv = *reinterpret_cast<const uint4*>(Atile + swz_off<D_>(r, c));
-                    c0 = fmaf(bf_lo(rv.x), bf_lo(atom[c].x), c0);
-                    c1 = fmaf(bf_hi(rv.x), bf_hi(atom[c].x), c1);
-                    c2 = fmaf(bf_lo(rv.y), bf_lo(atom[c].y), c2);
-                    c3 = fmaf(bf_hi(rv.y), bf_hi(atom[c].y), c3);
-                    c0 = fmaf(bf_lo(rv.z), bf_lo(atom[c].z), c0);
-                    c1 = fmaf(bf_hi(rv.z), bf_hi(atom[c].z), c1);
-                    c2 = fmaf(bf_lo(rv.w), bf_lo(atom[c].w), c2);
-                    c3 = fmaf(bf_hi(rv.w), bf_hi(atom[c].w), c3);
-                }
-                const float coef = (c0 + c1) + (c2 + c3);
+                const int gi = g & (CODE_BLOCK - 1);
+                const int n0 = static_cast<int>(best_t) * TILE_N +
+                               (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G;
+                pick_and_update<D_, G>(Atile, q, lane, Db, n0, g + 1 < s, code_idx, code_coef, gi);
                 if (g + 1 < s) {
-#pragma unroll
-                    for (int c = 0; c < CHUNKS; ++c) {
-                        uint4* p4 = reinterpret_cast<uint4*>(Atile + swz_off<D_>(r, c));
-                        uint4 rv = *p4;
-                        rv.x = pack_bf16(fmaf(-coef, bf_lo(atom[c].x), bf_lo(rv.x)), fmaf(-coef, bf_hi(atom[c].x), bf_hi(rv.x)));
-                        rv.y = pack_bf16(fmaf(-coef, bf_lo(atom[c].y), bf_lo(rv.y)), fmaf(-coef, bf_hi(atom[c].y), bf_hi(rv.y)));
-                        rv.z = pack_bf16(fmaf(-coef, bf_lo(atom[c].z), bf_lo(rv.z)), fmaf(-coef, bf_hi(atom[c].z), bf_hi(rv.z)));
-                        rv.w = pack_bf16(fmaf(-coef, bf_lo(atom[c].w), bf_lo(rv.w)), fmaf(-coef, bf_hi(atom[c].w), bf_hi(rv.w)));
-                        *p4 = rv;
-                    }
                     fence_proxy_async_smem();
                     mbar_arrive(&sm.res_ready[tile]);
                 }
-                // ---- collect the code; flush eight at a time ----
-                const int gi = g & (CODE_BLOCK - 1);
-                sm.code_idx[slot][gi] = static_cast<uint16_t>(n);
-                sm.code_coef[slot][gi] = coef;
+                __syncwarp();
+                // ---- flush the collected codes eight at a time ----
                 if ((gi == CODE_BLOCK - 1 || g == s - 1) && valid) {
                     const int g0 = g - gi;
                     const int64_t o = m * s + g0;
@@ -516,6 +659,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                         }
                     }
                 }
+                __syncwarp();
             }
         }
     }
@@ -545,18 +689,42 @@ EncodeTiledFn get_encode_tiled() {
     return fn;
 }
 
-template <int D_>
+template <int D_, int G>
 int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status) {
     const size_t smem = sizeof(FastSmem<D_>) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(encode_fast_kernel<D_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e =
+        cudaFuncSetAttribute(encode_fast_kernel<D_, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     const int64_t n_pairs = (a.M + 2 * TILE_M - 1) / (2 * TILE_M);
     const int grid = (int)(n_pairs < (int64_t)sm_count() ? n_pairs : (int64_t)sm_count());
-    encode_fast_kernel<D_><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.M, a.N, a.s, a.out_idx, a.out_coef,
-                                                        a.coef_dtype, status);
+    // keys keep the magnitude bits above the group tag; with G == 1 the key is built from the
+    // raw value, so the mask clears the sign bit as well
+    const uint32_t key_mask = (G == 1 ? 0x7FFFFFFFu : 0xFFFFFFFFu) & ~static_cast<uint32_t>(TILE_N / G - 1);
+    encode_fast_kernel<D_, G><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.M, a.N, a.s, a.out_idx,
+                                                           a.out_coef, a.coef_dtype, key_mask, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "encode_fast launch: %s", cudaGetErrorString(e));
     return CSR_OK;
+}
+
+// Atoms per arg-max group.  CSR_FAST_GROUP (1, 2, 4 or 8) overrides the default; it is a
+// tuning knob only: every setting returns a valid maximum of the same bf16 correlations.
+int group_size(int d) {
+    if (const char* e = getenv("CSR_FAST_GROUP")) {
+        const int v = atoi(e);
+        if (v == 1 || v == 2 || v == 4 || v == 8) return v;
+    }
+    return d == 128 ? 4 : 8;
+}
+
+template <int D_>
+int launch_d(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status) {
+    switch (group_size(D_)) {
+        case 1: return launch<D_, 1>(a, tmap, Db, status);
+        case 2: return launch<D_, 2>(a, tmap, Db, status);
+        case 8: return launch<D_, 8>(a, tmap, Db, status);
+        default: return launch<D_, 4>(a, tmap, Db, status);
+    }
 }
 
 }  // namespace
@@ -590,8 +758,8 @@ int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status) {
     if (r != CUDA_SUCCESS) return fail(CSR_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
 
     const uint16_t* Db = static_cast<const uint16_t*>(workspace);
-    if (a.d == 128) return launch<128>(a, tmap, Db, status);
-    return launch<64>(a, tmap, Db, status);
+    if (a.d == 128) return launch_d<128>(a, tmap, Db, status);
+    return launch_d<64>(a, tmap, Db, status);
 }
 
 }  // namespace csr
