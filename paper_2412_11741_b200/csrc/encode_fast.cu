@@ -707,19 +707,23 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
     return CSR_OK;
 }
 
-// Atoms per arg-max group.  CSR_FAST_GROUP (1, 2, 4 or 8) overrides the default; it is a
-// tuning knob only: every setting returns a valid maximum of the same bf16 correlations.
-int group_size(int d) {
+// Atoms per arg-max group.  Larger groups save arg-max arithmetic during the sweep (which
+// grows with N) and cost a wider gather at the end of every sweep (which does not); the
+// defaults are where the measured crossovers lie.  CSR_FAST_GROUP (1, 2, 4 or 8) overrides
+// them; it is a tuning knob only: every setting returns a valid maximum of the same bf16
+// correlations.
+int group_size(int d, int N) {
     if (const char* e = getenv("CSR_FAST_GROUP")) {
         const int v = atoi(e);
         if (v == 1 || v == 2 || v == 4 || v == 8) return v;
     }
-    return d == 128 ? 4 : 8;
+    if (d == 64) return 4;
+    return N >= 16384 ? 4 : 1;
 }
 
 template <int D_>
 int launch_d(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status) {
-    switch (group_size(D_)) {
+    switch (group_size(D_, a.N)) {
         case 1: return launch<D_, 1>(a, tmap, Db, status);
         case 2: return launch<D_, 2>(a, tmap, Db, status);
         case 8: return launch<D_, 8>(a, tmap, Db, status);

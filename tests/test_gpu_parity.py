@@ -245,6 +245,70 @@ def test_fast_full_size_llama2_layer_sampled(csr):
     assert abs(err / rep.mean_err - 1) < 0.02
 
 
+def _full_size_sampled(csr, w, rows, seed):
+    """Encodes the whole workload in the launch configuration the benchmark times and lets the
+    oracle check a stratified sample of the outputs; every index must be in range and the
+    whole tensor must reconstruct at the sample's error level."""
+    D = torch.from_numpy(w.D).to(DEV)
+    Xd = torch.from_numpy(w.X).to(DEV).to(torch.bfloat16)
+    idx, coef = csr.csr_encode(D, Xd, w.s)
+    assert csr.csr_device_status() == csr.CSR_OK
+    sel = wl.stratified_rows(w.M, rows, seed=seed)
+    st = torch.from_numpy(sel).to(DEV)
+    rep = parity.compare_fast(w.D, w.X[sel], w.s, _np_idx(_take_rows(idx, st)), coef[st].float().cpu().numpy())
+    assert rep.ok, rep.detail
+    assert int(idx.view(torch.int16).to(torch.int32).bitwise_and(0xFFFF).max()) < w.N
+    err = 0.0
+    step = 1 << 18
+    for r0 in range(0, w.M, step):                      # in slices: X_hat of the whole job is large
+        xh = csr.csr_reconstruct(D, _take_rows(idx, slice(r0, r0 + step)).contiguous(), coef[r0:r0 + step].contiguous())
+        xs = Xd[r0:r0 + step].float()
+        err += float(((xh.float() - xs).norm(dim=1) / xs.norm(dim=1)).sum())
+    assert abs(err / w.M / rep.mean_err - 1) < 0.03
+    return rep
+
+
+def test_fast_full_size_gqa_long_sampled(csr):
+    """Config 3 (the benchmark's workload) at full size."""
+    w = wl.gqa_long()
+    assert w.M == 2097152 and w.N == 8192 and w.s == 16
+    _full_size_sampled(csr, w, 1024, seed=31)
+
+
+@pytest.mark.parametrize("s", [4, 32])
+def test_fast_full_size_sparsity_sweep_sampled(csr, s):
+    """Config 4 at full size, the two ends of the sparsity sweep."""
+    w = wl.sparsity_sweep(s)
+    assert w.M == 1 << 20 and w.N == 8192
+    _full_size_sampled(csr, w, 768, seed=41 + s)
+
+
+@pytest.mark.parametrize("N,d", [(2048, 128), (16384, 128), (4096, 64)])
+def test_fast_full_size_dict_sweep_sampled(csr, N, d):
+    """Config 5 at full size: smallest and largest dictionary at d = 128, and d = 64."""
+    w = wl.dict_sweep(N, d=d)
+    assert w.M == 1 << 20
+    _full_size_sampled(csr, w, 768, seed=51 + N // 1024 + d)
+
+
+@pytest.mark.parametrize("G", [1, 2, 4, 8])
+@pytest.mark.parametrize("d", [64, 128])
+def test_fast_every_group_size(csr, G, d, monkeypatch):
+    """The arg-max group size is a tuning knob: every setting must meet the same gates, also
+    with a dictionary that ends in half an atom tile (N = 384) or is smaller than one (N = 128)."""
+    monkeypatch.setenv("CSR_FAST_GROUP", str(G))
+    rng = np.random.default_rng(100 * G + d)
+    for N, M, s in ((384, 700, 6), (128, 300, 3), (2048, 1500, 9)):
+        D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+        X = wl.round_to_bf16(rng.standard_normal((M, d)).astype(np.float32))
+        X[7] = 0.0
+        w = wl.Workload("grp", D, X, s, "bf16")
+        idx, coef = _encode(csr, w, X, csr.CSR_MODE_BF16_FAST)
+        assert idx[7].tolist() == [0] * s and np.all(coef[7] == 0)
+        rep = parity.compare_fast(D, X, s, idx, coef)
+        assert rep.ok, (G, d, N, rep.detail)
+
+
 # ---------------------------------------------------------------------------------------
 # de-sparse
 # ---------------------------------------------------------------------------------------
