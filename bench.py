@@ -35,6 +35,11 @@ UNIT = "vectors/s"
 WORKLOAD = "gqa_long_context: 8 seq x 16384 tok x 8 kv_heads x {K,V}, d=128, M=2097152, N=8192, s=16, bf16"
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of encode_fast_kernel<128, 1> at M = 524288, N = 8192,
+# s = 16 (profiles/encode_fast_small_case_ncu_full.md), per row; traffic grows in proportion to M.
+DRAM_BYTES_PER_ROW_NCU = (137.071104e6 + 18.424320e6) / 524288
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -239,13 +244,20 @@ def run_cuda(args):
     if csr.csr_device_status() != csr.CSR_OK:
         raise SystemExit("device-side wait expired: " + csr.csr_last_error_string())
 
-    # end to end through the host entry point (pinned host buffers, copies inside the timing)
+    # end to end through the host entry points (pinned host buffers, every copy inside the
+    # timing): X in, codes out, then codes in, X_hat out
+    xhat_host = torch.empty((M, d), dtype=torch.bfloat16).pin_memory()
+
+    def e2e_step():
+        csr.csr_encode_host(D, X_host, s, idx_host, coef_host)
+        csr.csr_reconstruct_host(D, idx_host, coef_host, xhat_host)
+
     e2e_steps = max(1, min(args.steps, 5))
-    csr.csr_encode_host(D, X_host, s, idx_host, coef_host)
+    e2e_step()
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        csr.csr_encode_host(D, X_host, s, idx_host, coef_host)
+        e2e_step()
     barrier()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
 
@@ -263,10 +275,11 @@ def run_cuda(args):
         achieved = flops / (enc * 1e-3) / 1e12
         hbm_bytes = M * d * 2 + N * d * 4 + M * s * 4
         roof = {
-            "bound": "tensor", "kernel": "encode_fast_kernel<128>", "achieved": achieved, "peak": peaks["bf16_tflops"],
+            "bound": "tensor", "kernel": "encode_fast_kernel<128, 1>", "achieved": achieved, "peak": peaks["bf16_tflops"],
             "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
             "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
-            "flops_per_launch": flops, "kernel_ms": enc, "traffic": None,
+            "flops_per_launch": flops, "kernel_ms": enc, "traffic": DRAM_BYTES_PER_ROW_NCU * M,
+            "traffic_source": "ncu dram read+write of one launch at M=524288 (profiles/), scaled by rows",
             "algorithmic_hbm_bytes": hbm_bytes,
         }
         line = {
@@ -279,8 +292,10 @@ def run_cuda(args):
             "encode_ms": enc, "reconstruct_ms": statistics.mean(rec_ms),
             "encode_vectors_per_sec": M / (enc * 1e-3),
             "clocks": clocks,
-            "e2e": {"value": world * M / e2e_s, "unit": UNIT, "h2d_bytes_per_step": M * d * 2,
-                    "d2h_bytes_per_step": M * s * 4, "call": "csr_encode_host (pinned host X in, host codes out)"},
+            "e2e": {"value": world * M / e2e_s, "unit": UNIT, "h2d_bytes_per_step": M * d * 2 + M * s * 4,
+                    "d2h_bytes_per_step": M * s * 4 + M * d * 2, "ms_per_step": e2e_s * 1e3,
+                    "call": "csr_encode_host (pinned host X in, host codes out) + csr_reconstruct_host "
+                            "(host codes in, pinned host X_hat out)"},
             "gpu_launches": 3 * args.steps,
             "roofline": roof,
         }

@@ -144,6 +144,15 @@ int csr_reconstruct_ex(const csr_reconstruct_params_t* p);
 int csr_encode_host(const csr_encode_params_t* p);
 
 /*
+ * De-sparse with HOST buffers (the same operation as csr_reconstruct_ex, Eq. 12; idx, coef
+ * and X_hat are host pointers, ideally page-locked): the case of codes kept in host memory
+ * and restored on demand.  Codes are copied to the device in chunks, X_hat chunks are
+ * copied back while the next chunk is computed, and the function returns after everything
+ * has finished.  D stays a device pointer.  Shares the staging buffers of csr_encode_host.
+ */
+int csr_reconstruct_host(const csr_reconstruct_params_t* p);
+
+/*
  * Fast encode without any allocation (the paper has no counterpart; this entry point
  * exists for the deployment reasons below).  Same operation, layouts and results as the
  * 8-argument csr_encode (bf16 X, fp16 coefficients, fast mode), on the given stream.

@@ -1,0 +1,108 @@
+"""Throughput and reconstruction error of the codec on every synthetic configuration.
+
+  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5] [--reps 30]
+
+One JSON line per case: vectors/s and TFLOP/s of the fast encoder (median of the last two
+thirds of `reps` back-to-back launches, i.e. after the clocks have settled under the power
+cap), mean relative reconstruction error ||x - x_hat|| / ||x|| over all rows, the de-sparse
+kernel's time with its HBM and L2-gather rates, and the fp32-exact encoder's rate on a
+prefix of the rows.  Timed with CUDA events on torch's current stream; inputs are larger
+than L2 except for the tiny configuration.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as csr
+from . import build, workloads as wl
+
+
+def _median_tail(xs):
+    tail = sorted(xs[len(xs) // 3:])
+    return tail[len(tail) // 2]
+
+
+def _time(fn, reps):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in ev:
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    return _median_tail([a.elapsed_time(b) for a, b in ev])
+
+
+def run_case(w, reps, exact_rows=16384):
+    dev = torch.device("cuda", torch.cuda.current_device())
+    M, N, d, s = w.M, w.N, w.d, w.s
+    D = torch.from_numpy(w.D).to(dev)
+    X = torch.from_numpy(w.X).to(dev)
+    if w.x_dtype == "bf16":
+        X = X.to(torch.bfloat16)
+    idx = torch.empty((M, s), dtype=torch.uint16, device=dev)
+    coef = torch.empty((M, s), dtype=torch.float16, device=dev)
+    enc_ms = _time(lambda: csr.csr_encode_ex(D, X, s, out_idx=idx, out_coef=coef), reps)
+    if csr.csr_device_status() != csr.CSR_OK:
+        raise RuntimeError(csr.csr_last_error_string())
+    xh = torch.empty((M, d), dtype=torch.bfloat16, device=dev)
+    rec_ms = _time(lambda: csr.csr_reconstruct_ex(D, idx, coef, X_hat=xh), max(5, reps // 3))
+    err_sum, step = 0.0, 1 << 18
+    for r0 in range(0, M, step):
+        xs = X[r0:r0 + step].float()
+        err_sum += float(((xh[r0:r0 + step].float() - xs).norm(dim=1) / xs.norm(dim=1).clamp_min(1e-30)).sum())
+    me = min(M, exact_rows)
+    Xe = X[:me].contiguous()
+    ie = torch.empty((me, s), dtype=torch.uint16, device=dev)
+    ce = torch.empty((me, s), dtype=torch.float32, device=dev)
+    ex_ms = _time(lambda: csr.csr_encode_ex(D, Xe, s, mode=csr.CSR_MODE_FP32_EXACT, out_idx=ie, out_coef=ce), 5)
+    flops = 2.0 * M * N * d * s
+    return {
+        "case": w.name, "M": M, "N": N, "d": d, "s": s, "x_dtype": w.x_dtype,
+        "encode_ms": round(enc_ms, 4), "vectors_per_s": M / (enc_ms * 1e-3), "tflops": flops / (enc_ms * 1e-3) / 1e12,
+        "mean_rel_error": err_sum / M,
+        "reconstruct_ms": round(rec_ms, 4),
+        "reconstruct_hbm_gbs": M * (4 * s + 2 * d) / (rec_ms * 1e-3) / 1e9,
+        "reconstruct_l2_gather_gbs": M * s * d * 4 / (rec_ms * 1e-3) / 1e9,
+        "exact_mode_vectors_per_s": me / (ex_ms * 1e-3), "exact_mode_rows": me,
+    }
+
+
+def cases(names):
+    for n in names:
+        if n == "c1":
+            yield wl.tiny()
+        elif n == "c2":
+            yield wl.llama2_layer()
+        elif n == "c3":
+            yield wl.gqa_long()
+        elif n == "c4":
+            for s in (4, 8, 16, 32):
+                yield wl.sparsity_sweep(s)
+        elif n == "c5":
+            for N in (2048, 4096, 8192, 16384):
+                yield wl.dict_sweep(N)
+            yield wl.dict_sweep(4096, d=64)
+        else:
+            raise SystemExit(f"unknown configuration {n}")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--configs", default="c1,c2,c3,c4,c5")
+    ap.add_argument("--reps", type=int, default=30)
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device (there is no CPU fallback)")
+    build.build()
+    for w in cases(args.configs.split(",")):
+        print(json.dumps(run_case(w, args.reps)), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -33,7 +33,7 @@ CSR_MODE_BF16_FAST = 1
 
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
-    "csr_encode_host", "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
+    "csr_encode_host", "csr_reconstruct_host", "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
 
@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
         L.csr_reconstruct.restype = i32
         L.csr_reconstruct_ex.argtypes = [ctypes.POINTER(csr_reconstruct_params_t)]
         L.csr_reconstruct_ex.restype = i32
+        L.csr_reconstruct_host.argtypes = [ctypes.POINTER(csr_reconstruct_params_t)]
+        L.csr_reconstruct_host.restype = i32
         L.csr_device_status.argtypes = [vp]
         L.csr_device_status.restype = i32
         L.csr_release_workspace.argtypes = []
@@ -238,6 +240,29 @@ def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *
     with torch.cuda.device(D.device):
         _check(lib().csr_reconstruct_ex(ctypes.byref(p)))
     return X_hat
+
+
+def csr_reconstruct_host(D: torch.Tensor, idx_host: torch.Tensor, coef_host: torch.Tensor,
+                         X_hat_host: torch.Tensor) -> None:
+    """csr_reconstruct_host: D on the device; the codes and X_hat are host tensors (pinned for
+    speed).  Returns after X_hat has arrived in the host tensor."""
+    assert D.is_cuda and not idx_host.is_cuda and not coef_host.is_cuda and not X_hat_host.is_cuda
+    assert idx_host.is_contiguous() and coef_host.is_contiguous() and X_hat_host.is_contiguous()
+    assert D.dtype == torch.float32 and idx_host.dtype == torch.uint16 and idx_host.shape == coef_host.shape
+    M, s = idx_host.shape
+    N, d = D.shape
+    assert tuple(X_hat_host.shape) == (M, d)
+    p = csr_reconstruct_params_t()
+    p.struct_size = ctypes.sizeof(csr_reconstruct_params_t)
+    p.D = D.data_ptr()
+    p.idx = idx_host.data_ptr()
+    p.coef = coef_host.data_ptr()
+    p.coef_dtype = _TORCH_DTYPE[coef_host.dtype]
+    p.out_dtype = _TORCH_DTYPE[X_hat_host.dtype]
+    p.M, p.d, p.N, p.s = M, d, N, s
+    p.X_hat = X_hat_host.data_ptr()
+    with torch.cuda.device(D.device):
+        _check(lib().csr_reconstruct_host(ctypes.byref(p)))
 
 
 def csr_reconstruct(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor,

@@ -118,6 +118,82 @@ int check_encode(const csr_encode_params_t* p, bool host_io) {
     return CSR_OK;
 }
 
+// Chunk of a host-side job: a multiple of 256 rows, about 1/8 of the job, at least 32768 rows.
+int64_t host_chunk_rows(int64_t M) {
+    int64_t chunk = ((M / 8 + 255) / 256) * 256;
+    if (chunk < 32768) chunk = 32768;
+    if (chunk > M) chunk = ((M + 255) / 256) * 256;
+    return chunk;
+}
+
+// Two copy streams with their events and two sets of staging buffers (rows of X or X_hat,
+// indices, coefficients), grown on demand.
+int ensure_staging(DeviceBuffers& b, size_t need_x, size_t need_c) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    cudaError_t e = cudaSuccess;
+    if (!b.copy_streams[0]) {
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaStreamCreateWithFlags(&b.copy_streams[i], cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b.ev_in[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b.ev_done[i], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "stream/event creation: %s", cudaGetErrorString(e));
+    }
+    if (b.stage_x_bytes < need_x || b.stage_code_bytes < need_c) {
+        if (need_x < b.stage_x_bytes) need_x = b.stage_x_bytes;
+        if (need_c < b.stage_code_bytes) need_c = b.stage_code_bytes;
+        cudaDeviceSynchronize();
+        for (int i = 0; i < 2; ++i) {
+            cudaFree(b.stage_x[i]);
+            cudaFree(b.stage_idx[i]);
+            cudaFree(b.stage_coef[i]);
+            b.stage_x[i] = b.stage_idx[i] = b.stage_coef[i] = nullptr;
+        }
+        b.stage_x_bytes = b.stage_code_bytes = 0;
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaMalloc(&b.stage_x[i], need_x);
+            if (e == cudaSuccess) e = cudaMalloc(&b.stage_idx[i], need_c);
+            if (e == cudaSuccess) e = cudaMalloc(&b.stage_coef[i], need_c);
+        }
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "staging cudaMalloc: %s", cudaGetErrorString(e));
+        b.stage_x_bytes = need_x;
+        b.stage_code_bytes = need_c;
+    }
+    return CSR_OK;
+}
+
+int check_reconstruct(const csr_reconstruct_params_t* p, bool host_io) {
+    if (!p) return fail(CSR_ERR_INVALID_ARG, "params is NULL");
+    if (p->struct_size != sizeof(csr_reconstruct_params_t))
+        return fail(CSR_ERR_INVALID_ARG, "struct_size %u != %zu", p->struct_size, sizeof(csr_reconstruct_params_t));
+    if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
+    if (p->coef_dtype != CSR_DTYPE_F32 && p->coef_dtype != CSR_DTYPE_F16)
+        return fail(CSR_ERR_INVALID_ARG, "coef_dtype must be F32 or F16");
+    if (p->out_dtype != CSR_DTYPE_F32 && p->out_dtype != CSR_DTYPE_BF16)
+        return fail(CSR_ERR_INVALID_ARG, "out_dtype must be F32 or BF16");
+    if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
+    if (p->M > 0 && (!p->idx || !p->coef || !p->X_hat)) return fail(CSR_ERR_INVALID_ARG, "idx, coef or X_hat is NULL");
+    if (!aligned16(p->D) || (!host_io && (!aligned16(p->idx) || !aligned16(p->coef) || !aligned16(p->X_hat))))
+        return fail(CSR_ERR_ALIGNMENT, "D, idx, coef and X_hat must be 16-byte aligned");
+    return CSR_OK;
+}
+
+ReconstructArgs reconstruct_args(const csr_reconstruct_params_t* p) {
+    ReconstructArgs a;
+    a.D = static_cast<const float*>(p->D);
+    a.idx = p->idx;
+    a.coef = p->coef;
+    a.coef_dtype = p->coef_dtype;
+    a.out_dtype = p->out_dtype;
+    a.M = p->M;
+    a.d = p->d;
+    a.N = p->N;
+    a.s = p->s;
+    a.X_hat = p->X_hat;
+    a.stream = static_cast<cudaStream_t>(p->stream);
+    return a;
+}
+
 int64_t workspace_bytes(int mode, int d, int N) {
     if (mode == CSR_MODE_FP32_EXACT) return 0;
     return (int64_t)(kStatusBytes + 1024 + encode_fast_workspace_bytes(d, N));
@@ -199,31 +275,8 @@ int csr_encode(const void* D, const void* X, int64_t M, int d, int N, int s, uin
 }
 
 int csr_reconstruct_ex(const csr_reconstruct_params_t* p) {
-    if (!p) return fail(CSR_ERR_INVALID_ARG, "params is NULL");
-    if (p->struct_size != sizeof(csr_reconstruct_params_t))
-        return fail(CSR_ERR_INVALID_ARG, "struct_size %u != %zu", p->struct_size, sizeof(csr_reconstruct_params_t));
-    if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
-    if (p->coef_dtype != CSR_DTYPE_F32 && p->coef_dtype != CSR_DTYPE_F16)
-        return fail(CSR_ERR_INVALID_ARG, "coef_dtype must be F32 or F16");
-    if (p->out_dtype != CSR_DTYPE_F32 && p->out_dtype != CSR_DTYPE_BF16)
-        return fail(CSR_ERR_INVALID_ARG, "out_dtype must be F32 or BF16");
-    if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
-    if (p->M > 0 && (!p->idx || !p->coef || !p->X_hat)) return fail(CSR_ERR_INVALID_ARG, "idx, coef or X_hat is NULL");
-    if (!aligned16(p->D) || !aligned16(p->idx) || !aligned16(p->coef) || !aligned16(p->X_hat))
-        return fail(CSR_ERR_ALIGNMENT, "D, idx, coef and X_hat must be 16-byte aligned");
-    ReconstructArgs a;
-    a.D = static_cast<const float*>(p->D);
-    a.idx = p->idx;
-    a.coef = p->coef;
-    a.coef_dtype = p->coef_dtype;
-    a.out_dtype = p->out_dtype;
-    a.M = p->M;
-    a.d = p->d;
-    a.N = p->N;
-    a.s = p->s;
-    a.X_hat = p->X_hat;
-    a.stream = static_cast<cudaStream_t>(p->stream);
-    return launch_reconstruct(a);
+    if (int rc = check_reconstruct(p, false)) return rc;
+    return launch_reconstruct(reconstruct_args(p));
 }
 
 int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_t M, int d, int N, int s,
@@ -252,42 +305,9 @@ int csr_encode_host(const csr_encode_params_t* p) {
     const size_t xb = (p->x_dtype == CSR_DTYPE_BF16 ? 2 : 4) * (size_t)p->d;
     const size_t cb = (p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4) * (size_t)p->s;
     const size_t ib = 2 * (size_t)p->s;
-    // chunk rows: a multiple of 256, about 1/8 of the job, at least 32768 rows
-    int64_t chunk = ((p->M / 8 + 255) / 256) * 256;
-    if (chunk < 32768) chunk = 32768;
-    if (chunk > p->M) chunk = ((p->M + 255) / 256) * 256;
+    const int64_t chunk = host_chunk_rows(p->M);
     DeviceBuffers& b = g_dev[dev];
-    {
-        std::lock_guard<std::mutex> lk(g_mu);
-        cudaError_t e = cudaSuccess;
-        if (!b.copy_streams[0]) {
-            for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
-                e = cudaStreamCreateWithFlags(&b.copy_streams[i], cudaStreamNonBlocking);
-                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b.ev_in[i], cudaEventDisableTiming);
-                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b.ev_done[i], cudaEventDisableTiming);
-            }
-            if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "stream/event creation: %s", cudaGetErrorString(e));
-        }
-        const size_t need_x = (size_t)chunk * xb, need_c = (size_t)chunk * (cb > ib ? cb : ib);
-        if (b.stage_x_bytes < need_x || b.stage_code_bytes < need_c) {
-            cudaDeviceSynchronize();
-            for (int i = 0; i < 2; ++i) {
-                cudaFree(b.stage_x[i]);
-                cudaFree(b.stage_idx[i]);
-                cudaFree(b.stage_coef[i]);
-                b.stage_x[i] = b.stage_idx[i] = b.stage_coef[i] = nullptr;
-            }
-            b.stage_x_bytes = b.stage_code_bytes = 0;
-            for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
-                e = cudaMalloc(&b.stage_x[i], need_x);
-                if (e == cudaSuccess) e = cudaMalloc(&b.stage_idx[i], need_c);
-                if (e == cudaSuccess) e = cudaMalloc(&b.stage_coef[i], need_c);
-            }
-            if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "staging cudaMalloc: %s", cudaGetErrorString(e));
-            b.stage_x_bytes = need_x;
-            b.stage_code_bytes = need_c;
-        }
-    }
+    if (int rc = ensure_staging(b, (size_t)chunk * xb, (size_t)chunk * (cb > ib ? cb : ib))) return rc;
     // Chunk j uses slot j % 2 with its own stream for copy-in, encode and copy-out, so the
     // copies of one chunk overlap the kernels of the other.
     const int64_t n_chunks = (p->M + chunk - 1) / chunk;
@@ -318,6 +338,54 @@ int csr_encode_host(const csr_encode_params_t* p) {
         if (e == cudaSuccess)
             e = cudaMemcpyAsync(static_cast<char*>(p->out_coef) + (size_t)r0 * cb, b.stage_coef[slot],
                                 (size_t)rows * cb, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) rc = fail(CSR_ERR_CUDA, "D2H copy: %s", cudaGetErrorString(e));
+    }
+    for (int i = 0; i < 2; ++i) {
+        cudaError_t e = cudaStreamSynchronize(b.copy_streams[i]);
+        if (e != cudaSuccess && rc == CSR_OK) rc = fail(CSR_ERR_CUDA, "stream sync: %s", cudaGetErrorString(e));
+    }
+    return rc;
+}
+
+int csr_reconstruct_host(const csr_reconstruct_params_t* p) {
+    if (int rc = check_reconstruct(p, true)) return rc;
+    if (p->M == 0) return CSR_OK;
+    int dev;
+    if (int rc = current_device(&dev)) return rc;
+    const size_t xb = (p->out_dtype == CSR_DTYPE_BF16 ? 2 : 4) * (size_t)p->d;
+    const size_t cb = (p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4) * (size_t)p->s;
+    const size_t ib = 2 * (size_t)p->s;
+    const int64_t chunk = host_chunk_rows(p->M);
+    DeviceBuffers& b = g_dev[dev];
+    if (int rc = ensure_staging(b, (size_t)chunk * xb, (size_t)chunk * (cb > ib ? cb : ib))) return rc;
+    // Chunk j uses slot j % 2 with its own stream: the copies of one chunk overlap the kernel
+    // of the other.
+    const int64_t n_chunks = (p->M + chunk - 1) / chunk;
+    int rc = CSR_OK;
+    for (int64_t j = 0; j < n_chunks && rc == CSR_OK; ++j) {
+        const int slot = (int)(j & 1);
+        const int64_t r0 = j * chunk;
+        const int64_t rows = (p->M - r0 < chunk) ? (p->M - r0) : chunk;
+        cudaStream_t st = b.copy_streams[slot];
+        cudaError_t e = cudaMemcpyAsync(b.stage_idx[slot], reinterpret_cast<const char*>(p->idx) + (size_t)r0 * ib,
+                                        (size_t)rows * ib, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(b.stage_coef[slot], static_cast<const char*>(p->coef) + (size_t)r0 * cb,
+                                (size_t)rows * cb, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) {
+            rc = fail(CSR_ERR_CUDA, "H2D copy: %s", cudaGetErrorString(e));
+            break;
+        }
+        csr_reconstruct_params_t q = *p;
+        q.idx = static_cast<const uint16_t*>(b.stage_idx[slot]);
+        q.coef = b.stage_coef[slot];
+        q.X_hat = b.stage_x[slot];
+        q.M = rows;
+        q.stream = st;
+        rc = launch_reconstruct(reconstruct_args(&q));
+        if (rc != CSR_OK) break;
+        e = cudaMemcpyAsync(static_cast<char*>(p->X_hat) + (size_t)r0 * xb, b.stage_x[slot], (size_t)rows * xb,
+                            cudaMemcpyDeviceToHost, st);
         if (e != cudaSuccess) rc = fail(CSR_ERR_CUDA, "D2H copy: %s", cudaGetErrorString(e));
     }
     for (int i = 0; i < 2; ++i) {

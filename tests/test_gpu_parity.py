@@ -354,3 +354,12 @@ def test_host_entry_point(csr):
     idx, coef = csr.csr_encode(D, Xh.to(DEV), w.s)
     torch.cuda.synchronize()
     assert np.array_equal(_np_idx(oi), _np_idx(idx)) and torch.equal(oc, coef.cpu())
+    # and back: host codes in, host X_hat out, equal to the device entry point bit for bit
+    xh_host = torch.empty((w.M, w.d), dtype=torch.bfloat16).pin_memory()
+    csr.csr_reconstruct_host(D, oi, oc, xh_host)
+    xh_dev = csr.csr_reconstruct(D, idx, coef)
+    torch.cuda.synchronize()
+    assert torch.equal(xh_host.view(torch.int16), xh_dev.cpu().view(torch.int16))
+    xh32 = torch.empty((w.M, w.d), dtype=torch.float32)          # pageable memory and fp32 output work too
+    csr.csr_reconstruct_host(D, oi, oc, xh32)
+    assert torch.equal(xh32, csr.csr_reconstruct_ex(D, idx, coef, out_dtype=torch.float32).cpu())
