@@ -86,6 +86,9 @@ typedef struct csr_encode_params {
     void* workspace;        /* scratch of at least csr_encode_workspace_bytes(); NULL = the
                                library keeps one grow-only allocation per device */
     size_t workspace_bytes;
+    int64_t ldx;            /* elements between consecutive rows of X; 0 = d (dense) */
+    int64_t ld_code;        /* elements between consecutive rows of out_idx and of out_coef;
+                               0 = s (dense) */
 } csr_encode_params_t;
 
 typedef struct csr_reconstruct_params {
@@ -101,6 +104,8 @@ typedef struct csr_reconstruct_params {
     int32_t reserved1;
     void* X_hat;            /* [M][d], out_dtype */
     void* stream;
+    int64_t ld_code;        /* elements between consecutive rows of idx and of coef; 0 = s */
+    int64_t ld_xhat;        /* elements between consecutive rows of X_hat; 0 = d */
 } csr_reconstruct_params_t;
 
 /*
@@ -133,6 +138,39 @@ int64_t csr_encode_workspace_bytes(int mode, int d, int N);
 int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_t M, int d, int N,
                     int s, void* X_hat);
 int csr_reconstruct_ex(const csr_reconstruct_params_t* p);
+
+/*
+ * Row strides ("KV Decomposition and Sparse Storage": a head vector of d_h channels may be
+ * split into s_n chunks of d = d_h / s_n channels, each with its own dictionary).  With
+ * ldx = d_h and X pointing at channel c*d of row 0, csr_encode_ex encodes chunk c of every
+ * head vector in place; with ld_code = s_n*s and out_idx / out_coef pointing at entry c*s,
+ * the s codes of chunk c land in columns c*s .. c*s+s-1 of [M][s_n*s] code arrays; the
+ * reconstruct strides are the mirror image.  Requirements: ldx >= d, ld_code >= s,
+ * ld_xhat >= d; every row of X and of X_hat must start on a 16-byte boundary; out_idx, idx,
+ * out_coef and coef need only the alignment of their element type when ld_code is given
+ * (dense code arrays must be 16-byte aligned as before).  The host entry points take
+ * dense arrays only.
+ *
+ * Several problems in one call (one dictionary per layer, per K / V, per chunk): the
+ * problems are validated first, all of them, and nothing is enqueued if one is invalid;
+ * then they are enqueued in order on their streams.  Returns the first failure.
+ */
+int csr_encode_grouped(const csr_encode_params_t* problems, int count);
+int csr_reconstruct_grouped(const csr_reconstruct_params_t* problems, int count);
+
+/*
+ * Online part of a dictionary ("Build dictionary": besides the offline atoms a prompt's
+ * dictionary holds atoms sampled from the KV cache just computed; atoms are kept at unit
+ * l2-norm, the ReNorm step of "NeuralDict").  For i = 0 .. n_rows-1:
+ *     D[N_cur + i][:] = X[rows[i]][:] / ||X[rows[i]][:]||_2        (fp32; norm accumulated in fp32)
+ * A row whose norm is zero gives a zero atom (which matching pursuit never selects for a
+ * non-zero residual).  Which rows are sampled is the caller's choice: `rows` is a DEVICE
+ * array of n_rows row numbers in [0, M).  D is the caller's [N_cap][d] fp32 device array of
+ * which rows [0, N_cur) are in use; N_cur + n_rows <= N_cap is required.  X is [M][d] with
+ * x_dtype F32 or BF16 and row stride ldx (0 = d).  Asynchronous on `stream`.
+ */
+int csr_dict_append(void* D, int N_cur, int N_cap, int d, const void* X, int x_dtype, int64_t M, int64_t ldx,
+                    const int64_t* rows, int n_rows, void* stream);
 
 /*
  * Encode with HOST buffers (the same operation as csr_encode_ex; only X, out_idx and

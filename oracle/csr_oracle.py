@@ -102,6 +102,42 @@ def reconstruct(D: np.ndarray, idx: np.ndarray, coef: np.ndarray) -> np.ndarray:
     return out
 
 
+# --- chunks and the online part of a dictionary -------------------------------------------
+
+def mp_encode_chunked(Ds, X: np.ndarray, s: int):
+    """"KV Decomposition and Sparse Storage" with s_n = len(Ds) chunks: a head vector of d_h
+    channels is cut into s_n consecutive pieces of d_h / s_n channels and piece c is encoded
+    by matching pursuit over its own dictionary Ds[c] ([N_c][d_h / s_n]).  Returns one
+    MPResult per chunk."""
+    s_n = len(Ds)
+    d_h = X.shape[1]
+    if s_n < 1 or d_h % s_n:
+        raise ValueError("d_h must be a multiple of the number of chunks")
+    dc = d_h // s_n
+    return [mp_encode(Ds[c], np.ascontiguousarray(X[:, c * dc:(c + 1) * dc]), s) for c in range(s_n)]
+
+
+def reconstruct_chunked(Ds, idx_list, coef_list) -> np.ndarray:
+    """Eq. 12 per chunk; the pieces are put back side by side."""
+    return np.concatenate([reconstruct(Ds[c], idx_list[c], coef_list[c]) for c in range(len(Ds))], axis=1)
+
+
+def dict_append(D: np.ndarray, N_cur: int, X: np.ndarray, rows) -> np.ndarray:
+    """Online part of a dictionary ("Build dictionary": atoms sampled from the KV cache just
+    computed; "NeuralDict": ReNorm keeps every atom at unit l2-norm).  Returns a copy of D
+    ([N_cap][d] fp32) in which rows N_cur .. N_cur+len(rows)-1 are X[rows] divided by their
+    l2-norm, computed in fp64 and rounded once to fp32; a zero row stays zero."""
+    D = np.array(D, dtype=np.float32, copy=True)
+    rows = np.asarray(rows, dtype=np.int64)
+    if N_cur < 0 or N_cur + rows.size > D.shape[0]:
+        raise ValueError("atoms do not fit")
+    for i, r in enumerate(rows):
+        x = np.asarray(X[r], np.float64)
+        n = np.sqrt(np.sum(x * x))
+        D[N_cur + i] = (x / n if n > 0 else x * 0).astype(np.float32)
+    return D
+
+
 # --- storage format ("Analysis for CSR") -------------------------------------------------
 
 def pack_codes(idx: np.ndarray, coef: np.ndarray):

@@ -33,7 +33,8 @@ CSR_MODE_BF16_FAST = 1
 
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
-    "csr_encode_host", "csr_reconstruct_host", "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
+    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append",
+    "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
 
@@ -46,6 +47,7 @@ class csr_encode_params_t(ctypes.Structure):
         ("d", ctypes.c_int32), ("N", ctypes.c_int32), ("s", ctypes.c_int32), ("reserved0", ctypes.c_int32),
         ("out_idx", ctypes.c_void_p), ("out_coef", ctypes.c_void_p),
         ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("ldx", ctypes.c_int64), ("ld_code", ctypes.c_int64),
     ]
 
 
@@ -57,6 +59,7 @@ class csr_reconstruct_params_t(ctypes.Structure):
         ("M", ctypes.c_int64),
         ("d", ctypes.c_int32), ("N", ctypes.c_int32), ("s", ctypes.c_int32), ("reserved1", ctypes.c_int32),
         ("X_hat", ctypes.c_void_p), ("stream", ctypes.c_void_p),
+        ("ld_code", ctypes.c_int64), ("ld_xhat", ctypes.c_int64),
     ]
 
 
@@ -94,6 +97,12 @@ def lib() -> ctypes.CDLL:
         L.csr_reconstruct_ex.restype = i32
         L.csr_reconstruct_host.argtypes = [ctypes.POINTER(csr_reconstruct_params_t)]
         L.csr_reconstruct_host.restype = i32
+        L.csr_encode_grouped.argtypes = [ctypes.POINTER(csr_encode_params_t), i32]
+        L.csr_encode_grouped.restype = i32
+        L.csr_reconstruct_grouped.argtypes = [ctypes.POINTER(csr_reconstruct_params_t), i32]
+        L.csr_reconstruct_grouped.restype = i32
+        L.csr_dict_append.argtypes = [vp, i32, i32, i32, vp, i32, i64, i64, vp, i32, vp]
+        L.csr_dict_append.restype = i32
         L.csr_device_status.argtypes = [vp]
         L.csr_device_status.restype = i32
         L.csr_release_workspace.argtypes = []
@@ -148,6 +157,11 @@ def _encode_params(D, X, s, out_idx, out_coef, mode, stream, workspace) -> csr_e
     p.out_idx = out_idx.data_ptr()
     p.out_coef = out_coef.data_ptr()
     p.stream = stream
+    if X.dim() == 2 and X.shape[0] > 1 and X.stride(0) != X.shape[1]:
+        p.ldx = X.stride(0)
+    if out_idx.shape[0] > 1 and out_idx.stride(0) != s:
+        assert out_coef.stride(0) == out_idx.stride(0), "out_idx and out_coef must share their row stride"
+        p.ld_code = out_idx.stride(0)
     if workspace is not None:
         p.workspace = workspace.data_ptr()
         p.workspace_bytes = workspace.numel() * workspace.element_size()
@@ -160,8 +174,8 @@ def csr_encode_ex(D: torch.Tensor, X: torch.Tensor, s: int, *, mode: int = CSR_M
                   workspace: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """csr_encode_ex on CUDA tensors: D [N][d] fp32, X [M][d] fp32 or bf16.
     Returns (idx [M][s] uint16, coef [M][s] coef_dtype); runs on torch's current stream."""
-    assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.is_contiguous()
-    assert D.dtype == torch.float32 and X.dim() == 2 and D.dim() == 2 and X.shape[1] == D.shape[1]
+    assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.dim() == 2 and X.stride(1) == 1
+    assert D.dtype == torch.float32 and D.dim() == 2 and X.shape[1] == D.shape[1]
     M = X.shape[0]
     if out_idx is None:
         out_idx = torch.empty((M, s), dtype=torch.uint16, device=X.device)
@@ -216,17 +230,15 @@ def csr_encode_host(D: torch.Tensor, X_host: torch.Tensor, s: int, out_idx_host:
         _check(lib().csr_encode_host(ctypes.byref(p)))
 
 
-def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *,
-                       out_dtype: torch.dtype = torch.bfloat16,
-                       X_hat: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """csr_reconstruct_ex on CUDA tensors; returns X_hat [M][d]."""
+def _reconstruct_params(D, idx, coef, out_dtype, X_hat):
     assert D.is_cuda and idx.is_cuda and coef.is_cuda
-    assert D.is_contiguous() and idx.is_contiguous() and coef.is_contiguous()
+    assert D.is_contiguous() and idx.stride(1) == 1 and coef.stride(1) == 1
     assert D.dtype == torch.float32 and idx.dtype == torch.uint16 and idx.shape == coef.shape
     M, s = idx.shape
     N, d = D.shape
     if X_hat is None:
         X_hat = torch.empty((M, d), dtype=out_dtype, device=D.device)
+    assert tuple(X_hat.shape) == (M, d) and X_hat.stride(1) == 1
     p = csr_reconstruct_params_t()
     p.struct_size = ctypes.sizeof(csr_reconstruct_params_t)
     p.D = D.data_ptr()
@@ -237,6 +249,56 @@ def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *
     p.M, p.d, p.N, p.s = M, d, N, s
     p.X_hat = X_hat.data_ptr()
     p.stream = _stream_ptr(D)
+    if M > 1 and idx.stride(0) != s:
+        assert coef.stride(0) == idx.stride(0), "idx and coef must share their row stride"
+        p.ld_code = idx.stride(0)
+    if M > 1 and X_hat.stride(0) != d:
+        p.ld_xhat = X_hat.stride(0)
+    return p, X_hat
+
+
+def csr_encode_grouped(problems, *, mode: int = CSR_MODE_BF16_FAST) -> None:
+    """csr_encode_grouped: `problems` is a sequence of (D, X, s, out_idx, out_coef) with CUDA
+    tensors; X, out_idx and out_coef may be column slices of wider arrays (row strides are
+    passed on).  All problems are validated before any is enqueued."""
+    arr = (csr_encode_params_t * len(problems))()
+    for i, (D, X, s, out_idx, out_coef) in enumerate(problems):
+        assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.stride(1) == 1 and D.dtype == torch.float32
+        assert out_idx.dtype == torch.uint16 and out_idx.stride(1) == 1 and out_coef.stride(1) == 1
+        arr[i] = _encode_params(D, X, s, out_idx, out_coef, mode, _stream_ptr(X), None)
+    if len(problems):
+        with torch.cuda.device(problems[0][0].device):
+            _check(lib().csr_encode_grouped(arr, len(problems)))
+
+
+def csr_reconstruct_grouped(problems) -> None:
+    """csr_reconstruct_grouped: `problems` is a sequence of (D, idx, coef, X_hat)."""
+    arr = (csr_reconstruct_params_t * len(problems))()
+    for i, (D, idx, coef, X_hat) in enumerate(problems):
+        arr[i], _ = _reconstruct_params(D, idx, coef, X_hat.dtype, X_hat)
+    if len(problems):
+        with torch.cuda.device(problems[0][0].device):
+            _check(lib().csr_reconstruct_grouped(arr, len(problems)))
+
+
+def csr_dict_append(D: torch.Tensor, N_cur: int, X: torch.Tensor, rows: torch.Tensor) -> int:
+    """csr_dict_append: writes normalised copies of X[rows] as atoms N_cur .. N_cur+len(rows)-1 of
+    D ([N_cap][d] fp32, CUDA); rows is an int64 CUDA tensor.  Returns the new atom count."""
+    assert D.is_cuda and X.is_cuda and rows.is_cuda and D.is_contiguous() and D.dtype == torch.float32
+    assert X.dim() == 2 and X.stride(1) == 1 and rows.dtype == torch.int64 and rows.is_contiguous()
+    n = int(rows.numel())
+    with torch.cuda.device(D.device):
+        _check(lib().csr_dict_append(D.data_ptr(), N_cur, D.shape[0], D.shape[1], X.data_ptr(), _TORCH_DTYPE[X.dtype],
+                                     X.shape[0], X.stride(0) if X.shape[0] > 1 else 0, rows.data_ptr(), n,
+                                     _stream_ptr(D)))
+    return N_cur + n
+
+
+def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *,
+                       out_dtype: torch.dtype = torch.bfloat16,
+                       X_hat: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """csr_reconstruct_ex on CUDA tensors; returns X_hat [M][d]."""
+    p, X_hat = _reconstruct_params(D, idx, coef, out_dtype, X_hat)
     with torch.cuda.device(D.device):
         _check(lib().csr_reconstruct_ex(ctypes.byref(p)))
     return X_hat

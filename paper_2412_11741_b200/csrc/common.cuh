@@ -25,6 +25,8 @@ struct EncodeArgs {
     int d, N, s;
     uint16_t* out_idx;
     void* out_coef;
+    int64_t ldx;       // elements between consecutive rows of X (>= d)
+    int64_t ld_code;   // elements between consecutive rows of out_idx and of out_coef (>= s)
     cudaStream_t stream;
 };
 
@@ -45,9 +47,15 @@ struct ReconstructArgs {
     int64_t M;
     int d, N, s;
     void* X_hat;
+    int64_t ld_code;   // elements between consecutive rows of idx and of coef (>= s)
+    int64_t ld_xhat;   // elements between consecutive rows of X_hat (>= d)
     cudaStream_t stream;
 };
 int launch_reconstruct(const ReconstructArgs& a);
+
+// D_new[i][:] = X[rows[i]][:] / ||X[rows[i]][:]||_2 for i < n_rows (zero rows stay zero).
+int launch_dict_append(float* D_new, int d, const void* X, int x_dtype, int64_t M, int64_t ldx, const int64_t* rows,
+                       int n_rows, cudaStream_t stream);
 
 int sm_count();
 

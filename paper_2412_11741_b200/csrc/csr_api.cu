@@ -112,8 +112,22 @@ int check_encode(const csr_encode_params_t* p, bool host_io) {
     if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
     if (p->M > 0 && (!p->X || !p->out_idx || !p->out_coef))
         return fail(CSR_ERR_INVALID_ARG, "X, out_idx or out_coef is NULL");
-    if (!aligned16(p->D) || (!host_io && (!aligned16(p->X) || !aligned16(p->out_idx) || !aligned16(p->out_coef))))
-        return fail(CSR_ERR_ALIGNMENT, "D, X, out_idx and out_coef must be 16-byte aligned");
+    if (p->ldx < 0 || p->ld_code < 0 || (p->ldx && p->ldx < p->d) || (p->ld_code && p->ld_code < p->s))
+        return fail(CSR_ERR_INVALID_ARG, "ldx (%lld) must be 0 or >= d, ld_code (%lld) 0 or >= s", (long long)p->ldx,
+                    (long long)p->ld_code);
+    if (host_io && (p->ldx || p->ld_code)) return fail(CSR_ERR_UNSUPPORTED, "the host entry points take dense arrays");
+    if (!aligned16(p->D)) return fail(CSR_ERR_ALIGNMENT, "D must be 16-byte aligned");
+    if (!host_io) {
+        const size_t xe = p->x_dtype == CSR_DTYPE_BF16 ? 2 : 4, ce = p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4;
+        if (!aligned16(p->X) || (p->ldx && (p->ldx * xe) % 16 != 0))
+            return fail(CSR_ERR_ALIGNMENT, "every row of X must start on a 16-byte boundary");
+        if (p->ld_code == 0) {
+            if (!aligned16(p->out_idx) || !aligned16(p->out_coef))
+                return fail(CSR_ERR_ALIGNMENT, "dense out_idx and out_coef must be 16-byte aligned");
+        } else if ((reinterpret_cast<uintptr_t>(p->out_idx) % 2) || (reinterpret_cast<uintptr_t>(p->out_coef) % ce)) {
+            return fail(CSR_ERR_ALIGNMENT, "out_idx / out_coef are not aligned to their element type");
+        }
+    }
     if (p->workspace && !aligned16(p->workspace)) return fail(CSR_ERR_ALIGNMENT, "workspace must be 16-byte aligned");
     return CSR_OK;
 }
@@ -173,8 +187,22 @@ int check_reconstruct(const csr_reconstruct_params_t* p, bool host_io) {
         return fail(CSR_ERR_INVALID_ARG, "out_dtype must be F32 or BF16");
     if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
     if (p->M > 0 && (!p->idx || !p->coef || !p->X_hat)) return fail(CSR_ERR_INVALID_ARG, "idx, coef or X_hat is NULL");
-    if (!aligned16(p->D) || (!host_io && (!aligned16(p->idx) || !aligned16(p->coef) || !aligned16(p->X_hat))))
-        return fail(CSR_ERR_ALIGNMENT, "D, idx, coef and X_hat must be 16-byte aligned");
+    if (p->ld_code < 0 || p->ld_xhat < 0 || (p->ld_code && p->ld_code < p->s) || (p->ld_xhat && p->ld_xhat < p->d))
+        return fail(CSR_ERR_INVALID_ARG, "ld_code (%lld) must be 0 or >= s, ld_xhat (%lld) 0 or >= d",
+                    (long long)p->ld_code, (long long)p->ld_xhat);
+    if (host_io && (p->ld_code || p->ld_xhat)) return fail(CSR_ERR_UNSUPPORTED, "the host entry points take dense arrays");
+    if (!aligned16(p->D)) return fail(CSR_ERR_ALIGNMENT, "D must be 16-byte aligned");
+    if (!host_io) {
+        const size_t xe = p->out_dtype == CSR_DTYPE_BF16 ? 2 : 4, ce = p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4;
+        if (!aligned16(p->X_hat) || (p->ld_xhat && (p->ld_xhat * xe) % 16 != 0))
+            return fail(CSR_ERR_ALIGNMENT, "every row of X_hat must start on a 16-byte boundary");
+        if (p->ld_code == 0) {
+            if (!aligned16(p->idx) || !aligned16(p->coef))
+                return fail(CSR_ERR_ALIGNMENT, "dense idx and coef must be 16-byte aligned");
+        } else if ((reinterpret_cast<uintptr_t>(p->idx) % 2) || (reinterpret_cast<uintptr_t>(p->coef) % ce)) {
+            return fail(CSR_ERR_ALIGNMENT, "idx / coef are not aligned to their element type");
+        }
+    }
     return CSR_OK;
 }
 
@@ -190,6 +218,8 @@ ReconstructArgs reconstruct_args(const csr_reconstruct_params_t* p) {
     a.N = p->N;
     a.s = p->s;
     a.X_hat = p->X_hat;
+    a.ld_code = p->ld_code ? p->ld_code : p->s;
+    a.ld_xhat = p->ld_xhat ? p->ld_xhat : p->d;
     a.stream = static_cast<cudaStream_t>(p->stream);
     return a;
 }
@@ -213,6 +243,8 @@ int encode_device(const csr_encode_params_t* p) {
     a.s = p->s;
     a.out_idx = p->out_idx;
     a.out_coef = p->out_coef;
+    a.ldx = p->ldx ? p->ldx : p->d;
+    a.ld_code = p->ld_code ? p->ld_code : p->s;
     a.stream = static_cast<cudaStream_t>(p->stream);
     if (p->mode == CSR_MODE_FP32_EXACT) return launch_encode_exact(a);
 
@@ -295,6 +327,41 @@ int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_
     p.s = s;
     p.X_hat = X_hat;
     return csr_reconstruct_ex(&p);
+}
+
+int csr_encode_grouped(const csr_encode_params_t* problems, int count) {
+    if (count < 0 || (count > 0 && !problems)) return fail(CSR_ERR_INVALID_ARG, "problems is NULL or count < 0");
+    for (int i = 0; i < count; ++i)
+        if (int rc = check_encode(&problems[i], false)) return rc;
+    for (int i = 0; i < count; ++i)
+        if (int rc = encode_device(&problems[i])) return rc;
+    return CSR_OK;
+}
+
+int csr_reconstruct_grouped(const csr_reconstruct_params_t* problems, int count) {
+    if (count < 0 || (count > 0 && !problems)) return fail(CSR_ERR_INVALID_ARG, "problems is NULL or count < 0");
+    for (int i = 0; i < count; ++i)
+        if (int rc = check_reconstruct(&problems[i], false)) return rc;
+    for (int i = 0; i < count; ++i)
+        if (int rc = launch_reconstruct(reconstruct_args(&problems[i]))) return rc;
+    return CSR_OK;
+}
+
+int csr_dict_append(void* D, int N_cur, int N_cap, int d, const void* X, int x_dtype, int64_t M, int64_t ldx,
+                    const int64_t* rows, int n_rows, void* stream) {
+    if (d != 64 && d != 128) return fail(CSR_ERR_UNSUPPORTED, "d = %d: only 64 and 128 are supported", d);
+    if (N_cap < 1 || N_cap > 65536 || N_cur < 0 || n_rows < 0 || (int64_t)N_cur + n_rows > N_cap)
+        return fail(CSR_ERR_INVALID_ARG, "N_cur = %d, n_rows = %d do not fit N_cap = %d (<= 65536)", N_cur, n_rows, N_cap);
+    if (x_dtype != CSR_DTYPE_F32 && x_dtype != CSR_DTYPE_BF16) return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32 or BF16");
+    if (M < 0 || ldx < 0 || (ldx && ldx < d)) return fail(CSR_ERR_INVALID_ARG, "M < 0 or ldx not 0 or >= d");
+    if (n_rows == 0) return CSR_OK;
+    if (!D || !X || !rows) return fail(CSR_ERR_INVALID_ARG, "D, X or rows is NULL");
+    if (M == 0) return fail(CSR_ERR_INVALID_ARG, "rows given but X is empty");
+    const size_t xe = x_dtype == CSR_DTYPE_BF16 ? 2 : 4;
+    if (!aligned16(D) || !aligned16(X) || (ldx && (ldx * xe) % 16 != 0) || (reinterpret_cast<uintptr_t>(rows) % 8))
+        return fail(CSR_ERR_ALIGNMENT, "D and every row of X must be 16-byte aligned, rows 8-byte aligned");
+    return launch_dict_append(static_cast<float*>(D) + (size_t)N_cur * d, d, X, x_dtype, M, ldx ? ldx : d, rows, n_rows,
+                              static_cast<cudaStream_t>(stream));
 }
 
 int csr_encode_host(const csr_encode_params_t* p) {

@@ -72,8 +72,8 @@ __device__ __forceinline__ void top2_merge(Top2& t, float ob, float os, int oi) 
 
 template <int D_>
 __global__ void __launch_bounds__(NT, 1)
-encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int x_dtype, int64_t M, int N, int s,
-                    uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype) {
+encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int x_dtype, int64_t ldx, int64_t M, int N,
+                    int s, uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype, int64_t ldc) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Smem<D_>& sm = *reinterpret_cast<Smem<D_>*>(smem_raw);
 
@@ -94,7 +94,7 @@ encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int
             const int64_t m = row0 + r;
             double nn = 0.0;
             for (int k = lane; k < D_; k += 32) {
-                float v = (m < M) ? load_x(X, x_dtype, m * D_ + k) : 0.f;
+                float v = (m < M) ? load_x(X, x_dtype, m * ldx + k) : 0.f;
                 sm.Rd[r][k] = (double)v;
                 sm.As[k][r] = v;
                 nn += (double)v * (double)v;
@@ -246,12 +246,12 @@ encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int
                 for (int o = 16; o; o >>= 1) nn += __shfl_xor_sync(0xffffffffu, nn, o);
                 if (lane == 0) {
                     sm.band[r] = kBandRel * (float)sqrt(nn);
-                    out_idx[m * s + g] = (uint16_t)bi;
+                    out_idx[m * ldc + g] = (uint16_t)bi;
                     const float cf = (float)c;
                     if (coef_dtype == CSR_DTYPE_F16)
-                        reinterpret_cast<__half*>(out_coef)[m * s + g] = __float2half_rn(cf);
+                        reinterpret_cast<__half*>(out_coef)[m * ldc + g] = __float2half_rn(cf);
                     else
-                        reinterpret_cast<float*>(out_coef)[m * s + g] = cf;
+                        reinterpret_cast<float*>(out_coef)[m * ldc + g] = cf;
                 }
             }
             __syncthreads();
@@ -270,14 +270,14 @@ int launch_encode_exact(const EncodeArgs& a) {
         const size_t smem = sizeof(Smem<128>);
         e = cudaFuncSetAttribute(encode_exact_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        encode_exact_kernel<128><<<grid, NT, smem, a.stream>>>(a.D, a.X, a.x_dtype, a.M, a.N, a.s, a.out_idx,
-                                                               a.out_coef, a.coef_dtype);
+        encode_exact_kernel<128><<<grid, NT, smem, a.stream>>>(a.D, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s,
+                                                               a.out_idx, a.out_coef, a.coef_dtype, a.ld_code);
     } else {
         const size_t smem = sizeof(Smem<64>);
         e = cudaFuncSetAttribute(encode_exact_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        encode_exact_kernel<64><<<grid, NT, smem, a.stream>>>(a.D, a.X, a.x_dtype, a.M, a.N, a.s, a.out_idx,
-                                                              a.out_coef, a.coef_dtype);
+        encode_exact_kernel<64><<<grid, NT, smem, a.stream>>>(a.D, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s,
+                                                              a.out_idx, a.out_coef, a.coef_dtype, a.ld_code);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "encode_exact launch: %s", cudaGetErrorString(e));

@@ -403,8 +403,9 @@ __global__ void dict_to_bf16_kernel(const float4* __restrict__ src, uint2* __res
 template <int D_, int G>
 __global__ void __launch_bounds__(NT, 1)
 encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* __restrict__ Db,
-                   const void* __restrict__ X, int x_dtype, int64_t M, int N, int s, uint16_t* __restrict__ out_idx,
-                   void* __restrict__ out_coef, int coef_dtype, uint32_t key_mask, uint32_t* status) {
+                   const void* __restrict__ X, int x_dtype, int64_t ldx, int64_t M, int N, int s,
+                   uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype, int64_t ldc, int vec_codes,
+                   uint32_t key_mask, uint32_t* status) {
     using S = FastSmem<D_>;
     extern __shared__ uint8_t smem_raw[];
     S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -542,7 +543,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             const bool valid = m < M;
             // ---- R_0 = x, rounded to bf16, into the operand tile ----
             if (x_dtype == CSR_DTYPE_BF16) {
-                const uint4* src = reinterpret_cast<const uint4*>(X) + m * CHUNKS;
+                const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(X) + m * ldx);
 #pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
                     uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -550,7 +551,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     *reinterpret_cast<uint4*>(Atile + swz_off(r, c)) = v;
                 }
             } else {
-                const float4* src = reinterpret_cast<const float4*>(X) + m * (CHUNKS * 2);
+                const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X) + m * ldx);
 #pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
                     float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
@@ -630,8 +631,8 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 // ---- flush the collected codes eight at a time ----
                 if ((gi == CODE_BLOCK - 1 || g == s - 1) && valid) {
                     const int g0 = g - gi;
-                    const int64_t o = m * s + g0;
-                    if (gi == CODE_BLOCK - 1 && (s & 7) == 0) {
+                    const int64_t o = m * ldc + g0;
+                    if (gi == CODE_BLOCK - 1 && vec_codes) {
                         *reinterpret_cast<uint4*>(out_idx + o) = *reinterpret_cast<const uint4*>(&sm.code_idx[slot][0]);
                         const float4 f0 = *reinterpret_cast<const float4*>(&sm.code_coef[slot][0]);
                         const float4 f1 = *reinterpret_cast<const float4*>(&sm.code_coef[slot][4]);
@@ -700,8 +701,12 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
     // keys keep the magnitude bits above the group tag; with G == 1 the key is built from the
     // raw value, so the mask clears the sign bit as well
     const uint32_t key_mask = (G == 1 ? 0x7FFFFFFFu : 0xFFFFFFFFu) & ~static_cast<uint32_t>(TILE_N / G - 1);
-    encode_fast_kernel<D_, G><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.M, a.N, a.s, a.out_idx,
-                                                           a.out_coef, a.coef_dtype, key_mask, status);
+    // 16-byte code stores need eight codes per flush and 16-byte aligned rows in both arrays
+    const uintptr_t ci = reinterpret_cast<uintptr_t>(a.out_idx), cc = reinterpret_cast<uintptr_t>(a.out_coef);
+    const int vec_codes = (a.s % 8 == 0) && (a.ld_code % 8 == 0) && (ci % 16 == 0) && (cc % 16 == 0);
+    encode_fast_kernel<D_, G><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
+                                                           a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask,
+                                                           status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "encode_fast launch: %s", cudaGetErrorString(e));
     return CSR_OK;

@@ -92,6 +92,8 @@ extern "C" int csr_encode_static(const void* D, const void* X, int64_t M, int d,
     a.s = s;
     a.out_idx = out_idx;
     a.out_coef = out_coef;
+    a.ldx = d;
+    a.ld_code = s;
     a.stream = st;
     return launch_encode_fast(a, reinterpret_cast<void*>(dict), status);
 }

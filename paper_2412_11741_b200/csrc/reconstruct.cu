@@ -36,30 +36,32 @@ __device__ __forceinline__ void axpy(float2& a, float c, const float2& v) {
 __device__ __forceinline__ void zero(float4& a) { a = make_float4(0.f, 0.f, 0.f, 0.f); }
 __device__ __forceinline__ void zero(float2& a) { a = make_float2(0.f, 0.f); }
 
-__device__ __forceinline__ void store_out(void* out, int out_dtype, int64_t row, int lane, const float4& a) {
+// `off` is the element offset of the row inside X_hat; the lane writes its 4 (or 2) channels.
+__device__ __forceinline__ void store_out(void* out, int out_dtype, int64_t off, int lane, const float4& a) {
     if (out_dtype == CSR_DTYPE_BF16) {
         __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
         uint2 u;
         u.x = *reinterpret_cast<uint32_t*>(&lo);
         u.y = *reinterpret_cast<uint32_t*>(&hi);
-        reinterpret_cast<uint2*>(out)[row * 32 + lane] = u;
+        reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + off)[lane] = u;
     } else {
-        reinterpret_cast<float4*>(out)[row * 32 + lane] = a;
+        reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + off)[lane] = a;
     }
 }
-__device__ __forceinline__ void store_out(void* out, int out_dtype, int64_t row, int lane, const float2& a) {
+__device__ __forceinline__ void store_out(void* out, int out_dtype, int64_t off, int lane, const float2& a) {
     if (out_dtype == CSR_DTYPE_BF16) {
         __nv_bfloat162 v = __floats2bfloat162_rn(a.x, a.y);
-        reinterpret_cast<uint32_t*>(out)[row * 32 + lane] = *reinterpret_cast<uint32_t*>(&v);
+        reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(out) + off)[lane] = *reinterpret_cast<uint32_t*>(&v);
     } else {
-        reinterpret_cast<float2*>(out)[row * 32 + lane] = a;
+        reinterpret_cast<float2*>(reinterpret_cast<float*>(out) + off)[lane] = a;
     }
 }
 
 template <int D_>
 __global__ void __launch_bounds__(NT)
 reconstruct_kernel(const float* __restrict__ D, const uint16_t* __restrict__ idx, const void* __restrict__ coef,
-                   int coef_dtype, int64_t M, int N, int s, void* __restrict__ X_hat, int out_dtype) {
+                   int coef_dtype, int64_t ldc, int64_t M, int N, int s, void* __restrict__ X_hat, int out_dtype,
+                   int64_t ldxh) {
     using V = typename Vec<D_>::T;
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = (int64_t)blockIdx.x * (NT / 32) + (threadIdx.x >> 5);
@@ -72,11 +74,11 @@ reconstruct_kernel(const float* __restrict__ D, const uint16_t* __restrict__ idx
         for (int h = 0; h < 2; ++h) {
             const int g = lane + 32 * h;
             if (g < s) {
-                int i = idx[m * s + g];
+                int i = idx[m * ldc + g];
                 my_i[h] = i < N ? i : N - 1;
                 my_c[h] = (coef_dtype == CSR_DTYPE_F16)
-                              ? __half2float(reinterpret_cast<const __half*>(coef)[m * s + g])
-                              : reinterpret_cast<const float*>(coef)[m * s + g];
+                              ? __half2float(reinterpret_cast<const __half*>(coef)[m * ldc + g])
+                              : reinterpret_cast<const float*>(coef)[m * ldc + g];
             }
         }
         V acc;
@@ -97,7 +99,7 @@ reconstruct_kernel(const float* __restrict__ D, const uint16_t* __restrict__ idx
             for (int u = 0; u < 4; ++u)
                 if (g0 + u < s) axpy(acc, c[u], v[u]);
         }
-        store_out(X_hat, out_dtype, m, lane, acc);
+        store_out(X_hat, out_dtype, m * ldxh, lane, acc);
     }
 }
 
@@ -110,11 +112,11 @@ int launch_reconstruct(const ReconstructArgs& a) {
     const int64_t cap = (int64_t)sm_count() * 8;
     if (blocks > cap) blocks = cap;
     if (a.d == 128)
-        reconstruct_kernel<128><<<(int)blocks, NT, 0, a.stream>>>(a.D, a.idx, a.coef, a.coef_dtype, a.M, a.N, a.s,
-                                                                  a.X_hat, a.out_dtype);
+        reconstruct_kernel<128><<<(int)blocks, NT, 0, a.stream>>>(a.D, a.idx, a.coef, a.coef_dtype, a.ld_code, a.M,
+                                                                  a.N, a.s, a.X_hat, a.out_dtype, a.ld_xhat);
     else
-        reconstruct_kernel<64><<<(int)blocks, NT, 0, a.stream>>>(a.D, a.idx, a.coef, a.coef_dtype, a.M, a.N, a.s,
-                                                                 a.X_hat, a.out_dtype);
+        reconstruct_kernel<64><<<(int)blocks, NT, 0, a.stream>>>(a.D, a.idx, a.coef, a.coef_dtype, a.ld_code, a.M,
+                                                                 a.N, a.s, a.X_hat, a.out_dtype, a.ld_xhat);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "reconstruct launch: %s", cudaGetErrorString(e));
     return CSR_OK;

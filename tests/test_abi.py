@@ -35,8 +35,8 @@ def test_exports_match_header(lib):
 def test_version_and_struct_sizes(lib):
     from paper_2412_11741_b200 import binding
     assert binding.csr_version() == 100
-    assert ctypes.sizeof(binding.csr_encode_params_t) == 96
-    assert ctypes.sizeof(binding.csr_reconstruct_params_t) == 80
+    assert ctypes.sizeof(binding.csr_encode_params_t) == 112
+    assert ctypes.sizeof(binding.csr_reconstruct_params_t) == 96
 
 
 def _params(binding, **kw):
@@ -81,6 +81,26 @@ def test_reconstruct_argument_errors(lib):
     assert lib.csr_reconstruct(0x1000, 0x2000, 0x3000, 10, 128, 1024, 0, 0x4000) == binding.CSR_ERR_INVALID_ARG
     assert lib.csr_reconstruct(0x1000, 0x2002, 0x3000, 10, 128, 1024, 8, 0x4000) == binding.CSR_ERR_ALIGNMENT
     assert lib.csr_reconstruct(0, 0x2000, 0x3000, 10, 128, 1024, 8, 0x4000) == binding.CSR_ERR_INVALID_ARG
+
+
+def test_stride_and_group_argument_errors(lib):
+    from paper_2412_11741_b200 import binding
+    assert lib.csr_encode_ex(ctypes.byref(_params(binding, ldx=64))) == binding.CSR_ERR_INVALID_ARG      # < d
+    assert lib.csr_encode_ex(ctypes.byref(_params(binding, ld_code=4))) == binding.CSR_ERR_INVALID_ARG   # < s
+    assert lib.csr_encode_ex(ctypes.byref(_params(binding, ldx=132))) == binding.CSR_ERR_ALIGNMENT       # rows off 16 B
+    assert lib.csr_encode_host(ctypes.byref(_params(binding, ldx=256))) == binding.CSR_ERR_UNSUPPORTED
+    assert lib.csr_encode_grouped(None, 1) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_encode_grouped(None, 0) == binding.CSR_OK
+    arr = (binding.csr_encode_params_t * 2)(_params(binding, M=0, X=0, out_idx=0, out_coef=0), _params(binding, d=96))
+    assert lib.csr_encode_grouped(arr, 2) == binding.CSR_ERR_UNSUPPORTED      # second problem invalid: nothing runs
+    assert lib.csr_reconstruct_grouped(None, 0) == binding.CSR_OK
+    # dict_append: capacity, dtype and alignment are checked before any device work
+    f = lib.csr_dict_append
+    assert f(0x1000, 10, 16, 128, 0x2000, 0, 100, 0, 0x3000, 7, None) == binding.CSR_ERR_INVALID_ARG    # 10 + 7 > 16
+    assert f(0x1000, 0, 16, 96, 0x2000, 0, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_UNSUPPORTED
+    assert f(0x1000, 0, 16, 128, 0x2000, 2, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_INVALID_ARG     # fp16 X
+    assert f(0x1000, 0, 16, 128, 0x2004, 0, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_ALIGNMENT
+    assert f(0x1000, 0, 16, 128, 0x2000, 0, 100, 0, 0x3000, 0, None) == binding.CSR_OK                  # nothing to add
 
 
 def test_workspace_query(lib):

@@ -1,0 +1,119 @@
+"""GPU parity of the chunked / multi-dictionary calls and of the online dictionary atoms
+("KV Decomposition and Sparse Storage", "Build dictionary") against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import csr_oracle as orc
+from paper_2412_11741_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _np_idx(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+@pytest.fixture(scope="module")
+def csr():
+    from paper_2412_11741_b200 import build
+    build.build()
+    import paper_2412_11741_b200 as pkg
+    return pkg
+
+
+def _value_cache(M, seed):
+    rng = np.random.default_rng(seed)
+    X = wl.round_to_bf16(rng.standard_normal((M, 128)).astype(np.float32))
+    Ds = [wl.normalise_rows(rng.standard_normal((1024, 64)).astype(np.float32)) for _ in range(2)]
+    return X, Ds
+
+
+@pytest.mark.parametrize("mode_name,s", [("exact", 4), ("fast", 4), ("fast", 8)])
+def test_two_chunks_with_their_own_dictionaries_in_place(csr, mode_name, s):
+    """Value cache with s_n = 2: both halves of every 128-channel head vector are encoded in
+    place (row stride 128) into one [M][2*s] code array by one grouped call, then restored
+    into one [M][128] array; each half must agree with the oracle's chunked pursuit."""
+    M = 3000
+    X, Ds = _value_cache(M, seed=s)
+    mode = csr.CSR_MODE_FP32_EXACT if mode_name == "exact" else csr.CSR_MODE_BF16_FAST
+    Xd = torch.from_numpy(X).to(DEV).to(torch.bfloat16)
+    Dd = [torch.from_numpy(D).to(DEV) for D in Ds]
+    idx = torch.zeros((M, 2 * s), dtype=torch.int16, device=DEV).view(torch.uint16)
+    coef = torch.zeros((M, 2 * s), dtype=torch.float32, device=DEV)
+    csr.csr_encode_grouped([(Dd[c], Xd[:, 64 * c:64 * (c + 1)], s, idx[:, s * c:s * (c + 1)], coef[:, s * c:s * (c + 1)])
+                            for c in range(2)], mode=mode)
+    assert csr.csr_device_status() == csr.CSR_OK
+    ref = orc.mp_encode_chunked(Ds, X, s)
+    gi, gc = _np_idx(idx), coef.cpu().numpy()
+    for c in range(2):
+        Xc = np.ascontiguousarray(X[:, 64 * c:64 * (c + 1)])
+        ic, cc = gi[:, s * c:s * (c + 1)], gc[:, s * c:s * (c + 1)]
+        rep = (parity.compare_exact if mode_name == "exact" else parity.compare_fast)(Ds[c], Xc, s, ic, cc, ref[c])
+        assert rep.ok, (c, rep.detail)
+        # in place == on a contiguous copy of the chunk, bit for bit
+        i2, c2 = csr.csr_encode_ex(Dd[c], Xd[:, 64 * c:64 * (c + 1)].contiguous(), s, mode=mode, coef_dtype=torch.float32)
+        assert np.array_equal(_np_idx(i2), ic) and np.array_equal(c2.cpu().numpy(), cc)
+    # restore both halves side by side
+    xh = torch.full((M, 128), 7.0, dtype=torch.float32, device=DEV)
+    csr.csr_reconstruct_grouped([(Dd[c], idx[:, s * c:s * (c + 1)], coef[:, s * c:s * (c + 1)], xh[:, 64 * c:64 * (c + 1)])
+                                 for c in range(2)])
+    want = orc.reconstruct_chunked(Ds, [gi[:, s * c:s * (c + 1)].astype(np.int32) for c in range(2)],
+                                   [gc[:, s * c:s * (c + 1)].astype(np.float64) for c in range(2)])
+    scale = np.abs(gc).sum(1, keepdims=True) + 1e-30
+    assert np.all(np.abs(xh.cpu().numpy() - want) <= 2e-6 * scale)
+
+
+def test_packed_codes_of_two_chunks_use_vector_stores_when_they_can(csr):
+    """s = 8 with fp16 coefficients: chunk c's codes start 16 bytes into the row, so the
+    16-byte store path is taken with a row stride; the result equals the dense call's."""
+    M, s = 1000, 8
+    X, Ds = _value_cache(M, seed=11)
+    Xd = torch.from_numpy(X).to(DEV).to(torch.bfloat16)
+    Dd = [torch.from_numpy(D).to(DEV) for D in Ds]
+    idx = torch.zeros((M, 2 * s), dtype=torch.int16, device=DEV).view(torch.uint16)
+    coef = torch.zeros((M, 2 * s), dtype=torch.float16, device=DEV)
+    csr.csr_encode_grouped([(Dd[c], Xd[:, 64 * c:64 * (c + 1)], s, idx[:, s * c:s * (c + 1)], coef[:, s * c:s * (c + 1)])
+                            for c in range(2)])
+    for c in range(2):
+        i2, c2 = csr.csr_encode(Dd[c], Xd[:, 64 * c:64 * (c + 1)].contiguous(), s)
+        assert np.array_equal(_np_idx(i2), _np_idx(idx)[:, s * c:s * (c + 1)])
+        assert torch.equal(c2.cpu(), coef[:, s * c:s * (c + 1)].cpu())
+
+
+@pytest.mark.parametrize("d,dtype", [(128, "bf16"), (64, "f32")])
+def test_online_atoms_match_oracle_and_are_used_by_the_encoder(csr, d, dtype):
+    """Sampled rows of the cache become unit-norm atoms behind the offline part; the encoder
+    then finds each sampled row's own atom first."""
+    rng = np.random.default_rng(d)
+    N_off, n_on, M = 896, 128, 5000
+    D0 = np.zeros((N_off + n_on, d), np.float32)
+    D0[:N_off] = wl.normalise_rows(rng.standard_normal((N_off, d)).astype(np.float32))
+    Xw = rng.standard_normal((M, 2 * d)).astype(np.float32)          # rows are slices of a wider array
+    Xw[17] = 0.0
+    if dtype == "bf16":
+        Xw = wl.round_to_bf16(Xw)
+    X = Xw[:, d:]
+    rows = rng.choice(M, n_on, replace=False).astype(np.int64)
+    rows[5] = 17                                                      # a zero row gives a zero atom
+    Dd = torch.from_numpy(D0).to(DEV)
+    Xd = torch.from_numpy(Xw).to(DEV)
+    if dtype == "bf16":
+        Xd = Xd.to(torch.bfloat16)
+    n_new = csr.csr_dict_append(Dd, N_off, Xd[:, d:], torch.from_numpy(rows).to(DEV))
+    assert n_new == N_off + n_on
+    got = Dd.cpu().numpy()
+    want = orc.dict_append(D0, N_off, X, rows)
+    assert np.array_equal(got[:N_off], D0[:N_off])
+    assert np.all(got[N_off + 5] == 0)
+    assert np.all(np.abs(got - want) <= 4e-7 * np.abs(want) + 1e-9)   # fp32 norm against fp64
+    # downstream: the oracle and the exact encoder, both on the GPU-built dictionary
+    sel = np.delete(rows, 5)[:64]
+    Xs = np.ascontiguousarray(X[sel])
+    i, c = csr.csr_encode_ex(Dd, torch.from_numpy(Xs).to(DEV), 3, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
+    rep = parity.compare_exact(got, Xs, 3, _np_idx(i), c.cpu().numpy())
+    assert rep.ok, rep.detail
+    own = N_off + np.array([int(np.flatnonzero(rows == r)[0]) for r in sel])
+    assert np.array_equal(_np_idx(i)[:, 0].astype(np.int64), own)

@@ -282,3 +282,65 @@ def test_pins_detect_unsigned_coefficient():
         e += c[i] ** 2
     # with an unsigned coefficient the energy identity breaks for this input
     assert abs((x ** 2).sum() - (R ** 2).sum() - e) > 1e-3
+
+
+# ---------------------------------------------------------------------------------------
+# chunks and the online part of a dictionary
+# ---------------------------------------------------------------------------------------
+
+def test_dict_append_closed_forms():
+    """3-4-0 triangle, unit norm, direction, scale invariance, zero row, untouched atoms."""
+    rng = np.random.default_rng(3)
+    D = np.zeros((6, 4), np.float32)
+    D[0] = [1, 0, 0, 0]
+    X = np.array([[3, 4, 0, 0], [0, 0, 0, 0], [-2, 0, 0, 0], [1, 1, 1, 1]], np.float32)
+    out = orc.dict_append(D, 1, X, [0, 1, 2, 3])
+    assert np.array_equal(out[0], D[0]) and np.array_equal(out[5], D[5])
+    assert np.allclose(out[1], [0.6, 0.8, 0, 0], rtol=0, atol=1e-7)
+    assert np.array_equal(out[2], np.zeros(4, np.float32))
+    assert np.array_equal(out[3], np.array([-1, 0, 0, 0], np.float32))
+    assert np.allclose(out[4], 0.5)
+    Y = rng.standard_normal((50, 64)).astype(np.float32)
+    E = orc.dict_append(np.zeros((50, 64), np.float32), 0, Y, np.arange(50))
+    assert np.allclose(np.linalg.norm(E.astype(np.float64), axis=1), 1.0, atol=1e-7)
+    cos = np.sum(E.astype(np.float64) * Y, axis=1) / np.linalg.norm(Y.astype(np.float64), axis=1)
+    assert np.allclose(cos, 1.0, atol=1e-7)
+    E2 = orc.dict_append(np.zeros((50, 64), np.float32), 0, Y * np.float32(8.0), np.arange(50))
+    assert np.array_equal(E, E2)                          # scaling by a power of two changes nothing
+    with pytest.raises(ValueError):
+        orc.dict_append(D, 4, X, [0, 1, 2])
+
+
+def test_an_appended_atom_encodes_its_own_row_in_one_step():
+    """A sampled row becomes an atom that represents it exactly: first pick = that atom,
+    coefficient = the row's norm, residual zero."""
+    rng = np.random.default_rng(4)
+    X = rng.standard_normal((8, 32)).astype(np.float32)
+    D0 = np.zeros((40, 32), np.float32)
+    D0[:32] = np.eye(32, dtype=np.float32)
+    D = orc.dict_append(D0, 32, X, np.arange(8))
+    res = orc.mp_encode(D, X, 1)
+    assert np.array_equal(res.idx[:, 0], 32 + np.arange(8))
+    assert np.allclose(res.coef[:, 0], np.linalg.norm(X.astype(np.float64), axis=1), rtol=1e-6)
+    assert np.all(res.resnorm[:, 0] < 1e-6 * np.linalg.norm(X, axis=1))
+
+
+def test_chunked_encode_is_independent_per_chunk():
+    """s_n = 2 with an orthonormal dictionary per chunk and s = d_h / s_n recovers x exactly;
+    changing chunk 1 of x or its dictionary leaves the codes of chunk 0 alone; the stored size
+    is 4 * s * s_n bytes per head vector."""
+    rng = np.random.default_rng(5)
+    d_h, s_n = 16, 2
+    Q0 = np.linalg.qr(rng.standard_normal((8, 8)))[0].astype(np.float32)
+    Q1 = np.linalg.qr(rng.standard_normal((8, 8)))[0].astype(np.float32)
+    X = rng.standard_normal((20, d_h)).astype(np.float32)
+    res = orc.mp_encode_chunked([Q0, Q1], X, 8)
+    xh = orc.reconstruct_chunked([Q0, Q1], [r.idx for r in res], [r.coef for r in res])
+    assert np.allclose(xh, X, atol=1e-5)
+    X2 = X.copy()
+    X2[:, 8:] = rng.standard_normal((20, 8)).astype(np.float32)
+    res2 = orc.mp_encode_chunked([Q0, Q0], X2, 8)
+    assert np.array_equal(res2[0].idx, res[0].idx) and np.array_equal(res2[0].coef, res[0].coef)
+    assert orc.code_bytes_per_vector(8, s_n) == 4 * 8 * 2 and orc.code_bits_per_channel(d_h, 8, s_n) == 32.0
+    with pytest.raises(ValueError):
+        orc.mp_encode_chunked([Q0, Q1, Q0], X, 4)
