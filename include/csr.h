@@ -62,10 +62,18 @@ extern "C" {
  *                        re-scored in fp64.  The coefficient and the residual update
  *                        are fp64.  Selects the same atoms as an fp64 evaluation of the
  *                        pursuit except at exact-to-rounding ties.
+ *                        With few rows (the vectors one decoding step adds: fewer row
+ *                        tiles of 64 than half the SMs) the dictionary is split across
+ *                        the SMs instead of the rows, two launches per iteration, with
+ *                        identical codes; this path uses the library-owned scratch
+ *                        (not taken when a caller workspace is given, or when the
+ *                        environment variable CSR_EXACT_NO_SPLIT is set).
  *   CSR_MODE_BF16_FAST   correlations on the tcgen05 tensor cores with bf16 operands
  *                        (residual and atoms rounded to bf16) and fp32 accumulation.
  *                        Near-tied picks may differ from an fp64 evaluation; the mean
- *                        reconstruction error does not.
+ *                        reconstruction error does not.  The environment variable
+ *                        CSR_FAST_GROUP (1, 2, 4 or 8) overrides the arg-max group size
+ *                        the kernel would choose; every setting meets the same gates.
  */
 #define CSR_MODE_FP32_EXACT 0
 #define CSR_MODE_BF16_FAST 1

@@ -1,6 +1,6 @@
 """Throughput and reconstruction error of the codec on every synthetic configuration.
 
-  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5] [--reps 30]
+  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5,decode] [--reps 30]
 
 One JSON line per case: vectors/s and TFLOP/s of the fast encoder (median of the last two
 thirds of `reps` back-to-back launches, i.e. after the clocks have settled under the power
@@ -73,6 +73,27 @@ def run_case(w, reps, exact_rows=16384):
     }
 
 
+def run_decode_case(seqs, kv_heads, N, s, reps):
+    """Latency of encoding the vectors ONE decoding step adds (seqs x kv_heads x {K, V} rows of
+    d = 128) in each mode."""
+    import os
+    dev = torch.device("cuda", torch.cuda.current_device())
+    w = wl.gqa_long(tokens=1, N=N, s=s, seqs=seqs, kv_heads=kv_heads)
+    D = torch.from_numpy(w.D).to(dev)
+    X = torch.from_numpy(w.X).to(dev)
+    Xb = X.to(torch.bfloat16)
+    M = w.M
+    idx = torch.empty((M, s), dtype=torch.uint16, device=dev)
+    coef = torch.empty((M, s), dtype=torch.float16, device=dev)
+    out = {"case": f"decode_step_{seqs}x{kv_heads}x2", "M": M, "N": N, "d": w.d, "s": s}
+    out["exact_split_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, X, s, mode=csr.CSR_MODE_FP32_EXACT, out_idx=idx, out_coef=coef), reps)
+    os.environ["CSR_EXACT_NO_SPLIT"] = "1"
+    out["exact_row_tile_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, X, s, mode=csr.CSR_MODE_FP32_EXACT, out_idx=idx, out_coef=coef), 3)
+    del os.environ["CSR_EXACT_NO_SPLIT"]
+    out["fast_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, Xb, s, out_idx=idx, out_coef=coef), reps)
+    return out
+
+
 def cases(names):
     for n in names:
         if n == "c1":
@@ -94,14 +115,18 @@ def cases(names):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--configs", default="c1,c2,c3,c4,c5")
+    ap.add_argument("--configs", default="c1,c2,c3,c4,c5,decode")
     ap.add_argument("--reps", type=int, default=30)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device (there is no CPU fallback)")
     build.build()
-    for w in cases(args.configs.split(",")):
+    names = args.configs.split(",")
+    for w in cases([n for n in names if n != "decode"]):
         print(json.dumps(run_case(w, args.reps)), flush=True)
+    if "decode" in names:
+        for seqs, kv_heads in ((1, 8), (8, 8), (64, 8)):
+            print(json.dumps(run_decode_case(seqs, kv_heads, 8192, 16, args.reps)), flush=True)
 
 
 if __name__ == "__main__":

@@ -33,6 +33,13 @@ struct EncodeArgs {
 // fp32-operand matching pursuit with fp64 re-scoring of unresolved picks.
 int launch_encode_exact(const EncodeArgs& a);
 
+// The same encoder for few rows (the vectors one decoding step adds): the dictionary is
+// split across CTAs, two launches per iteration; identical codes.  `scratch` must hold
+// encode_exact_split_scratch_bytes() bytes, 256-byte aligned.
+bool encode_exact_split_applies(int64_t M, int N);
+size_t encode_exact_split_scratch_bytes(int64_t M, int d, int N);
+int launch_encode_exact_split(const EncodeArgs& a, void* scratch);
+
 // tcgen05 bf16 matching pursuit.  `workspace` holds the bf16 copy of D (N*d*2 bytes,
 // 1024-byte aligned); `status` is a device word that receives kStatusTimeout.
 int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status);

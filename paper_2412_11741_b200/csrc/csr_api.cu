@@ -2,6 +2,7 @@
 // Every computation is done by the kernels in the other translation units.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -246,7 +247,16 @@ int encode_device(const csr_encode_params_t* p) {
     a.ldx = p->ldx ? p->ldx : p->d;
     a.ld_code = p->ld_code ? p->ld_code : p->s;
     a.stream = static_cast<cudaStream_t>(p->stream);
-    if (p->mode == CSR_MODE_FP32_EXACT) return launch_encode_exact(a);
+    if (p->mode == CSR_MODE_FP32_EXACT) {
+        // few rows: split the dictionary across the SMs (library-owned scratch; a caller
+        // workspace is sized for the fast mode only, so with one the row-tile encoder runs)
+        if (!p->workspace && encode_exact_split_applies(p->M, p->N) && !getenv("CSR_EXACT_NO_SPLIT")) {
+            void* base = nullptr;
+            if (int rc = ensure_work(encode_exact_split_scratch_bytes(p->M, p->d, p->N), &base)) return rc;
+            return launch_encode_exact_split(a, align_up(static_cast<char*>(base) + kStatusBytes, 1024));
+        }
+        return launch_encode_exact(a);
+    }
 
     void* base = nullptr;
     if (p->workspace) {

@@ -8,25 +8,18 @@
 //
 // fp32 rounding can reorder two correlations that are closer than about
 // 2 * 128 * 2^-24 * ||R||.  A row whose two largest values are inside that band is
-// re-scored: one warp recomputes all N correlations of that row in fp64 and takes the
+// re-scored by the whole CTA: an fp32 pass collects the atoms within the band of the
+// maximum, their correlations are recomputed in fp64 and the largest is taken, as an
 // arg-max with the lowest-index tie rule.  The coefficient (Eq. 2, signed) is always an
 // fp64 dot product of the fp64 residual with the fp32 atom, and the residual update
 // (Eq. 4) is fp64; the fp32 copy of the residual that feeds the next sweep is rounded
 // from it.
-#include "common.cuh"
+#include "exact_common.cuh"
 
 namespace csr {
 namespace {
 
-constexpr int BM = 64;        // rows per CTA
-constexpr int BN = 128;       // atoms per dictionary tile
-constexpr int BK = 16;        // channels per staged chunk
-constexpr int NT = 256;       // threads per CTA
-constexpr int AS_LD = BM + 4; // leading dimension of the transposed fp32 residual
-constexpr int BS_LD = BN + 4;
-// |fp32 dot - exact dot| <= d * 2^-24 * ||R|| * ||atom|| for d <= 128 sequential FMAs plus
-// the rounding of R itself; two candidates can therefore swap when closer than twice that.
-constexpr float kBandRel = 1.6e-5f;
+using namespace exact;
 
 template <int D_>
 struct Smem {
@@ -37,38 +30,8 @@ struct Smem {
     float second[BM];
     int bidx[BM];
     float band[BM];
+    RescoreSmem rs;
 };
-
-__device__ __forceinline__ float load_x(const void* X, int x_dtype, int64_t off) {
-    if (x_dtype == CSR_DTYPE_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(X)[off]);
-    return reinterpret_cast<const float*>(X)[off];
-}
-
-struct Top2 {
-    float best, second;
-    int idx;
-};
-
-__device__ __forceinline__ void top2_push(Top2& t, float a, int n) {
-    if (a > t.best) {
-        t.second = t.best;
-        t.best = a;
-        t.idx = n;
-    } else if (a > t.second) {
-        t.second = a;
-    }
-}
-
-__device__ __forceinline__ void top2_merge(Top2& t, float ob, float os, int oi) {
-    bool other_wins = (ob > t.best) || (ob == t.best && oi < t.idx);
-    float loser = other_wins ? t.best : ob;
-    float sec = fmaxf(fmaxf(t.second, os), loser);
-    if (other_wins) {
-        t.best = ob;
-        t.idx = oi;
-    }
-    t.second = sec;
-}
 
 template <int D_>
 __global__ void __launch_bounds__(NT, 1)
@@ -84,7 +47,6 @@ encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int
     const int ty = tid >> 4;   // row group: rows ty*4 .. ty*4+3
     const int64_t n_tiles = (M + BM - 1) / BM;
     const int n_btiles = (N + BN - 1) / BN;
-    constexpr int KCH = D_ / BK;
 
     for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int64_t row0 = tile * BM;
@@ -110,70 +72,7 @@ encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int
             for (int i = 0; i < 4; ++i) top[i] = Top2{-1.f, -1.f, 0};
 
             // ---- sweep over the dictionary (Eq. 2-3) ----
-            const int total_chunks = n_btiles * KCH;
-            float4 stage[2];
-            auto gload = [&](int chunk) {
-                const int bt = chunk / KCH, kc = chunk % KCH;
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const int f = tid + i * NT;
-                    const int atom = f >> 2, kq = f & 3;
-                    const int n = bt * BN + atom;
-                    stage[i] = (n < N) ? *reinterpret_cast<const float4*>(D + (int64_t)n * D_ + kc * BK + kq * 4)
-                                       : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            };
-            auto sstore = [&](int buf) {
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const int f = tid + i * NT;
-                    const int atom = f >> 2, kq = f & 3;
-                    sm.Bs[buf][kq * 4 + 0][atom] = stage[i].x;
-                    sm.Bs[buf][kq * 4 + 1][atom] = stage[i].y;
-                    sm.Bs[buf][kq * 4 + 2][atom] = stage[i].z;
-                    sm.Bs[buf][kq * 4 + 3][atom] = stage[i].w;
-                }
-            };
-            gload(0);
-            sstore(0);
-            __syncthreads();
-            float acc[4][8];
-            for (int chunk = 0; chunk < total_chunks; ++chunk) {
-                const int buf = chunk & 1;
-                const int kc = chunk % KCH;
-                if (kc == 0) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
-                }
-                if (chunk + 1 < total_chunks) gload(chunk + 1);
-#pragma unroll
-                for (int k = 0; k < BK; ++k) {
-                    const float4 a4 = *reinterpret_cast<const float4*>(&sm.As[kc * BK + k][ty * 4]);
-                    const float4 b0 = *reinterpret_cast<const float4*>(&sm.Bs[buf][k][tx * 4]);
-                    const float4 b1 = *reinterpret_cast<const float4*>(&sm.Bs[buf][k][64 + tx * 4]);
-                    const float a[4] = {a4.x, a4.y, a4.z, a4.w};
-                    const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-                }
-                if (kc == KCH - 1) {
-                    const int nb = (chunk / KCH) * BN;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int n = nb + (j < 4 ? tx * 4 + j : 64 + tx * 4 + (j - 4));
-                        if (n < N) {
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) top2_push(top[i], fabsf(acc[i][j]), n);
-                        }
-                    }
-                }
-                if (chunk + 1 < total_chunks) sstore(buf ^ 1);
-                __syncthreads();
-            }
+            sweep_tiles<D_>(D, N, 0, n_btiles, sm.As, sm.Bs, top);
             // Each thread visited its atoms in ascending order, so its strict ">" kept the
             // lowest index among equal values; top2_merge applies the same rule across the
             // 16 threads that share a row.  Equal fp32 values are re-scored in fp64 anyway.
@@ -194,43 +93,21 @@ encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int
             }
             __syncthreads();
 
+            // ---- rows that fp32 cannot decide are re-scored by the whole CTA ----
+            for (int r = 0; r < BM; ++r) {
+                const bool unresolved = (row0 + r < M) && (N > 1) && (sm.best[r] > 0.f) &&
+                                        (sm.best[r] - sm.second[r] <= sm.band[r]);
+                if (!unresolved) continue;                // uniform over the CTA
+                const int bn = rescore_cta<D_>(D, N, sm.Rd[r], sm.best[r], sm.band[r], sm.rs);
+                if (tid == 0) sm.bidx[r] = bn;
+                __syncthreads();
+            }
             // ---- pick, coefficient and residual update (Eq. 2-4), one warp per row ----
             for (int r = warp; r < BM; r += NT / 32) {
                 const int64_t m = row0 + r;
                 if (m >= M) continue;
-                int bi = sm.bidx[r];
-                const bool unresolved = (N > 1) && (sm.best[r] - sm.second[r] <= sm.band[r]);
+                const int bi = sm.best[r] > 0.f ? sm.bidx[r] : 0;   // an all-zero sweep picks atom 0
                 const double* Rr = sm.Rd[r];
-                if (unresolved) {
-                    double bb = -1.0;
-                    int bn = 0;
-                    for (int n = lane; n < N; n += 32) {
-                        const float4* dn = reinterpret_cast<const float4*>(D + (int64_t)n * D_);
-                        double c = 0.0;
-#pragma unroll 4
-                        for (int q = 0; q < D_ / 4; ++q) {
-                            const float4 v = dn[q];
-                            c = fma(Rr[4 * q + 0], (double)v.x, c);
-                            c = fma(Rr[4 * q + 1], (double)v.y, c);
-                            c = fma(Rr[4 * q + 2], (double)v.z, c);
-                            c = fma(Rr[4 * q + 3], (double)v.w, c);
-                        }
-                        const double a = fabs(c);
-                        if (a > bb) {
-                            bb = a;
-                            bn = n;
-                        }
-                    }
-                    for (int o = 16; o; o >>= 1) {
-                        const double ob = __shfl_xor_sync(0xffffffffu, bb, o);
-                        const int on = __shfl_xor_sync(0xffffffffu, bn, o);
-                        if (ob > bb || (ob == bb && on < bn)) {
-                            bb = ob;
-                            bn = on;
-                        }
-                    }
-                    bi = bn;
-                }
                 const float* db = D + (int64_t)bi * D_;
                 double part = 0.0;
                 for (int k = lane; k < D_; k += 32) part = fma(Rr[k], (double)db[k], part);

@@ -135,6 +135,27 @@ def test_exact_identity_dictionary_recovers_exactly(csr):
     assert np.array_equal(coef, np.take_along_axis(X, order, 1))
 
 
+@pytest.mark.parametrize("M,N,d,s", [(1, 8192, 128, 16), (128, 8192, 128, 16), (200, 272, 128, 5), (1000, 4096, 64, 8),
+                                     (4000, 2048, 128, 4)])
+def test_exact_few_rows_split_dictionary_path(csr, M, N, d, s, monkeypatch):
+    """Few rows (what one decoding step adds): the dictionary is split across CTAs.  The codes
+    must be those of the one-CTA-per-row-tile encoder bit for bit, and the oracle's."""
+    rng = np.random.default_rng(M + N)
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    D[N // 2] = D[3]                                     # a duplicated atom: the lower index must win
+    X = rng.standard_normal((M, d)).astype(np.float32)
+    X[0] = D[3] * np.float32(1.25)
+    w = wl.Workload("decode", D, X, s, "f32")
+    idx, coef = _encode(csr, w, X, csr.CSR_MODE_FP32_EXACT)
+    monkeypatch.setenv("CSR_EXACT_NO_SPLIT", "1")
+    idx2, coef2 = _encode(csr, w, X, csr.CSR_MODE_FP32_EXACT)
+    monkeypatch.delenv("CSR_EXACT_NO_SPLIT")
+    assert np.array_equal(idx, idx2) and np.array_equal(coef, coef2)
+    assert idx[0, 0] == 3
+    rep = parity.compare_exact(D, X, s, idx, coef)
+    assert rep.ok, rep.detail
+
+
 # ---------------------------------------------------------------------------------------
 # fast mode
 # ---------------------------------------------------------------------------------------
