@@ -181,6 +181,31 @@ int csr_dict_append(void* D, int N_cur, int N_cap, int d, const void* X, int x_d
                     const int64_t* rows, int n_rows, void* stream);
 
 /*
+ * Attention straight from the codes ("De-Sparse to restore": the restored X~ = D r of
+ * Eq. 12 is what the attention scores are computed from; both products below are that
+ * computation with X~ never written to memory, which is possible because X~ is linear in
+ * the atoms).  B code streams (one per sequence and KV head) of T tokens each share the
+ * dictionary D; H query heads attend to each stream (H = 1 without grouped queries).
+ *
+ * csr_key_scores:  scores[b][h][t] = scale * Q[b][h][:] . X~_K[b][t][:]
+ *                                  = sum_g coef[b][t][g] * (scale * D[idx[b][t][g]][:] . Q[b][h][:]),
+ *     terms added in stored order g = 0 .. s-1 in fp32.  Q is [B][H][d], q_dtype F32 or BF16;
+ *     scores is [B][H][T] fp32 (before softmax).
+ * csr_value_mix:   out[b][h][:] = sum_t W[b][h][t] * X~_V[b][t][:],
+ *     W is [B][H][T] fp32 (attention weights), out is [B][H][d] fp32.  Accumulated with
+ *     atomic fp32 adds: results are reproducible to rounding, not bit for bit.
+ *
+ * idx and coef are [B][T][s] (coef_dtype F16 or F32); an idx >= N is clamped to N-1.
+ * Limits: d in {64, 128}, 1 <= N <= 49152 (one head's N partial products must fit in
+ * shared memory), 1 <= s <= 64, 1 <= H <= 64, B, T >= 0.  All pointers are device pointers,
+ * 16-byte aligned.  Asynchronous on `stream`.
+ */
+int csr_key_scores(const void* D, int N, int d, const void* Q, int q_dtype, int B, int H, const uint16_t* idx,
+                   const void* coef, int coef_dtype, int64_t T, int s, float scale, float* scores, void* stream);
+int csr_value_mix(const void* D, int N, int d, const float* W, int B, int H, const uint16_t* idx, const void* coef,
+                  int coef_dtype, int64_t T, int s, float* out, void* stream);
+
+/*
  * Encode with HOST buffers (the same operation as csr_encode_ex; only X, out_idx and
  * out_coef are host pointers, ideally page-locked).  X is copied to the device in
  * chunks that overlap with the encoding of the previous chunk, the codes are copied

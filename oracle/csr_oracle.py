@@ -138,6 +138,29 @@ def dict_append(D: np.ndarray, N_cur: int, X: np.ndarray, rows) -> np.ndarray:
     return D
 
 
+# --- attention from the restored tensors ("De-Sparse to restore") ---------------------------
+
+def key_scores(D: np.ndarray, Q: np.ndarray, idx: np.ndarray, coef: np.ndarray, scale: float = 1.0) -> np.ndarray:
+    """scores[b][h][t] = scale * Q[b][h] . X~[b][t], with X~ = Eq. 12 restored from the codes
+    [B][T][s]; Q is [B][H][d].  The restored tensor is formed explicitly, fp64 throughout."""
+    B, T, s = idx.shape
+    out = np.empty((B, Q.shape[1], T), np.float64)
+    for b in range(B):
+        xt = reconstruct(D, idx[b], coef[b])                  # [T][d]
+        out[b] = scale * (np.asarray(Q[b], np.float64) @ xt.T)
+    return out
+
+
+def value_mix(D: np.ndarray, W: np.ndarray, idx: np.ndarray, coef: np.ndarray) -> np.ndarray:
+    """out[b][h] = sum_t W[b][h][t] * X~[b][t] with X~ restored by Eq. 12; W is [B][H][T]."""
+    B, T, s = idx.shape
+    out = np.empty((B, W.shape[1], D.shape[1]), np.float64)
+    for b in range(B):
+        xt = reconstruct(D, idx[b], coef[b])
+        out[b] = np.asarray(W[b], np.float64) @ xt
+    return out
+
+
 # --- storage format ("Analysis for CSR") -------------------------------------------------
 
 def pack_codes(idx: np.ndarray, coef: np.ndarray):

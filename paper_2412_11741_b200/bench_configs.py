@@ -1,6 +1,6 @@
 """Throughput and reconstruction error of the codec on every synthetic configuration.
 
-  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5,decode] [--reps 30]
+  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5,decode,attention] [--reps 30]
 
 One JSON line per case: vectors/s and TFLOP/s of the fast encoder (median of the last two
 thirds of `reps` back-to-back launches, i.e. after the clocks have settled under the power
@@ -94,6 +94,33 @@ def run_decode_case(seqs, kv_heads, N, s, reps):
     return out
 
 
+def run_attention_case(reps):
+    """Attention straight from the codes on the GQA long-context shape: 64 code streams (8
+    sequences x 8 KV heads) of 16384 tokens, s = 16, 4 query heads per KV head.  Rates are
+    algorithmic HBM bytes (codes read once, scores written / weights read once) over time;
+    the restored-tensor route (de-sparse kernel to bf16, then reading it back once) is timed
+    beside it as the traffic it avoids."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    B, H, T, s, N, d = 64, 4, 16384, 16, 8192, 128
+    g = torch.Generator(device=dev).manual_seed(0)
+    D = torch.nn.functional.normalize(torch.randn((N, d), device=dev, generator=g), dim=1).contiguous()
+    idx = torch.randint(0, N, (B, T, s), device=dev, generator=g, dtype=torch.int32).to(torch.int16).view(torch.uint16)
+    coef = torch.randn((B, T, s), device=dev, generator=g).to(torch.float16)
+    Q = torch.randn((B, H, d), device=dev, generator=g)
+    W = torch.softmax(torch.randn((B, H, T), device=dev, generator=g), dim=-1)
+    sc = torch.empty((B, H, T), dtype=torch.float32, device=dev)
+    out = torch.empty((B, H, d), dtype=torch.float32, device=dev)
+    xh = torch.empty((B * T, d), dtype=torch.bfloat16, device=dev)
+    t_sc = _time(lambda: csr.csr_key_scores(D, Q, idx, coef, 1.0, scores=sc), reps)
+    t_mx = _time(lambda: csr.csr_value_mix(D, W, idx, coef, out=out), reps)
+    t_rc = _time(lambda: csr.csr_reconstruct_ex(D, idx.view(B * T, s), coef.view(B * T, s), X_hat=xh), reps)
+    code_b, sw_b = B * T * s * 4.0, B * H * T * 4.0
+    return {"case": "attention_from_codes", "B": B, "H": H, "T": T, "N": N, "d": d, "s": s,
+            "key_scores_ms": round(t_sc, 4), "key_scores_hbm_gbs": (code_b + sw_b) / (t_sc * 1e-3) / 1e9,
+            "value_mix_ms": round(t_mx, 4), "value_mix_hbm_gbs": (code_b + sw_b) / (t_mx * 1e-3) / 1e9,
+            "restore_to_bf16_ms": round(t_rc, 4), "restored_bytes": B * T * d * 2.0, "code_bytes": code_b}
+
+
 def cases(names):
     for n in names:
         if n == "c1":
@@ -115,18 +142,20 @@ def cases(names):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--configs", default="c1,c2,c3,c4,c5,decode")
+    ap.add_argument("--configs", default="c1,c2,c3,c4,c5,decode,attention")
     ap.add_argument("--reps", type=int, default=30)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device (there is no CPU fallback)")
     build.build()
     names = args.configs.split(",")
-    for w in cases([n for n in names if n != "decode"]):
+    for w in cases([n for n in names if n not in ("decode", "attention")]):
         print(json.dumps(run_case(w, args.reps)), flush=True)
     if "decode" in names:
         for seqs, kv_heads in ((1, 8), (8, 8), (64, 8)):
             print(json.dumps(run_decode_case(seqs, kv_heads, 8192, 16, args.reps)), flush=True)
+    if "attention" in names:
+        print(json.dumps(run_attention_case(args.reps)), flush=True)
 
 
 if __name__ == "__main__":

@@ -33,7 +33,7 @@ CSR_MODE_BF16_FAST = 1
 
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
-    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append",
+    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append", "csr_key_scores", "csr_value_mix",
     "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
@@ -103,6 +103,11 @@ def lib() -> ctypes.CDLL:
         L.csr_reconstruct_grouped.restype = i32
         L.csr_dict_append.argtypes = [vp, i32, i32, i32, vp, i32, i64, i64, vp, i32, vp]
         L.csr_dict_append.restype = i32
+        f32 = ctypes.c_float
+        L.csr_key_scores.argtypes = [vp, i32, i32, vp, i32, i32, i32, vp, vp, i32, i64, i32, f32, vp, vp]
+        L.csr_key_scores.restype = i32
+        L.csr_value_mix.argtypes = [vp, i32, i32, vp, i32, i32, vp, vp, i32, i64, i32, vp, vp]
+        L.csr_value_mix.restype = i32
         L.csr_device_status.argtypes = [vp]
         L.csr_device_status.restype = i32
         L.csr_release_workspace.argtypes = []
@@ -292,6 +297,48 @@ def csr_dict_append(D: torch.Tensor, N_cur: int, X: torch.Tensor, rows: torch.Te
                                      X.shape[0], X.stride(0) if X.shape[0] > 1 else 0, rows.data_ptr(), n,
                                      _stream_ptr(D)))
     return N_cur + n
+
+
+def _check_codes(D, idx, coef):
+    assert D.is_cuda and D.is_contiguous() and D.dtype == torch.float32
+    assert idx.is_cuda and coef.is_cuda and idx.is_contiguous() and coef.is_contiguous()
+    assert idx.dtype == torch.uint16 and idx.dim() == 3 and idx.shape == coef.shape
+
+
+def csr_key_scores(D: torch.Tensor, Q: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, scale: float = 1.0,
+                   scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """csr_key_scores: Q [B][H][d] (fp32 or bf16), codes [B][T][s]; returns scores [B][H][T] fp32."""
+    _check_codes(D, idx, coef)
+    B, T, s = idx.shape
+    N, d = D.shape
+    assert Q.is_cuda and Q.is_contiguous() and Q.dim() == 3 and Q.shape[0] == B and Q.shape[2] == d
+    H = Q.shape[1]
+    if scores is None:
+        scores = torch.empty((B, H, T), dtype=torch.float32, device=D.device)
+    assert scores.is_contiguous() and scores.dtype == torch.float32 and tuple(scores.shape) == (B, H, T)
+    with torch.cuda.device(D.device):
+        _check(lib().csr_key_scores(D.data_ptr(), N, d, Q.data_ptr(), _TORCH_DTYPE[Q.dtype], B, H, idx.data_ptr(),
+                                    coef.data_ptr(), _TORCH_DTYPE[coef.dtype], T, s, float(scale), scores.data_ptr(),
+                                    _stream_ptr(D)))
+    return scores
+
+
+def csr_value_mix(D: torch.Tensor, W: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor,
+                  out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """csr_value_mix: W [B][H][T] fp32 attention weights, codes [B][T][s]; returns [B][H][d] fp32."""
+    _check_codes(D, idx, coef)
+    B, T, s = idx.shape
+    N, d = D.shape
+    assert W.is_cuda and W.is_contiguous() and W.dtype == torch.float32 and W.dim() == 3
+    assert W.shape[0] == B and W.shape[2] == T
+    H = W.shape[1]
+    if out is None:
+        out = torch.empty((B, H, d), dtype=torch.float32, device=D.device)
+    assert out.is_contiguous() and out.dtype == torch.float32 and tuple(out.shape) == (B, H, d)
+    with torch.cuda.device(D.device):
+        _check(lib().csr_value_mix(D.data_ptr(), N, d, W.data_ptr(), B, H, idx.data_ptr(), coef.data_ptr(),
+                                   _TORCH_DTYPE[coef.dtype], T, s, out.data_ptr(), _stream_ptr(D)))
+    return out
 
 
 def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *,

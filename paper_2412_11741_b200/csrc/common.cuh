@@ -64,6 +64,28 @@ int launch_reconstruct(const ReconstructArgs& a);
 int launch_dict_append(float* D_new, int d, const void* X, int x_dtype, int64_t M, int64_t ldx, const int64_t* rows,
                        int n_rows, cudaStream_t stream);
 
+// Attention straight from the codes.  key_scores: Q = queries [B][H][d] (q_dtype), out = scores
+// [B][H][T].  value_mix: Q = attention weights [B][H][T] fp32, out = [B][H][d] fp32.
+struct AttnArgs {
+    const float* D;
+    int N, d;
+    const void* Q;
+    int q_dtype;
+    int B, H;
+    const uint16_t* idx;   // [B][T][s]
+    const void* coef;      // [B][T][s]
+    int coef_dtype;
+    int64_t T;
+    int s;
+    float scale;
+    float* out;
+    cudaStream_t stream;
+};
+// `scratch` holds attn_scratch_bytes() bytes: the [B*H][N] fp32 array of partial products.
+size_t attn_scratch_bytes(int B, int H, int N);
+int launch_key_scores(const AttnArgs& a, float* scratch);
+int launch_value_mix(const AttnArgs& a, float* scratch);
+
 int sm_count();
 
 }  // namespace csr

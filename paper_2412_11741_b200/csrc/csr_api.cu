@@ -374,6 +374,47 @@ int csr_dict_append(void* D, int N_cur, int N_cap, int d, const void* X, int x_d
                               static_cast<cudaStream_t>(stream));
 }
 
+static int check_attn(const void* D, int N, int d, const void* Q, int B, int H, const uint16_t* idx, const void* coef,
+                      int coef_dtype, int64_t T, int s, const void* out) {
+    if (d != 64 && d != 128) return fail(CSR_ERR_UNSUPPORTED, "d = %d: only 64 and 128 are supported", d);
+    if (N < 1 || N > 49152) return fail(CSR_ERR_INVALID_ARG, "N = %d outside [1, 49152]", N);
+    if (s < 1 || s > 64) return fail(CSR_ERR_INVALID_ARG, "s = %d outside [1, 64]", s);
+    if (H < 1 || H > 64) return fail(CSR_ERR_INVALID_ARG, "H = %d outside [1, 64]", H);
+    if (B < 0 || T < 0) return fail(CSR_ERR_INVALID_ARG, "B or T is negative");
+    if (coef_dtype != CSR_DTYPE_F32 && coef_dtype != CSR_DTYPE_F16)
+        return fail(CSR_ERR_INVALID_ARG, "coef_dtype must be F32 or F16");
+    if (!D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
+    if (B > 0 && T > 0 && (!Q || !out || !idx || !coef))
+        return fail(CSR_ERR_INVALID_ARG, "a query / weight / code / output pointer is NULL");
+    if (!aligned16(D) || !aligned16(Q) || !aligned16(idx) || !aligned16(coef) || !aligned16(out))
+        return fail(CSR_ERR_ALIGNMENT, "all pointers must be 16-byte aligned");
+    return CSR_OK;
+}
+
+int csr_key_scores(const void* D, int N, int d, const void* Q, int q_dtype, int B, int H, const uint16_t* idx,
+                   const void* coef, int coef_dtype, int64_t T, int s, float scale, float* scores, void* stream) {
+    if (int rc = check_attn(D, N, d, Q, B, H, idx, coef, coef_dtype, T, s, scores)) return rc;
+    if (q_dtype != CSR_DTYPE_F32 && q_dtype != CSR_DTYPE_BF16) return fail(CSR_ERR_INVALID_ARG, "q_dtype must be F32 or BF16");
+    AttnArgs a{static_cast<const float*>(D), N, d, Q, q_dtype, B, H, idx, coef, coef_dtype, T, s, scale, scores,
+               static_cast<cudaStream_t>(stream)};
+    if (B == 0 || T == 0) return CSR_OK;
+    void* base = nullptr;
+    if (int rc = ensure_work(attn_scratch_bytes(B, H, N), &base)) return rc;
+    return launch_key_scores(a, static_cast<float*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)));
+}
+
+int csr_value_mix(const void* D, int N, int d, const float* W, int B, int H, const uint16_t* idx, const void* coef,
+                  int coef_dtype, int64_t T, int s, float* out, void* stream) {
+    if (int rc = check_attn(D, N, d, W, B, H, idx, coef, coef_dtype, T, s, out)) return rc;
+    if (B > 0 && !out) return fail(CSR_ERR_INVALID_ARG, "out is NULL");     // zeroed even when T == 0
+    AttnArgs a{static_cast<const float*>(D), N, d, W, CSR_DTYPE_F32, B, H, idx, coef, coef_dtype, T, s, 1.0f, out,
+               static_cast<cudaStream_t>(stream)};
+    if (B == 0) return CSR_OK;
+    void* base = nullptr;
+    if (int rc = ensure_work(attn_scratch_bytes(B, H, N), &base)) return rc;
+    return launch_value_mix(a, static_cast<float*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)));
+}
+
 int csr_encode_host(const csr_encode_params_t* p) {
     if (int rc = check_encode(p, true)) return rc;
     if (p->M == 0) return CSR_OK;

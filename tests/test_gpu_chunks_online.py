@@ -117,3 +117,54 @@ def test_online_atoms_match_oracle_and_are_used_by_the_encoder(csr, d, dtype):
     assert rep.ok, rep.detail
     own = N_off + np.array([int(np.flatnonzero(rows == r)[0]) for r in sel])
     assert np.array_equal(_np_idx(i)[:, 0].astype(np.int64), own)
+
+
+@pytest.mark.parametrize("B,H,T,N,d,s,coef_dtype", [
+    (3, 4, 5000, 2048, 128, 8, torch.float16), (2, 1, 1500, 8192, 128, 16, torch.float32),
+    (2, 8, 700, 1024, 64, 4, torch.float16), (1, 9, 300, 16384, 128, 3, torch.float32), (2, 2, 0, 256, 64, 2, torch.float16),
+])
+def test_attention_from_codes_matches_oracle(csr, B, H, T, N, d, s, coef_dtype):
+    """Scores and weighted value sums computed straight from the codes against the oracle,
+    which restores the tensor (Eq. 12) and multiplies in fp64."""
+    rng = np.random.default_rng(B * 1000 + T + N)
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    idx = rng.integers(0, N, (B, T, s)).astype(np.int32)
+    if T:
+        idx[:, :, -1] = idx[:, :, 0]                                   # repeated atoms accumulate
+    coef = (rng.standard_normal((B, T, s)) * 2).astype(np.float32)
+    if coef_dtype == torch.float16:
+        coef = coef.astype(np.float16).astype(np.float32)
+    Q = rng.standard_normal((B, H, d)).astype(np.float32)
+    W = rng.random((B, H, T)).astype(np.float32)
+    W /= np.maximum(W.sum(-1, keepdims=True), 1e-30)                   # rows of a softmax
+    Dd = torch.from_numpy(D).to(DEV)
+    it = torch.from_numpy(idx.astype(np.uint16).view(np.int16)).to(DEV).view(torch.uint16)
+    ct = torch.from_numpy(coef).to(DEV).to(coef_dtype)
+    scale = 1.0 / np.sqrt(d)
+    sc = csr.csr_key_scores(Dd, torch.from_numpy(Q).to(DEV), it, ct, scale).cpu().numpy()
+    want = orc.key_scores(D, Q, idx, coef.astype(np.float64), scale)
+    bound = scale * np.linalg.norm(Q, axis=2)[:, :, None] * np.abs(coef).sum(2)[:, None, :]   # sum |coef| ||q|| ||atom||
+    assert sc.shape == want.shape and np.all(np.abs(sc - want) <= 2e-6 * bound + 1e-30)
+    Qb = wl.round_to_bf16(Q)                                            # bf16 queries are read exactly
+    sc = csr.csr_key_scores(Dd, torch.from_numpy(Qb).to(DEV).to(torch.bfloat16), it, ct, scale).cpu().numpy()
+    assert np.all(np.abs(sc - orc.key_scores(D, Qb, idx, coef.astype(np.float64), scale)) <= 2e-6 * bound + 1e-30)
+    mix = csr.csr_value_mix(Dd, torch.from_numpy(W).to(DEV), it, ct).cpu().numpy()
+    want = orc.value_mix(D, W, idx, coef.astype(np.float64))
+    mbound = (W[:, :, :, None] * np.abs(coef)[:, None, :, :]).sum((2, 3))[:, :, None]       # sum w |coef| ||atom||
+    assert mix.shape == want.shape and np.all(np.abs(mix - want) <= 4e-6 * mbound + 1e-30)
+
+
+def test_scores_from_codes_equal_scores_from_the_restored_tensor(csr):
+    """End to end on key-like data: encode, then q . x~ from the codes equals q . x~ from the
+    de-sparse kernel's output (fp32), to fp32 rounding."""
+    w = wl.llama2_layer(tokens=256, N=1024)
+    T = 256
+    D = torch.from_numpy(w.D).to(DEV)
+    X = torch.from_numpy(w.X[:32 * T]).to(DEV).to(torch.bfloat16)          # 32 key heads x 256 tokens
+    idx, coef = csr.csr_encode(D, X, w.s)
+    xh = csr.csr_reconstruct_ex(D, idx, coef, out_dtype=torch.float32).view(32, T, 128)
+    Q = torch.randn((32, 2, 128), device=DEV, generator=torch.Generator(device=DEV).manual_seed(1))
+    sc = csr.csr_key_scores(D, Q, idx.view(32, T, w.s), coef.view(32, T, w.s))
+    ref = torch.einsum("bhd,btd->bht", Q.double(), xh.double())
+    tol = 2e-6 * (Q.norm(dim=2)[:, :, None] * coef.float().abs().sum(1).view(32, 1, T))
+    assert bool(((sc.double() - ref).abs() <= tol.double() + 1e-30).all())

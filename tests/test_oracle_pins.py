@@ -344,3 +344,38 @@ def test_chunked_encode_is_independent_per_chunk():
     assert orc.code_bytes_per_vector(8, s_n) == 4 * 8 * 2 and orc.code_bits_per_channel(d_h, 8, s_n) == 32.0
     with pytest.raises(ValueError):
         orc.mp_encode_chunked([Q0, Q1, Q0], X, 4)
+
+
+# ---------------------------------------------------------------------------------------
+# attention from the restored tensors
+# ---------------------------------------------------------------------------------------
+
+def test_attention_from_codes_closed_forms():
+    """Identity dictionary: the restored row is the scatter of its coefficients, so the score
+    is sum_g coef * q[idx] and the mix is a weighted scatter (written here with np.add.at,
+    not with the oracle's reconstruct); repeated indices accumulate; scale is linear; with
+    the oracle's own codes plus the final residual the exact q . x comes back."""
+    rng = np.random.default_rng(9)
+    B, H, T, s, d = 2, 3, 40, 4, 16
+    D = np.eye(d, dtype=np.float32)
+    idx = rng.integers(0, d, (B, T, s)).astype(np.int32)
+    idx[:, :, 3] = idx[:, :, 0]
+    coef = rng.standard_normal((B, T, s))
+    Q = rng.standard_normal((B, H, d))
+    W = rng.random((B, H, T))
+    sc = orc.key_scores(D, Q, idx, coef, scale=0.5)
+    want = 0.5 * np.einsum("btg,bhtg->bht", coef, Q[np.arange(B)[:, None, None, None], np.arange(H)[None, :, None, None], idx[:, None]])
+    assert np.allclose(sc, want, atol=1e-12)
+    mix = orc.value_mix(D, W, idx, coef)
+    want = np.zeros((B, H, d))
+    for b in range(B):
+        for h in range(H):
+            np.add.at(want[b, h], idx[b].ravel(), (W[b, h][:, None] * coef[b]).ravel())
+    assert np.allclose(mix, want, atol=1e-12)
+    # real dictionary: q . x = scores from the codes + q . final residual
+    Dn = wl.normalise_rows(rng.standard_normal((64, d)).astype(np.float32))
+    X = rng.standard_normal((T, d)).astype(np.float32)
+    res = orc.mp_encode(Dn, X, 5)
+    q = rng.standard_normal((1, 1, d))
+    sc = orc.key_scores(Dn, q, res.idx[None], res.coef[None])
+    assert np.allclose(sc[0, 0] + res.residual @ q[0, 0], X.astype(np.float64) @ q[0, 0], atol=1e-12)
