@@ -206,6 +206,40 @@ int csr_value_mix(const void* D, int N, int d, const float* W, int B, int H, con
                   int coef_dtype, int64_t T, int s, float* out, void* stream);
 
 /*
+ * One training step of the offline dictionary ("NeuralDict": Algorithm 1, procedure
+ * TrainNeurDict, with the MSE loss, the diversity loss, the complete loss and ReNorm).  For
+ * the batch X ([M][d], dense):
+ *   1. r(x) for every row by matching pursuit with s iterations over the current D (the
+ *      encoder of `mode`; its codes are then held fixed: the loss is differentiated with
+ *      respect to the atoms only);
+ *   2. L_MSE = sum_x ||x - D^T r(x)||^2 and its gradient, which touches only the selected
+ *      atoms: -2 * sum_{(x,g): i_g = n} c_g (x - x^);
+ *   3. L_div = ||I - D D^T||_F^2 / N^2 and its gradient (4 / N^2) (D D^T - I) D; the N x N
+ *      matrix is formed block by block on chip and never stored;
+ *   4. D <- ReNorm(D - lr * (grad L_MSE + beta * grad L_div)), every atom back to unit l2-norm.
+ * losses (device, two doubles, 8-byte aligned) receives L_MSE and L_div of the dictionary
+ * BEFORE the update; the paper's adaptive weight for the next batch is
+ * beta = min(0.1 * L_MSE / L_div, 1.0), which the caller forms from them.  The optimiser is
+ * a plain gradient step (the paper names none).  D is updated in place and must not be
+ * used by other work on the device meanwhile.  Uses the library-owned scratch; asynchronous
+ * on `stream`.  Gradient sums use atomic fp32 adds: reproducible to rounding.
+ */
+typedef struct csr_train_params {
+    uint32_t struct_size;   /* sizeof(csr_train_params_t) */
+    int32_t mode;           /* CSR_MODE_* of the matching-pursuit forward pass */
+    void* D;                /* [N][d] fp32, updated in place */
+    const void* X;          /* [M][d], x_dtype (F32 or BF16), dense */
+    int32_t x_dtype;
+    int32_t d, N, s;
+    int64_t M;
+    float lr;
+    float beta;
+    double* losses;         /* device, [2] */
+    void* stream;
+} csr_train_params_t;
+int csr_dict_train_step(const csr_train_params_t* p);
+
+/*
  * Encode with HOST buffers (the same operation as csr_encode_ex; only X, out_idx and
  * out_coef are host pointers, ideally page-locked).  X is copied to the device in
  * chunks that overlap with the encoding of the previous chunk, the codes are copied

@@ -161,6 +161,47 @@ def value_mix(D: np.ndarray, W: np.ndarray, idx: np.ndarray, coef: np.ndarray) -
     return out
 
 
+# --- one training step of the offline dictionary ("NeuralDict") -----------------------------
+
+def mse_loss_and_grad(D: np.ndarray, X: np.ndarray, idx: np.ndarray, coef: np.ndarray):
+    """L_MSE = sum_x ||x - W_D r(x)||^2 for given (fixed) codes, and its gradient with respect
+    to the atoms, [N][d]: every stored entry (x, g) contributes -2 c_g (x - x^) to atom i_g."""
+    Dd = np.asarray(D, np.float64)
+    E = np.asarray(X, np.float64) - reconstruct(D, idx, coef)
+    grad = np.zeros_like(Dd)
+    for g in range(idx.shape[1]):
+        np.add.at(grad, idx[:, g], -2.0 * coef[:, g][:, None] * E)
+    return float(np.sum(E * E)), grad
+
+
+def div_loss_and_grad(D: np.ndarray):
+    """L_div = ||I - W^T W||_F^2 / N^2 (W = D^T, one atom per column) and its gradient
+    (4 / N^2) (D D^T - I) D, [N][d]."""
+    Dd = np.asarray(D, np.float64)
+    N = Dd.shape[0]
+    G = Dd @ Dd.T - np.eye(N)
+    return float(np.sum(G * G) / N ** 2), (4.0 / N ** 2) * (G @ Dd)
+
+
+def adaptive_beta(l_mse: float, l_div: float) -> float:
+    """beta = min(0.1 * L_MSE / L_div, 1.0), from the last batch's loss values."""
+    return 1.0 if l_div <= 0 else min(0.1 * l_mse / l_div, 1.0)
+
+
+def dict_train_step(D: np.ndarray, X: np.ndarray, s: int, lr: float, beta: float):
+    """One batch of TrainNeurDict (Algorithm 1): codes by matching pursuit over the current
+    dictionary, L = L_MSE + beta * L_div differentiated with the codes held fixed, a plain
+    gradient step and ReNorm.  Returns (new D as fp32, L_MSE, L_div, MPResult); the losses
+    are those of the dictionary before the update."""
+    res = mp_encode(D, X, s)
+    l_mse, g_mse = mse_loss_and_grad(D, X, res.idx, res.coef)
+    l_div, g_div = div_loss_and_grad(D)
+    W = np.asarray(D, np.float64) - lr * (g_mse + beta * g_div)
+    n = np.linalg.norm(W, axis=1, keepdims=True)
+    W = np.where(n > 0, W / np.where(n > 0, n, 1.0), 0.0)
+    return W.astype(np.float32), l_mse, l_div, res
+
+
 # --- storage format ("Analysis for CSR") -------------------------------------------------
 
 def pack_codes(idx: np.ndarray, coef: np.ndarray):

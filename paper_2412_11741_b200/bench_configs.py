@@ -1,6 +1,6 @@
 """Throughput and reconstruction error of the codec on every synthetic configuration.
 
-  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5,decode,attention] [--reps 30]
+  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5,decode,attention,train] [--reps 30]
 
 One JSON line per case: vectors/s and TFLOP/s of the fast encoder (median of the last two
 thirds of `reps` back-to-back launches, i.e. after the clocks have settled under the power
@@ -121,6 +121,24 @@ def run_attention_case(reps):
             "restore_to_bf16_ms": round(t_rc, 4), "restored_bytes": B * T * d * 2.0, "code_bytes": code_b}
 
 
+def run_train_case(reps):
+    """One NeuralDict training step (N = 8192 atoms, d = 128, s = 8 as in the paper's training,
+    batch of 65536 key-like rows) with the tensor-core encoder as forward pass."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    w = wl.sparsity_sweep(8, tokens=2048)                    # 65536 key-like rows, 8192 atoms
+    D = torch.from_numpy(w.D).to(dev)
+    X = torch.from_numpy(w.X).to(dev).to(torch.bfloat16)
+    losses = torch.empty(2, dtype=torch.float64, device=dev)
+    t = _time(lambda: csr.csr_dict_train_step(D, X, 8, 1e-4, 0.1, mode=csr.CSR_MODE_BF16_FAST, losses=losses), max(5, reps // 3))
+    idx = torch.empty((w.M, 8), dtype=torch.uint16, device=dev)
+    coef = torch.empty((w.M, 8), dtype=torch.float32, device=dev)
+    t_enc = _time(lambda: csr.csr_encode_ex(D, X, 8, out_idx=idx, out_coef=coef), max(5, reps // 3))
+    l = losses.cpu().tolist()
+    return {"case": "neuraldict_train_step", "M": w.M, "N": w.N, "d": w.d, "s": 8, "step_ms": round(t, 4),
+            "encode_part_ms": round(t_enc, 4), "gradient_update_part_ms": round(t - t_enc, 4),
+            "rows_per_s": w.M / (t * 1e-3), "L_MSE": l[0], "L_div": l[1]}
+
+
 def cases(names):
     for n in names:
         if n == "c1":
@@ -142,20 +160,22 @@ def cases(names):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--configs", default="c1,c2,c3,c4,c5,decode,attention")
+    ap.add_argument("--configs", default="c1,c2,c3,c4,c5,decode,attention,train")
     ap.add_argument("--reps", type=int, default=30)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device (there is no CPU fallback)")
     build.build()
     names = args.configs.split(",")
-    for w in cases([n for n in names if n not in ("decode", "attention")]):
+    for w in cases([n for n in names if n not in ("decode", "attention", "train")]):
         print(json.dumps(run_case(w, args.reps)), flush=True)
     if "decode" in names:
         for seqs, kv_heads in ((1, 8), (8, 8), (64, 8)):
             print(json.dumps(run_decode_case(seqs, kv_heads, 8192, 16, args.reps)), flush=True)
     if "attention" in names:
         print(json.dumps(run_attention_case(args.reps)), flush=True)
+    if "train" in names:
+        print(json.dumps(run_train_case(args.reps)), flush=True)
 
 
 if __name__ == "__main__":

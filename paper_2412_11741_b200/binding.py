@@ -33,7 +33,7 @@ CSR_MODE_BF16_FAST = 1
 
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
-    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append", "csr_key_scores", "csr_value_mix",
+    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append", "csr_dict_train_step", "csr_key_scores", "csr_value_mix",
     "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
@@ -60,6 +60,17 @@ class csr_reconstruct_params_t(ctypes.Structure):
         ("d", ctypes.c_int32), ("N", ctypes.c_int32), ("s", ctypes.c_int32), ("reserved1", ctypes.c_int32),
         ("X_hat", ctypes.c_void_p), ("stream", ctypes.c_void_p),
         ("ld_code", ctypes.c_int64), ("ld_xhat", ctypes.c_int64),
+    ]
+
+
+class csr_train_params_t(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("mode", ctypes.c_int32),
+        ("D", ctypes.c_void_p), ("X", ctypes.c_void_p),
+        ("x_dtype", ctypes.c_int32), ("d", ctypes.c_int32), ("N", ctypes.c_int32), ("s", ctypes.c_int32),
+        ("M", ctypes.c_int64),
+        ("lr", ctypes.c_float), ("beta", ctypes.c_float),
+        ("losses", ctypes.c_void_p), ("stream", ctypes.c_void_p),
     ]
 
 
@@ -108,6 +119,8 @@ def lib() -> ctypes.CDLL:
         L.csr_key_scores.restype = i32
         L.csr_value_mix.argtypes = [vp, i32, i32, vp, i32, i32, vp, vp, i32, i64, i32, vp, vp]
         L.csr_value_mix.restype = i32
+        L.csr_dict_train_step.argtypes = [ctypes.POINTER(csr_train_params_t)]
+        L.csr_dict_train_step.restype = i32
         L.csr_device_status.argtypes = [vp]
         L.csr_device_status.restype = i32
         L.csr_release_workspace.argtypes = []
@@ -339,6 +352,30 @@ def csr_value_mix(D: torch.Tensor, W: torch.Tensor, idx: torch.Tensor, coef: tor
         _check(lib().csr_value_mix(D.data_ptr(), N, d, W.data_ptr(), B, H, idx.data_ptr(), coef.data_ptr(),
                                    _TORCH_DTYPE[coef.dtype], T, s, out.data_ptr(), _stream_ptr(D)))
     return out
+
+
+def csr_dict_train_step(D: torch.Tensor, X: torch.Tensor, s: int, lr: float, beta: float, *,
+                        mode: int = CSR_MODE_FP32_EXACT, losses: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """csr_dict_train_step: updates D ([N][d] fp32, CUDA) in place on the batch X ([M][d]);
+    returns the device tensor [L_MSE, L_div] (float64) of the dictionary before the update."""
+    assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.is_contiguous() and D.dtype == torch.float32
+    assert X.dim() == 2 and X.shape[1] == D.shape[1]
+    if losses is None:
+        losses = torch.empty(2, dtype=torch.float64, device=D.device)
+    assert losses.dtype == torch.float64 and losses.numel() >= 2 and losses.is_cuda
+    p = csr_train_params_t()
+    p.struct_size = ctypes.sizeof(csr_train_params_t)
+    p.mode = mode
+    p.D = D.data_ptr()
+    p.X = X.data_ptr()
+    p.x_dtype = _TORCH_DTYPE[X.dtype]
+    p.d, p.N, p.s, p.M = D.shape[1], D.shape[0], s, X.shape[0]
+    p.lr, p.beta = float(lr), float(beta)
+    p.losses = losses.data_ptr()
+    p.stream = _stream_ptr(D)
+    with torch.cuda.device(D.device):
+        _check(lib().csr_dict_train_step(ctypes.byref(p)))
+    return losses
 
 
 def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *,

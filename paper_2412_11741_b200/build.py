@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcsr.so")
-SOURCES = ["attention_ops.cu", "csr_api.cu", "dict_ops.cu", "encode_exact.cu", "encode_exact_split.cu", "encode_fast.cu", "encode_static.cu", "reconstruct.cu"]
+SOURCES = ["attention_ops.cu", "csr_api.cu", "dict_ops.cu", "encode_exact.cu", "encode_exact_split.cu", "encode_fast.cu", "encode_static.cu", "reconstruct.cu", "train_ops.cu"]
 
 
 def _nvcc() -> str:

@@ -86,6 +86,25 @@ size_t attn_scratch_bytes(int B, int H, int N);
 int launch_key_scores(const AttnArgs& a, float* scratch);
 int launch_value_mix(const AttnArgs& a, float* scratch);
 
+// Gradient step of the dictionary on one batch whose codes (idx, fp32 coef, dense [M][s])
+// are given; losses[0] = L_MSE, losses[1] = L_div of the dictionary before the update.
+struct TrainArgs {
+    float* D;
+    int N, d;
+    const void* X;
+    int x_dtype;
+    int64_t M;
+    int s;
+    const uint16_t* idx;
+    const float* coef;
+    float* grad_mse;   // [N][d] scratch
+    float* grad_div;   // [N][d] scratch
+    double* losses;    // [2]
+    float lr, beta;
+    cudaStream_t stream;
+};
+int launch_dict_train(const TrainArgs& a);
+
 int sm_count();
 
 }  // namespace csr

@@ -415,6 +415,71 @@ int csr_value_mix(const void* D, int N, int d, const float* W, int B, int H, con
     return launch_value_mix(a, static_cast<float*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)));
 }
 
+int csr_dict_train_step(const csr_train_params_t* p) {
+    if (!p) return fail(CSR_ERR_INVALID_ARG, "params is NULL");
+    if (p->struct_size != sizeof(csr_train_params_t))
+        return fail(CSR_ERR_INVALID_ARG, "struct_size %u != %zu", p->struct_size, sizeof(csr_train_params_t));
+    if (p->mode != CSR_MODE_FP32_EXACT && p->mode != CSR_MODE_BF16_FAST)
+        return fail(CSR_ERR_INVALID_ARG, "unknown mode %d", p->mode);
+    if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
+    if (p->mode == CSR_MODE_BF16_FAST && (p->N % 128) != 0)
+        return fail(CSR_ERR_UNSUPPORTED, "fast mode needs N %% 128 == 0 (N = %d)", p->N);
+    if (p->x_dtype != CSR_DTYPE_F32 && p->x_dtype != CSR_DTYPE_BF16)
+        return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32 or BF16");
+    if (!p->D || !p->losses || (p->M > 0 && !p->X)) return fail(CSR_ERR_INVALID_ARG, "D, losses or X is NULL");
+    if (!aligned16(p->D) || !aligned16(p->X) || (reinterpret_cast<uintptr_t>(p->losses) % 8))
+        return fail(CSR_ERR_ALIGNMENT, "D and X must be 16-byte aligned, losses 8-byte aligned");
+    if (!(p->lr >= 0.f) || !(p->beta >= 0.f)) return fail(CSR_ERR_INVALID_ARG, "lr and beta must be >= 0");
+    // scratch layout: [encoder's own region][idx][coef][grad_mse][grad_div]
+    size_t enc = encode_fast_workspace_bytes(p->d, p->N);
+    if (p->M > 0 && encode_exact_split_applies(p->M, p->N)) {
+        const size_t sp = encode_exact_split_scratch_bytes(p->M, p->d, p->N);
+        if (sp > enc) enc = sp;
+    }
+    enc = (enc + 1023) / 1024 * 1024;
+    const size_t idx_b = ((size_t)p->M * p->s * 2 + 255) / 256 * 256;
+    const size_t coef_b = ((size_t)p->M * p->s * 4 + 255) / 256 * 256;
+    const size_t g_b = ((size_t)p->N * p->d * 4 + 255) / 256 * 256;
+    void* base = nullptr;
+    if (int rc = ensure_work(enc + idx_b + coef_b + 2 * g_b, &base)) return rc;
+    char* q = static_cast<char*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)) + enc;
+    TrainArgs a;
+    a.D = static_cast<float*>(p->D);
+    a.N = p->N;
+    a.d = p->d;
+    a.X = p->X;
+    a.x_dtype = p->x_dtype;
+    a.M = p->M;
+    a.s = p->s;
+    a.idx = reinterpret_cast<uint16_t*>(q);
+    a.coef = reinterpret_cast<float*>(q + idx_b);
+    a.grad_mse = reinterpret_cast<float*>(q + idx_b + coef_b);
+    a.grad_div = reinterpret_cast<float*>(q + idx_b + coef_b + g_b);
+    a.losses = p->losses;
+    a.lr = p->lr;
+    a.beta = p->beta;
+    a.stream = static_cast<cudaStream_t>(p->stream);
+    if (p->M > 0) {
+        csr_encode_params_t e;
+        memset(&e, 0, sizeof(e));
+        e.struct_size = sizeof(e);
+        e.mode = p->mode;
+        e.D = p->D;
+        e.X = p->X;
+        e.x_dtype = p->x_dtype;
+        e.coef_dtype = CSR_DTYPE_F32;
+        e.M = p->M;
+        e.d = p->d;
+        e.N = p->N;
+        e.s = p->s;
+        e.out_idx = const_cast<uint16_t*>(a.idx);
+        e.out_coef = const_cast<float*>(a.coef);
+        e.stream = p->stream;
+        if (int rc = encode_device(&e)) return rc;      // its ensure_work request is smaller: no regrowth
+    }
+    return launch_dict_train(a);
+}
+
 int csr_encode_host(const csr_encode_params_t* p) {
     if (int rc = check_encode(p, true)) return rc;
     if (p->M == 0) return CSR_OK;

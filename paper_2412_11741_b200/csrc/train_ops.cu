@@ -1,0 +1,193 @@
+// One training step of the offline dictionary ("NeuralDict", Algorithm 1, procedure
+// TrainNeurDict; the MSE loss, the diversity loss L_div = ||I - W^T W||_F^2 / N^2, the complete
+// loss L = L_MSE + beta * L_div and ReNorm).  The sparse codes of the batch are computed by
+// the matching-pursuit encoder before these kernels run and are held fixed while the loss
+// is differentiated (the alternating scheme of dictionary learning), so with
+// e_x = x - W r(x):
+//
+//   dL_MSE / d d_n = -2 * sum over (x, g) with i_g(x) = n of  c_g(x) * e_x
+//   dL_div / d d_n = (4 / N^2) * sum_j (G[n][j] - delta_nj) * d_j,      G = D D^T
+//
+//   mse_grad_kernel   one warp per row: restores x^ from the codes, forms e = x - x^, adds
+//                     ||e||^2 to the loss (fp64 atomic) and scatters -2 c_g e into the
+//                     gradient rows of the s selected atoms (fp32 atomic adds).
+//   div_grad_kernel   one CTA per block of 64 atoms: sweeps all atoms in blocks of 64,
+//                     forms the 64 x 64 block of G - I in shared memory (never in global
+//                     memory), adds its squares to L_div and multiplies it into the
+//                     gradient block held in registers.  No atomics except the loss.
+//   update_kernel     one warp per atom: d_n <- ReNorm(d_n - lr * (g_mse + beta * g_div)).
+#include "common.cuh"
+
+namespace csr {
+namespace {
+
+__device__ __forceinline__ float load_x(const void* X, int x_dtype, int64_t off) {
+    if (x_dtype == CSR_DTYPE_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(X)[off]);
+    return reinterpret_cast<const float*>(X)[off];
+}
+
+template <int D_>
+__global__ void __launch_bounds__(256)
+mse_grad_kernel(const float* __restrict__ D, int N, const void* __restrict__ X, int x_dtype, int64_t M, int s,
+                const uint16_t* __restrict__ idx, const float* __restrict__ coef, float* __restrict__ grad,
+                double* __restrict__ losses) {
+    constexpr int PER = D_ / 32;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    double local = 0.0;
+    for (int64_t m = warp0; m < M; m += nwarps) {
+        float e[PER];
+#pragma unroll
+        for (int k = 0; k < PER; ++k) e[k] = load_x(X, x_dtype, m * D_ + lane * PER + k);
+        for (int g = 0; g < s; ++g) {                     // e = x - sum_g c_g d_{i_g}, stored order
+            int i = idx[m * s + g];
+            i = i < N ? i : N - 1;
+            const float c = coef[m * s + g];
+            const float* dn = D + (int64_t)i * D_ + lane * PER;
+#pragma unroll
+            for (int k = 0; k < PER; ++k) e[k] = fmaf(-c, dn[k], e[k]);
+        }
+        float ss = 0.f;
+#pragma unroll
+        for (int k = 0; k < PER; ++k) ss = fmaf(e[k], e[k], ss);
+        for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        local += (double)ss;
+        for (int g = 0; g < s; ++g) {
+            int i = idx[m * s + g];
+            i = i < N ? i : N - 1;
+            const float c2 = -2.f * coef[m * s + g];
+            float* gn = grad + (int64_t)i * D_ + lane * PER;
+#pragma unroll
+            for (int k = 0; k < PER; ++k) atomicAdd(gn + k, c2 * e[k]);
+        }
+    }
+    if (lane == 0 && local != 0.0) atomicAdd(&losses[0], local);
+}
+
+// CTA = 64 atoms (rows i) against all atoms in blocks of 64 (rows j); 256 threads.
+constexpr int GB = 64;
+template <int D_>
+__global__ void __launch_bounds__(256)
+div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div, double* __restrict__ losses) {
+    extern __shared__ __align__(16) float sm[];
+    float (*Di)[D_ + 1] = reinterpret_cast<float (*)[D_ + 1]>(sm);                        // [GB][D_+1]
+    float (*Dj)[D_ + 1] = reinterpret_cast<float (*)[D_ + 1]>(sm + GB * (D_ + 1));        // [GB][D_+1]
+    float (*Gs)[GB + 1] = reinterpret_cast<float (*)[GB + 1]>(sm + 2 * GB * (D_ + 1));    // [GB][GB+1]
+    const int tid = threadIdx.x;
+    const int i0 = blockIdx.x * GB;
+    for (int f = tid; f < GB * D_; f += 256) {
+        const int r = f / D_, k = f % D_;
+        Di[r][k] = (i0 + r < N) ? D[(int64_t)(i0 + r) * D_ + k] : 0.f;
+    }
+    // gradient block: thread owns row gi = tid / 4 and channels (tid % 4) + 4 * q
+    constexpr int CPT = D_ / 4;
+    const int gi = tid >> 2, gc = tid & 3;
+    float acc[CPT];
+#pragma unroll
+    for (int q = 0; q < CPT; ++q) acc[q] = 0.f;
+    // G block: thread owns a 4 x 4 patch: rows (tid / 16) * 4 .., columns (tid % 16) * 4 ..
+    const int pr = (tid >> 4) * 4, pc = (tid & 15) * 4;
+    double lsum = 0.0;
+    for (int j0 = 0; j0 < N; j0 += GB) {
+        __syncthreads();
+        for (int f = tid; f < GB * D_; f += 256) {
+            const int r = f / D_, k = f % D_;
+            Dj[r][k] = (j0 + r < N) ? D[(int64_t)(j0 + r) * D_ + k] : 0.f;
+        }
+        __syncthreads();
+        float g[4][4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) g[a][b] = 0.f;
+        for (int k = 0; k < D_; ++k) {
+            float x[4], y[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) x[a] = Di[pr + a][k];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) y[b] = Dj[pc + b][k];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) g[a][b] = fmaf(x[a], y[b], g[a][b]);
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int i = i0 + pr + a, j = j0 + pc + b;
+                float v = g[a][b] - (i == j ? 1.f : 0.f);
+                if (i >= N || j >= N) v = 0.f;
+                Gs[pr + a][pc + b] = v;
+                lsum += (double)v * (double)v;
+            }
+        __syncthreads();
+        // acc[gi][c] += sum_j (G - I)[gi][j] * Dj[j][c]
+        for (int j = 0; j < GB; ++j) {
+            const float w = Gs[gi][j];
+#pragma unroll
+            for (int q = 0; q < CPT; ++q) acc[q] = fmaf(w, Dj[j][gc + 4 * q], acc[q]);
+        }
+    }
+    const float scale = 4.0f / ((float)N * (float)N);
+    if (i0 + gi < N) {
+#pragma unroll
+        for (int q = 0; q < CPT; ++q) grad_div[(int64_t)(i0 + gi) * D_ + gc + 4 * q] = scale * acc[q];
+    }
+    for (int o = 16; o; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+    if ((tid & 31) == 0) atomicAdd(&losses[1], lsum / ((double)N * (double)N));
+}
+
+template <int D_>
+__global__ void update_kernel(float* __restrict__ D, int N, const float* __restrict__ grad_mse,
+                              const float* __restrict__ grad_div, float lr, float beta) {
+    constexpr int PER = D_ / 32;
+    const int lane = threadIdx.x & 31;
+    const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (n >= N) return;
+    float w[PER];
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+        const int64_t o = (int64_t)n * D_ + lane * PER + k;
+        w[k] = D[o] - lr * fmaf(beta, grad_div[o], grad_mse[o]);
+        ss = fmaf(w[k], w[k], ss);
+    }
+    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const float inv = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) D[(int64_t)n * D_ + lane * PER + k] = w[k] * inv;
+}
+
+template <int D_>
+int run(const TrainArgs& a) {
+    const size_t gbytes = (size_t)a.N * D_ * sizeof(float);
+    cudaError_t e = cudaMemsetAsync(a.grad_mse, 0, gbytes, a.stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(a.losses, 0, 2 * sizeof(double), a.stream);
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    if (a.M > 0) {
+        int64_t blocks = (a.M + 7) / 8;
+        const int64_t cap = (int64_t)sm_count() * 8;
+        if (blocks > cap) blocks = cap;
+        mse_grad_kernel<D_><<<(int)blocks, 256, 0, a.stream>>>(a.D, a.N, a.X, a.x_dtype, a.M, a.s, a.idx, a.coef,
+                                                              a.grad_mse, a.losses);
+    }
+    const size_t smem = (size_t)(2 * GB * (D_ + 1) + GB * (GB + 1)) * sizeof(float);
+    e = cudaFuncSetAttribute(div_grad_kernel<D_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    div_grad_kernel<D_><<<(a.N + GB - 1) / GB, 256, smem, a.stream>>>(a.D, a.N, a.grad_div, a.losses);
+    update_kernel<D_><<<(a.N + 7) / 8, 256, 0, a.stream>>>(a.D, a.N, a.grad_mse, a.grad_div, a.lr, a.beta);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "dict_train launch: %s", cudaGetErrorString(e));
+    return CSR_OK;
+}
+
+}  // namespace
+
+int launch_dict_train(const TrainArgs& a) {
+    if (a.d == 128) return run<128>(a);
+    return run<64>(a);
+}
+
+}  // namespace csr

@@ -168,3 +168,32 @@ def test_scores_from_codes_equal_scores_from_the_restored_tensor(csr):
     ref = torch.einsum("bhd,btd->bht", Q.double(), xh.double())
     tol = 2e-6 * (Q.norm(dim=2)[:, :, None] * coef.float().abs().sum(1).view(32, 1, T))
     assert bool(((sc.double() - ref).abs() <= tol.double() + 1e-30).all())
+
+
+@pytest.mark.parametrize("N,d,M,s", [(256, 128, 3000, 8), (200, 64, 1000, 4)])
+def test_dictionary_training_step_matches_oracle(csr, N, d, M, s):
+    """One batch of NeuralDict training (matching pursuit forward, both gradients, gradient
+    step, ReNorm) against the oracle; then the adaptive weight and a few more steps."""
+    rng = np.random.default_rng(N + M)
+    D0 = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    X = rng.standard_normal((M, d)).astype(np.float32)
+    lr, beta = 1e-3, 0.7
+    Dd = torch.from_numpy(D0.copy()).to(DEV)
+    Xd = torch.from_numpy(X).to(DEV)
+    losses = csr.csr_dict_train_step(Dd, Xd, s, lr, beta).cpu().numpy()
+    want_D, l_mse, l_div, res = orc.dict_train_step(D0, X, s, lr, beta)
+    assert res.gap.min() > 2e-6                              # no tie in this batch: same codes on both sides
+    assert losses[0] == pytest.approx(l_mse, rel=2e-6) and losses[1] == pytest.approx(l_div, rel=2e-5)
+    got = Dd.cpu().numpy()
+    assert np.abs(got - want_D).max() <= 2e-6
+    assert np.allclose(np.linalg.norm(got.astype(np.float64), axis=1), 1.0, atol=3e-7)
+    moved = np.abs(got - D0).max(axis=1) > 0
+    assert moved.all()                                       # the diversity term reaches every atom
+    # a short run with the adaptive weight lowers the MSE loss on this batch; the tensor-core
+    # encoder may drive the forward pass just as well
+    first = losses[0]
+    for mode in (csr.CSR_MODE_FP32_EXACT,) * 8 + ((csr.CSR_MODE_BF16_FAST,) * 4 if N % 128 == 0 else ()):
+        beta = orc.adaptive_beta(float(losses[0]), float(losses[1]))
+        losses = csr.csr_dict_train_step(Dd, Xd, s, 2e-3, beta, mode=mode).cpu().numpy()
+    assert csr.csr_device_status() == csr.CSR_OK
+    assert losses[0] < first and np.isfinite(losses).all()

@@ -379,3 +379,58 @@ def test_attention_from_codes_closed_forms():
     q = rng.standard_normal((1, 1, d))
     sc = orc.key_scores(Dn, q, res.idx[None], res.coef[None])
     assert np.allclose(sc[0, 0] + res.residual @ q[0, 0], X.astype(np.float64) @ q[0, 0], atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------
+# one training step of the offline dictionary
+# ---------------------------------------------------------------------------------------
+
+def test_training_gradients_match_finite_differences():
+    """Both gradients against central differences of the losses themselves (codes fixed)."""
+    rng = np.random.default_rng(21)
+    N, d, M, s = 12, 6, 30, 3
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    X = rng.standard_normal((M, d)).astype(np.float32)
+    res = orc.mp_encode(D, X, s)
+    l0, g_mse = orc.mse_loss_and_grad(D, X, res.idx, res.coef)
+    _, g_div = orc.div_loss_and_grad(D)
+    h = 1e-3                                              # fp32 storage of D limits the step size
+    for (n, k) in [(0, 0), (3, 2), (7, 5), (11, 1), (int(res.idx[0, 0]), 4)]:
+        Dp, Dm = D.copy(), D.copy()
+        Dp[n, k] += np.float32(h)
+        Dm[n, k] -= np.float32(h)
+        step = float(Dp[n, k]) - float(Dm[n, k])
+        fd = (orc.mse_loss_and_grad(Dp, X, res.idx, res.coef)[0] - orc.mse_loss_and_grad(Dm, X, res.idx, res.coef)[0]) / step
+        assert abs(fd - g_mse[n, k]) <= 1e-3 * max(1.0, abs(fd)), (n, k, fd, g_mse[n, k])
+        fd = (orc.div_loss_and_grad(Dp)[0] - orc.div_loss_and_grad(Dm)[0]) / step
+        assert abs(fd - g_div[n, k]) <= 1e-3 * max(1e-3, abs(fd)), (n, k, fd, g_div[n, k])
+    assert l0 == pytest.approx(float(np.sum(res.resnorm[:, -1] ** 2)), rel=1e-12)   # L_MSE is the squared MP residual
+
+
+def test_diversity_loss_closed_forms_and_beta():
+    """Orthonormal atoms: L_div = 0 and zero gradient; two copies of one atom among
+    orthonormal ones: ||I - G||_F^2 = 2, so L_div = 2 / N^2; beta's cap and ratio."""
+    Q = np.linalg.qr(np.random.default_rng(2).standard_normal((8, 8)))[0].astype(np.float64)
+    l, g = orc.div_loss_and_grad(Q)
+    assert l < 1e-28 and np.abs(g).max() < 1e-14
+    D = Q[:5].copy()
+    D[4] = D[0]
+    l, _ = orc.div_loss_and_grad(D)
+    assert l == pytest.approx(2.0 / 25.0, rel=1e-12)
+    assert orc.adaptive_beta(5.0, 1.0) == 0.5 and orc.adaptive_beta(50.0, 1.0) == 1.0 and orc.adaptive_beta(1.0, 0.0) == 1.0
+
+
+def test_training_steps_renormalise_and_lower_the_loss():
+    rng = np.random.default_rng(22)
+    N, d, M, s = 64, 16, 400, 4
+    basis = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    codes = rng.integers(0, N, (M, 2))
+    X = (basis[codes[:, 0]] * 2 + basis[codes[:, 1]] + 0.05 * rng.standard_normal((M, d))).astype(np.float32)
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    beta, first = 0.0, None
+    for it in range(30):
+        D, l_mse, l_div, _ = orc.dict_train_step(D, X, s, lr=2e-3, beta=beta)
+        beta = orc.adaptive_beta(l_mse, l_div)
+        first = l_mse if first is None else first
+        assert np.allclose(np.linalg.norm(D.astype(np.float64), axis=1), 1.0, atol=1e-6)
+    assert l_mse < 0.8 * first
