@@ -71,7 +71,9 @@ extern "C" {
  *   CSR_MODE_BF16_FAST   correlations on the tcgen05 tensor cores with bf16 operands
  *                        (residual and atoms rounded to bf16) and fp32 accumulation.
  *                        Near-tied picks may differ from an fp64 evaluation; the mean
- *                        reconstruction error does not.  The environment variable
+ *                        reconstruction error does not, down to a floor of about
+ *                        2^-8 * ||x|| (the residual is carried in bf16); use the exact
+ *                        mode for errors below 1e-2 * ||x||.  The environment variable
  *                        CSR_FAST_GROUP (1, 2, 4 or 8) overrides the arg-max group size
  *                        the kernel would choose; every setting meets the same gates.
  */

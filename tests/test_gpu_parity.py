@@ -330,6 +330,40 @@ def test_fast_every_group_size(csr, G, d, monkeypatch):
         assert rep.ok, (G, d, N, rep.detail)
 
 
+def test_largest_dictionary_and_most_iterations(csr):
+    """The limits of the interface: N = 65536 (indices fill the uint16 range) and s = 64, in
+    both modes, against the oracle."""
+    rng = np.random.default_rng(65536)
+    N, d, M, s = 65536, 64, 192, 64
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    X = wl.round_to_bf16(rng.standard_normal((M, d)).astype(np.float32))
+    X[3] = D[65535] * np.float32(2.0)                     # the last atom must be reachable
+    X = wl.round_to_bf16(X)
+    w = wl.Workload("limits", D, X, s, "bf16")
+    res = orc.mp_encode(D, X, s)
+    idx, coef = _encode(csr, w, X, csr.CSR_MODE_FP32_EXACT)
+    rep = parity.compare_exact(D, X, s, idx, coef, res)
+    assert rep.ok, rep.detail
+    assert idx[3, 0] == 65535 and int(idx.max()) > 60000
+    # Fast mode at s = d with 65536 atoms: the oracle drives the error down to 5e-5 of ||x||.
+    # The fast mode carries its residual in bf16, and the rounding of every intermediate
+    # residual (2^-9 of its size) stays in the true error for good, so its error cannot
+    # fall below about 2^-8 ||x|| (mean 3e-3, worst row 4e-3 here); down to that floor it
+    # must follow the oracle.
+    idx, coef = _encode(csr, w, X, csr.CSR_MODE_BF16_FAST)
+    assert int(idx.max()) < N and idx[3, 0] == 65535
+    e_gpu = orc.relative_error(X, orc.reconstruct(D, idx.astype(np.int32), coef.astype(np.float64)))
+    e_or = res.resnorm[:, -1] / np.linalg.norm(X.astype(np.float64), axis=1)
+    assert e_or.mean() < 1e-4
+    assert np.all(e_gpu <= 1.05 * e_or + 2.0 ** -7.5) and e_gpu.mean() < 2.0 ** -8, float(e_gpu.max())
+    # and at s = 16, where the error (0.1) is far above the floor, the usual gates hold
+    # (row 3 is left out: it is one atom up to bf16 rounding, so after its first step both
+    # sides chase rounding noise)
+    keep = np.arange(M) != 3
+    rep = parity.compare_fast(D, X[keep], 16, idx[keep, :16], coef[keep, :16])
+    assert rep.ok, rep.detail
+
+
 # ---------------------------------------------------------------------------------------
 # de-sparse
 # ---------------------------------------------------------------------------------------
