@@ -23,8 +23,7 @@
  *     idx [M][s] and coef [M][s] row-major, entry g of a row being iteration g of the
  *     pursuit.
  *   - Limits: d in {64, 128}; 1 <= N <= 65536 (indices are stored as uint16); 1 <= s <= 64;
- *     M >= 0 (M == 0 succeeds and does nothing).  The fast mode additionally needs
- *     N % 128 == 0.  Data pointers must be 16-byte aligned.
+ *     M >= 0 (M == 0 succeeds and does nothing).  Data pointers must be 16-byte aligned.
  *   - NaN or Inf in X or D: results are unspecified; the call neither crashes nor hangs.
  *   - Device-side waits are bounded.  If one expires the kernel stops early, the outputs
  *     are unspecified and csr_device_status() reports CSR_ERR_TIMEOUT.
@@ -274,7 +273,8 @@ int csr_reconstruct_host(const csr_reconstruct_params_t* p);
  * other allocating routine.
  *
  * Limits and rules
- *   - N * d <= CSR_STATIC_MAX_DICT_ELEMS (8192 atoms of 128 channels, a 2 MiB bf16 copy);
+ *   - N8 * d <= CSR_STATIC_MAX_DICT_ELEMS with N8 = N rounded up to a multiple of 8 (8192
+ *     atoms of 128 channels, a 2 MiB bf16 copy);
  *     larger dictionaries are rejected with CSR_ERR_UNSUPPORTED.  Every GPU on which the
  *     library is loaded holds the array (2 MiB + 2 KiB) until the process exits.
  *   - The first call on a device looks up the array's device address, once, with that

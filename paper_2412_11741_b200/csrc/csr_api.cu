@@ -108,8 +108,6 @@ int check_encode(const csr_encode_params_t* p, bool host_io) {
         return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32 or BF16");
     if (p->coef_dtype != CSR_DTYPE_F32 && p->coef_dtype != CSR_DTYPE_F16)
         return fail(CSR_ERR_INVALID_ARG, "coef_dtype must be F32 or F16");
-    if (p->mode == CSR_MODE_BF16_FAST && (p->N % 128) != 0)
-        return fail(CSR_ERR_UNSUPPORTED, "fast mode needs N %% 128 == 0 (N = %d); pad D with zero atoms", p->N);
     if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
     if (p->M > 0 && (!p->X || !p->out_idx || !p->out_coef))
         return fail(CSR_ERR_INVALID_ARG, "X, out_idx or out_coef is NULL");
@@ -422,8 +420,6 @@ int csr_dict_train_step(const csr_train_params_t* p) {
     if (p->mode != CSR_MODE_FP32_EXACT && p->mode != CSR_MODE_BF16_FAST)
         return fail(CSR_ERR_INVALID_ARG, "unknown mode %d", p->mode);
     if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
-    if (p->mode == CSR_MODE_BF16_FAST && (p->N % 128) != 0)
-        return fail(CSR_ERR_UNSUPPORTED, "fast mode needs N %% 128 == 0 (N = %d)", p->N);
     if (p->x_dtype != CSR_DTYPE_F32 && p->x_dtype != CSR_DTYPE_BF16)
         return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32 or BF16");
     if (!p->D || !p->losses || (p->M > 0 && !p->X)) return fail(CSR_ERR_INVALID_ARG, "D, losses or X is NULL");

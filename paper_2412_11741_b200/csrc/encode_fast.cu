@@ -738,7 +738,10 @@ int launch_d(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, u
 
 }  // namespace
 
-size_t encode_fast_workspace_bytes(int d, int N) { return (size_t)N * (size_t)d * 2; }
+// The bf16 copy holds N rounded up to a multiple of 8 atoms; the extra rows are zero, so a
+// group of up to 8 candidate atoms never reaches past the copy.
+static int padded_atoms(int N) { return (N + 7) / 8 * 8; }
+size_t encode_fast_workspace_bytes(int d, int N) { return (size_t)padded_atoms(N) * (size_t)d * 2; }
 
 int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status) {
     if (a.M == 0) return CSR_OK;
@@ -755,9 +758,16 @@ int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status) {
                                                       reinterpret_cast<uint2*>(workspace), n_vec4);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "dict_to_bf16 launch: %s", cudaGetErrorString(e));
+    const int n_pad = padded_atoms(a.N);
+    if (n_pad > a.N) {
+        e = cudaMemsetAsync(static_cast<char*>(workspace) + (size_t)a.N * a.d * 2, 0, (size_t)(n_pad - a.N) * a.d * 2,
+                            a.stream);
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    }
 
+    // rows past the padded copy (the rest of the last 256-atom tile) are filled with zeros by TMA
     CUtensorMap tmap;
-    const cuuint64_t gdim[2] = {(cuuint64_t)a.d, (cuuint64_t)a.N};
+    const cuuint64_t gdim[2] = {(cuuint64_t)a.d, (cuuint64_t)n_pad};
     const cuuint64_t gstride[1] = {(cuuint64_t)a.d * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)TILE_N};
     const cuuint32_t estr[2] = {1, 1};

@@ -56,10 +56,9 @@ extern "C" int csr_encode_static(const void* D, const void* X, int64_t M, int d,
                                  void* out_coef, void* stream, uint32_t* dev_status) {
     if (d != 64 && d != 128) return fail(CSR_ERR_UNSUPPORTED, "d = %d: only 64 and 128 are supported", d);
     if (N < 1 || N > 65536) return fail(CSR_ERR_INVALID_ARG, "N = %d outside [1, 65536]", N);
-    if ((N % 128) != 0) return fail(CSR_ERR_UNSUPPORTED, "N = %d is not a multiple of 128; pad D with zero atoms", N);
     if (s < 1 || s > 64) return fail(CSR_ERR_INVALID_ARG, "s = %d outside [1, 64]", s);
     if (M < 0) return fail(CSR_ERR_INVALID_ARG, "M = %lld is negative", (long long)M);
-    if ((size_t)N * (size_t)d > kStaticMaxDictElems)
+    if (encode_fast_workspace_bytes(d, N) > kStaticMaxDictElems * 2)
         return fail(CSR_ERR_UNSUPPORTED,
                     "dictionary of N*d = %zu elements exceeds the static scratch (CSR_STATIC_MAX_DICT_ELEMS = %zu); "
                     "use csr_encode_ex with a caller workspace",

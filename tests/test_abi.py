@@ -53,7 +53,7 @@ def _params(binding, **kw):
 
 @pytest.mark.parametrize("kw,code", [
     (dict(d=96), -2), (dict(N=0), -1), (dict(N=70000), -1), (dict(s=0), -1), (dict(s=65), -1), (dict(M=-1), -1),
-    (dict(N=1000), -2), (dict(D=0), -1), (dict(X=0), -1), (dict(out_idx=0), -1), (dict(D=0x1008), -3),
+    (dict(D=0), -1), (dict(X=0), -1), (dict(out_idx=0), -1), (dict(D=0x1008), -3),
     (dict(X=0x2004), -3), (dict(mode=7), -1), (dict(x_dtype=2), -1), (dict(coef_dtype=1), -1),
     (dict(struct_size=8), -1), (dict(workspace=0x5008), -3),
 ])

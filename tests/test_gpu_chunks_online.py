@@ -192,7 +192,7 @@ def test_dictionary_training_step_matches_oracle(csr, N, d, M, s):
     # a short run with the adaptive weight lowers the MSE loss on this batch; the tensor-core
     # encoder may drive the forward pass just as well
     first = losses[0]
-    for mode in (csr.CSR_MODE_FP32_EXACT,) * 8 + ((csr.CSR_MODE_BF16_FAST,) * 4 if N % 128 == 0 else ()):
+    for mode in (csr.CSR_MODE_FP32_EXACT,) * 8 + (csr.CSR_MODE_BF16_FAST,) * 4:
         beta = orc.adaptive_beta(float(losses[0]), float(losses[1]))
         losses = csr.csr_dict_train_step(Dd, Xd, s, 2e-3, beta, mode=mode).cpu().numpy()
     assert csr.csr_device_status() == csr.CSR_OK

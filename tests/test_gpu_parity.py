@@ -210,6 +210,29 @@ def test_fast_ragged_rows_match_full_tiles(csr, M):
         assert rep.mean_ratio < 1.05 and rep.ratio_max < 1.5, rep
 
 
+@pytest.mark.parametrize("N", [1, 5, 100, 1000, 4100])
+@pytest.mark.parametrize("G", [0, 8])
+def test_fast_any_dictionary_size(csr, N, G, monkeypatch):
+    """N need not be a multiple of anything: the bf16 copy is padded with zero atoms, which
+    are never selected (indices stay below N) unless the residual is zero (then atom 0)."""
+    if G:
+        monkeypatch.setenv("CSR_FAST_GROUP", str(G))
+    rng = np.random.default_rng(N)
+    D = wl.normalise_rows(rng.standard_normal((N, 128)).astype(np.float32))
+    X = wl.round_to_bf16(rng.standard_normal((600, 128)).astype(np.float32))
+    X[11] = 0.0
+    s = 4
+    idx, coef = _encode(csr, wl.Workload("anyN", D, X, s, "bf16"), X, csr.CSR_MODE_BF16_FAST)
+    assert int(idx.max()) < N and idx[11].tolist() == [0] * s and np.all(coef[11] == 0)
+    if N >= 5:
+        rep = parity.compare_fast(D, X, s, idx, coef, max_gap=2.0 ** -3 if N < 100 else 2.0 ** -4)
+        assert rep.ok, rep.detail
+    else:                                                 # one atom: every step projects onto it
+        res = orc.mp_encode(D, X, s)
+        xn = np.linalg.norm(X.astype(np.float64), axis=1)
+        assert np.array_equal(idx, res.idx) and np.all(np.abs(coef[:, 0] - res.coef[:, 0]) <= 2.0 ** -8 * xn)   # bf16 atom
+
+
 def test_fast_fp32_input_and_odd_s(csr):
     rng = np.random.default_rng(13)
     D = wl.normalise_rows(rng.standard_normal((1024, 128)).astype(np.float32))
