@@ -35,45 +35,54 @@ __device__ __forceinline__ float load_q(const void* Q, int q_dtype, int64_t off)
 }
 
 // ---- P[r][n] = scale * Q[r][:] . D[n][:]  (r = b*H + h) -----------------------------------
-// CTA = 64 atoms x all rows, 16 rows at a time; thread = (atom, group of 4 rows).
+// CTA = 64 atoms x 64 rows; thread = 4 rows x 4 atoms; channels staged 32 at a time,
+// transposed, and summed in ascending order.
 constexpr int PA = 64;    // atoms per CTA
-constexpr int PR = 16;    // rows per pass
 constexpr int QROWS = 64; // rows per CTA (grid.y)
+constexpr int PK = 32;    // channels per staged block
 template <int D_>
 __global__ void __launch_bounds__(NT)
 qd_kernel(const float* __restrict__ D, int N, const void* __restrict__ Q, int q_dtype, int R, float scale,
           float* __restrict__ P) {
-    __shared__ float Ds[PA][D_ + 1];
-    __shared__ __align__(16) float Qs[PR][D_];
-    const int n0 = blockIdx.x * PA;
-    for (int f = threadIdx.x; f < PA * D_; f += NT) {
-        const int a = f / D_, k = f % D_;
-        Ds[a][k] = (n0 + a < N) ? D[(int64_t)(n0 + a) * D_ + k] : 0.f;
+    __shared__ __align__(16) float Ds[PK][PA + 4];         // Ds[k][atom]
+    __shared__ __align__(16) float Qs[PK][QROWS + 4];      // Qs[k][row]
+    const int n0 = blockIdx.x * PA, r0 = blockIdx.y * QROWS;
+    const int ta = (threadIdx.x & 15) * 4, tr = (threadIdx.x >> 4) * 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int k0 = 0; k0 < D_; k0 += PK) {
+        __syncthreads();
+        for (int f = threadIdx.x; f < PA * PK; f += NT) {
+            const int a = f / PK, k = f % PK;
+            Ds[k][a] = (n0 + a < N) ? D[(int64_t)(n0 + a) * D_ + k0 + k] : 0.f;
+        }
+        for (int f = threadIdx.x; f < QROWS * PK; f += NT) {
+            const int r = f / PK, k = f % PK;
+            Qs[k][r] = (r0 + r < R) ? load_q(Q, q_dtype, (int64_t)(r0 + r) * D_ + k0 + k) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int k = 0; k < PK; ++k) {
+            const float4 dv = *reinterpret_cast<const float4*>(&Ds[k][ta]);
+            const float4 qv = *reinterpret_cast<const float4*>(&Qs[k][tr]);
+            const float d[4] = {dv.x, dv.y, dv.z, dv.w};
+            const float q[4] = {qv.x, qv.y, qv.z, qv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(q[i], d[j], acc[i][j]);
+        }
     }
-    const int a = threadIdx.x % PA, rg = threadIdx.x / PA;     // rows rg*4 .. rg*4+3 of the pass
-    const int r_end = min(R, (int)(blockIdx.y + 1) * QROWS);
-    for (int r0 = blockIdx.y * QROWS; r0 < r_end; r0 += PR) {
-        __syncthreads();
-        for (int f = threadIdx.x; f < PR * D_; f += NT) {
-            const int r = f / D_, k = f % D_;
-            Qs[r][k] = (r0 + r < R) ? load_q(Q, q_dtype, (int64_t)(r0 + r) * D_ + k) : 0.f;
-        }
-        __syncthreads();
-        float acc[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[i] = 0.f;
-        for (int k = 0; k < D_; k += 4) {
-            const float d0 = Ds[a][k], d1 = Ds[a][k + 1], d2 = Ds[a][k + 2], d3 = Ds[a][k + 3];
+    for (int i = 0; i < 4; ++i) {
+        const int r = r0 + tr + i;
+        if (r < R) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float4 q = *reinterpret_cast<const float4*>(&Qs[rg * 4 + i][k]);
-                acc[i] = fmaf(q.w, d3, fmaf(q.z, d2, fmaf(q.y, d1, fmaf(q.x, d0, acc[i]))));
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int r = r0 + rg * 4 + i;
-            if (r < R && n0 + a < N) P[(int64_t)r * N + n0 + a] = scale * acc[i];
+            for (int j = 0; j < 4; ++j)
+                if (n0 + ta + j < N) P[(int64_t)r * N + n0 + ta + j] = scale * acc[i][j];
         }
     }
 }
@@ -153,120 +162,171 @@ __device__ __forceinline__ void load_codes8(const uint16_t* idx, const void* coe
 }
 
 // ---- code streams --------------------------------------------------------------------------
-// blockIdx.x = code stream, blockIdx.y = token range; dynamic smem: HG * N floats.
+// Work = (code stream, chunk of CHUNK_T tokens); each persistent CTA takes a contiguous,
+// balanced range of it, so it changes stream (and reloads its shared-memory table) at most
+// a few times.  The table is interleaved, tab[atom][HGP] with HGP = 1, 2, 4 or 8 query heads
+// side by side, so that one vector access per stored entry serves all heads of the group.
+constexpr int CHUNK_T = 1024;
+
+template <int HGP>
+struct HeadVec {
+    float v[HGP];
+};
+template <int HGP>
+__device__ __forceinline__ HeadVec<HGP> load_heads(const float* p) {
+    HeadVec<HGP> r;
+    if constexpr (HGP == 1) {
+        r.v[0] = p[0];
+    } else if constexpr (HGP == 2) {
+        const float2 t = *reinterpret_cast<const float2*>(p);
+        r.v[0] = t.x;
+        r.v[1] = t.y;
+    } else {
+#pragma unroll
+        for (int q = 0; q < HGP / 4; ++q) {
+            const float4 t = *reinterpret_cast<const float4*>(p + 4 * q);
+            r.v[4 * q + 0] = t.x;
+            r.v[4 * q + 1] = t.y;
+            r.v[4 * q + 2] = t.z;
+            r.v[4 * q + 3] = t.w;
+        }
+    }
+    return r;
+}
+
+// Calls f(g, atom, coef) for the s stored entries of the token whose codes start at `o`.
+template <typename F>
+__device__ __forceinline__ void for_each_code(const uint16_t* idx, const void* coef, int coef_dtype, int64_t o, int s, int N,
+                                              int vec, F&& f) {
+    if (vec) {
+        for (int g0 = 0; g0 < s; g0 += 8) {
+            int i8[8];
+            float c8[8];
+            load_codes8(idx, coef, coef_dtype, o + g0, i8, c8);
+#pragma unroll
+            for (int g = 0; g < 8; ++g) f(i8[g] < N ? i8[g] : N - 1, c8[g]);
+        }
+    } else {
+        for (int g = 0; g < s; ++g) {
+            const int i = idx[o + g];
+            f(i < N ? i : N - 1, load_coef(coef, coef_dtype, o + g));
+        }
+    }
+}
+
+template <int HGP>
 __global__ void __launch_bounds__(NTS)
-key_scores_kernel(const float* __restrict__ P, int N, int H, int HG, const uint16_t* __restrict__ idx,
-                  const void* __restrict__ coef, int coef_dtype, int64_t T, int s, int vec, int64_t tokens_per_cta,
-                  float* __restrict__ scores) {
-    extern __shared__ __align__(16) float p[];             // [HG][N]
-    const int b = blockIdx.x;
-    const int64_t t0 = (int64_t)blockIdx.y * tokens_per_cta;
-    const int64_t t1 = t0 + tokens_per_cta < T ? t0 + tokens_per_cta : T;
-    for (int h0 = 0; h0 < H; h0 += HG) {
-        const int hg = H - h0 < HG ? H - h0 : HG;
-        __syncthreads();
-        const float* src = P + ((int64_t)b * H + h0) * N;
-        for (int j = threadIdx.x; j < hg * N; j += NTS) p[j] = src[j];
-        __syncthreads();
-        for (int64_t t = t0 + threadIdx.x; t < t1; t += NTS) {
-            const int64_t o = ((int64_t)b * T + t) * s;
-            float acc[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) acc[h] = 0.f;
-            if (vec) {
-                for (int g0 = 0; g0 < s; g0 += 8) {
-                    int i8[8];
-                    float c8[8];
-                    load_codes8(idx, coef, coef_dtype, o + g0, i8, c8);
-#pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        const int i = i8[g] < N ? i8[g] : N - 1;
-#pragma unroll
-                        for (int h = 0; h < 8; ++h)
-                            if (h < hg) acc[h] = fmaf(c8[g], p[h * N + i], acc[h]);
-                    }
-                }
-            } else {
-                for (int g = 0; g < s; ++g) {
-                    int i = idx[o + g];
-                    i = i < N ? i : N - 1;
-                    const float c = load_coef(coef, coef_dtype, o + g);
-#pragma unroll
-                    for (int h = 0; h < 8; ++h)
-                        if (h < hg) acc[h] = fmaf(c, p[h * N + i], acc[h]);
-                }
+key_scores_kernel(const float* __restrict__ P, int N, int B, int H, const uint16_t* __restrict__ idx,
+                  const void* __restrict__ coef, int coef_dtype, int64_t T, int s, int vec, float* __restrict__ scores) {
+    extern __shared__ __align__(16) float tab[];           // [N][HGP]
+    const int64_t chunks_per_b = (T + CHUNK_T - 1) / CHUNK_T;
+    const int64_t total = (int64_t)B * chunks_per_b;
+    const int64_t w0 = total * blockIdx.x / gridDim.x, w1 = total * (blockIdx.x + 1) / gridDim.x;
+    for (int h0 = 0; h0 < H; h0 += HGP) {
+        const int hg = H - h0 < HGP ? H - h0 : HGP;
+        int cur_b = -1;
+        for (int64_t w = w0; w < w1; ++w) {
+            const int b = (int)(w / chunks_per_b);
+            if (b != cur_b) {
+                __syncthreads();
+                const float* src = P + ((int64_t)b * H + h0) * N;
+                for (int j = threadIdx.x; j < hg * N; j += NTS) tab[(j % N) * HGP + j / N] = src[j];
+                __syncthreads();
+                cur_b = b;
             }
+            const int64_t t = (w % chunks_per_b) * CHUNK_T + threadIdx.x;
+            if (t >= T) continue;
+            float acc[HGP];
 #pragma unroll
-            for (int h = 0; h < 8; ++h)
+            for (int h = 0; h < HGP; ++h) acc[h] = 0.f;
+            for_each_code(idx, coef, coef_dtype, ((int64_t)b * T + t) * s, s, N, vec, [&](int i, float c) {
+                const HeadVec<HGP> pv = load_heads<HGP>(tab + i * HGP);
+#pragma unroll
+                for (int h = 0; h < HGP; ++h) acc[h] = fmaf(c, pv.v[h], acc[h]);
+            });
+#pragma unroll
+            for (int h = 0; h < HGP; ++h)
                 if (h < hg) scores[((int64_t)b * H + h0 + h) * T + t] = acc[h];
         }
     }
 }
 
+template <int HGP>
 __global__ void __launch_bounds__(NTS)
-value_scatter_kernel(int N, const float* __restrict__ W, int H, int HG, const uint16_t* __restrict__ idx,
-                     const void* __restrict__ coef, int coef_dtype, int64_t T, int s, int vec, int64_t tokens_per_cta,
-                     float* __restrict__ A) {
-    extern __shared__ __align__(16) float a[];             // [HG][N]
-    const int b = blockIdx.x;
-    const int64_t t0 = (int64_t)blockIdx.y * tokens_per_cta;
-    const int64_t t1 = t0 + tokens_per_cta < T ? t0 + tokens_per_cta : T;
-    for (int h0 = 0; h0 < H; h0 += HG) {
-        const int hg = H - h0 < HG ? H - h0 : HG;
-        __syncthreads();
-        for (int j = threadIdx.x; j < hg * N; j += NTS) a[j] = 0.f;
-        __syncthreads();
-        for (int64_t t = t0 + threadIdx.x; t < t1; t += NTS) {
-            const int64_t o = ((int64_t)b * T + t) * s;
-            float w[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) w[h] = h < hg ? W[((int64_t)b * H + h0 + h) * T + t] : 0.f;
-            if (vec) {
-                for (int g0 = 0; g0 < s; g0 += 8) {
-                    int i8[8];
-                    float c8[8];
-                    load_codes8(idx, coef, coef_dtype, o + g0, i8, c8);
-#pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        const int i = i8[g] < N ? i8[g] : N - 1;
-#pragma unroll
-                        for (int h = 0; h < 8; ++h)
-                            if (h < hg) atomicAdd(&a[h * N + i], w[h] * c8[g]);
-                    }
-                }
-            } else {
-                for (int g = 0; g < s; ++g) {
-                    int i = idx[o + g];
-                    i = i < N ? i : N - 1;
-                    const float c = load_coef(coef, coef_dtype, o + g);
-#pragma unroll
-                    for (int h = 0; h < 8; ++h)
-                        if (h < hg) atomicAdd(&a[h * N + i], w[h] * c);
+value_scatter_kernel(int N, const float* __restrict__ W, int B, int H, const uint16_t* __restrict__ idx,
+                     const void* __restrict__ coef, int coef_dtype, int64_t T, int s, int vec, float* __restrict__ A) {
+    extern __shared__ __align__(16) float tab[];           // [HGP][N]: scalar atomics want the heads apart
+    const int64_t chunks_per_b = (T + CHUNK_T - 1) / CHUNK_T;
+    const int64_t total = (int64_t)B * chunks_per_b;
+    const int64_t w0 = total * blockIdx.x / gridDim.x, w1 = total * (blockIdx.x + 1) / gridDim.x;
+    for (int h0 = 0; h0 < H; h0 += HGP) {
+        const int hg = H - h0 < HGP ? H - h0 : HGP;
+        int cur_b = -1;
+        auto flush = [&]() {                               // add this CTA's table to the stream's rows of A
+            __syncthreads();
+            if (cur_b >= 0) {
+                float* dst = A + ((int64_t)cur_b * H + h0) * N;
+                for (int j = threadIdx.x; j < hg * N; j += NTS) {
+                    const float v = tab[j];
+                    if (v != 0.f) atomicAdd(&dst[j], v);
                 }
             }
+            __syncthreads();
+        };
+        for (int64_t w = w0; w < w1; ++w) {
+            const int b = (int)(w / chunks_per_b);
+            if (b != cur_b) {
+                flush();
+                for (int j = threadIdx.x; j < N * HGP; j += NTS) tab[j] = 0.f;
+                __syncthreads();
+                cur_b = b;
+            }
+            const int64_t t = (w % chunks_per_b) * CHUNK_T + threadIdx.x;
+            if (t >= T) continue;
+            float wv[HGP];
+#pragma unroll
+            for (int h = 0; h < HGP; ++h) wv[h] = h < hg ? W[((int64_t)b * H + h0 + h) * T + t] : 0.f;
+            for_each_code(idx, coef, coef_dtype, ((int64_t)b * T + t) * s, s, N, vec, [&](int i, float c) {
+#pragma unroll
+                for (int h = 0; h < HGP; ++h)
+                    if (h < hg) atomicAdd(&tab[h * N + i], wv[h] * c);
+            });
         }
-        __syncthreads();
-        float* dst = A + ((int64_t)b * H + h0) * N;
-        for (int j = threadIdx.x; j < hg * N; j += NTS)
-            if (a[j] != 0.f) atomicAdd(&dst[j], a[j]);
+        flush();
     }
 }
 
-// Query heads whose N-vectors fit in shared memory together (at most 8).
+// Query heads whose N-vectors fit in shared memory side by side: 8, 4, 2 or 1 (0 = none fits).
 int head_group(int N, int H) {
-    int hg = (200 * 1024) / (N * 4);
-    if (hg > 8) hg = 8;
-    if (hg > H) hg = H;
-    return hg;
+    int hgp = 8;
+    while (hgp > 1 && (hgp / 2 >= H || (size_t)hgp * N * 4 > 200 * 1024)) hgp /= 2;
+    return (size_t)hgp * N * 4 > 200 * 1024 ? 0 : hgp;
 }
 
-// Token ranges per code stream: enough CTAs to fill the GPU about twice, at least 1024 tokens each.
-int64_t tokens_per_cta(int B, int64_t T) {
-    int64_t splits = (2 * (int64_t)sm_count() + B - 1) / B;
-    if (splits < 1) splits = 1;
-    int64_t per = (T + splits - 1) / splits;
-    if (per < 1024) per = 1024;
-    return per;
+int stream_grid(int B, int64_t T) {
+    const int64_t total = (int64_t)B * ((T + CHUNK_T - 1) / CHUNK_T);
+    return (int)(total < (int64_t)sm_count() ? total : (int64_t)sm_count());
+}
+
+template <int HGP>
+cudaError_t run_key_scores(const AttnArgs& a, const float* P) {
+    const size_t smem = (size_t)HGP * a.N * 4;
+    cudaError_t e = cudaFuncSetAttribute(key_scores_kernel<HGP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    key_scores_kernel<HGP><<<stream_grid(a.B, a.T), NTS, smem, a.stream>>>(P, a.N, a.B, a.H, a.idx, a.coef, a.coef_dtype,
+                                                                          a.T, a.s, a.s % 8 == 0, a.out);
+    return cudaGetLastError();
+}
+
+template <int HGP>
+cudaError_t run_value_scatter(const AttnArgs& a, float* A) {
+    const size_t smem = (size_t)HGP * a.N * 4;
+    cudaError_t e = cudaFuncSetAttribute(value_scatter_kernel<HGP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    value_scatter_kernel<HGP><<<stream_grid(a.B, a.T), NTS, smem, a.stream>>>(a.N, static_cast<const float*>(a.Q), a.B, a.H,
+                                                                             a.idx, a.coef, a.coef_dtype, a.T, a.s,
+                                                                             a.s % 8 == 0, A);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -283,14 +343,8 @@ int launch_key_scores(const AttnArgs& a, float* P) {
         qd_kernel<128><<<pgrid, NT, 0, a.stream>>>(a.D, a.N, a.Q, a.q_dtype, R, a.scale, P);
     else
         qd_kernel<64><<<pgrid, NT, 0, a.stream>>>(a.D, a.N, a.Q, a.q_dtype, R, a.scale, P);
-    const size_t smem = (size_t)hg * a.N * 4;
-    const int64_t per = tokens_per_cta(a.B, a.T);
-    const dim3 grid(a.B, (unsigned)((a.T + per - 1) / per));
-    cudaError_t e = cudaFuncSetAttribute(key_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-        key_scores_kernel<<<grid, NTS, smem, a.stream>>>(P, a.N, a.H, hg, a.idx, a.coef, a.coef_dtype, a.T, a.s, a.s % 8 == 0,
-                                                         per, a.out);
-    if (e == cudaSuccess) e = cudaGetLastError();
+    cudaError_t e = hg == 8 ? run_key_scores<8>(a, P) : hg == 4 ? run_key_scores<4>(a, P)
+                    : hg == 2 ? run_key_scores<2>(a, P) : run_key_scores<1>(a, P);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "key_scores launch: %s", cudaGetErrorString(e));
     return CSR_OK;
 }
@@ -307,14 +361,8 @@ int launch_value_mix(const AttnArgs& a, float* A) {
     if (hg < 1) return fail(CSR_ERR_UNSUPPORTED, "N = %d: one head's N fp32 values do not fit in shared memory", a.N);
     cudaError_t e = cudaMemsetAsync(A, 0, attn_scratch_bytes(a.B, a.H, a.N), a.stream);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
-    const size_t smem = (size_t)hg * a.N * 4;
-    const int64_t per = tokens_per_cta(a.B, a.T);
-    const dim3 grid(a.B, (unsigned)((a.T + per - 1) / per));
-    e = cudaFuncSetAttribute(value_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-        value_scatter_kernel<<<grid, NTS, smem, a.stream>>>(a.N, static_cast<const float*>(a.Q), a.H, hg, a.idx, a.coef,
-                                                            a.coef_dtype, a.T, a.s, a.s % 8 == 0, per, A);
-    if (e == cudaSuccess) e = cudaGetLastError();
+    e = hg == 8 ? run_value_scatter<8>(a, A) : hg == 4 ? run_value_scatter<4>(a, A)
+        : hg == 2 ? run_value_scatter<2>(a, A) : run_value_scatter<1>(a, A);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "value_scatter launch: %s", cudaGetErrorString(e));
     // out = A D: row blocks of 16; with few row blocks the atoms are split over CTAs as well
     const int row_blocks = (R + OR - 1) / OR;
