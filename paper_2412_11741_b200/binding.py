@@ -33,7 +33,7 @@ CSR_MODE_BF16_FAST = 1
 
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
-    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append", "csr_dict_train_step", "csr_key_scores", "csr_value_mix",
+    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append", "csr_dict_create", "csr_dict_destroy", "csr_dict_train_step", "csr_key_scores", "csr_value_mix",
     "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
@@ -48,6 +48,7 @@ class csr_encode_params_t(ctypes.Structure):
         ("out_idx", ctypes.c_void_p), ("out_coef", ctypes.c_void_p),
         ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("ldx", ctypes.c_int64), ("ld_code", ctypes.c_int64),
+        ("dict", ctypes.c_void_p),
     ]
 
 
@@ -119,6 +120,10 @@ def lib() -> ctypes.CDLL:
         L.csr_key_scores.restype = i32
         L.csr_value_mix.argtypes = [vp, i32, i32, vp, i32, i32, vp, vp, i32, i64, i32, vp, vp]
         L.csr_value_mix.restype = i32
+        L.csr_dict_create.argtypes = [vp, i32, i32, vp, ctypes.POINTER(vp)]
+        L.csr_dict_create.restype = i32
+        L.csr_dict_destroy.argtypes = [vp]
+        L.csr_dict_destroy.restype = i32
         L.csr_dict_train_step.argtypes = [ctypes.POINTER(csr_train_params_t)]
         L.csr_dict_train_step.restype = i32
         L.csr_device_status.argtypes = [vp]
@@ -160,6 +165,20 @@ def csr_encode_workspace_bytes(mode: int, d: int, N: int) -> int:
     return n
 
 
+def csr_dict_create(D: torch.Tensor) -> int:
+    """csr_dict_create: builds the fast mode's bf16 copy of D once (on torch's current stream);
+    returns the handle to pass as `dict=` to csr_encode_ex.  Free it with csr_dict_destroy."""
+    assert D.is_cuda and D.is_contiguous() and D.dtype == torch.float32 and D.dim() == 2
+    h = ctypes.c_void_p()
+    with torch.cuda.device(D.device):
+        _check(lib().csr_dict_create(D.data_ptr(), D.shape[0], D.shape[1], _stream_ptr(D), ctypes.byref(h)))
+    return h.value
+
+
+def csr_dict_destroy(handle: int) -> None:
+    _check(lib().csr_dict_destroy(handle))
+
+
 def _encode_params(D, X, s, out_idx, out_coef, mode, stream, workspace) -> csr_encode_params_t:
     p = csr_encode_params_t()
     p.struct_size = ctypes.sizeof(csr_encode_params_t)
@@ -188,8 +207,8 @@ def _encode_params(D, X, s, out_idx, out_coef, mode, stream, workspace) -> csr_e
 
 def csr_encode_ex(D: torch.Tensor, X: torch.Tensor, s: int, *, mode: int = CSR_MODE_BF16_FAST,
                   coef_dtype: torch.dtype = torch.float16, out_idx: Optional[torch.Tensor] = None,
-                  out_coef: Optional[torch.Tensor] = None,
-                  workspace: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+                  out_coef: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                  dict: Optional[int] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """csr_encode_ex on CUDA tensors: D [N][d] fp32, X [M][d] fp32 or bf16.
     Returns (idx [M][s] uint16, coef [M][s] coef_dtype); runs on torch's current stream."""
     assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.dim() == 2 and X.stride(1) == 1
@@ -200,6 +219,8 @@ def csr_encode_ex(D: torch.Tensor, X: torch.Tensor, s: int, *, mode: int = CSR_M
     if out_coef is None:
         out_coef = torch.empty((M, s), dtype=coef_dtype, device=X.device)
     p = _encode_params(D, X, s, out_idx, out_coef, mode, _stream_ptr(X), workspace)
+    if dict is not None:
+        p.dict = dict
     with torch.cuda.device(X.device):
         _check(lib().csr_encode_ex(ctypes.byref(p)))
     return out_idx, out_coef

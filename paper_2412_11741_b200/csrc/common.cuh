@@ -44,6 +44,9 @@ int launch_encode_exact_split(const EncodeArgs& a, void* scratch);
 // 1024-byte aligned); `status` is a device word that receives kStatusTimeout.
 int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status);
 size_t encode_fast_workspace_bytes(int d, int N);
+// The two halves of launch_encode_fast: build the bf16 copy once, encode against it many times.
+int prepare_fast_dictionary(const float* D, int N, int d, void* workspace, cudaStream_t stream);
+int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint32_t* status);
 
 struct ReconstructArgs {
     const float* D;

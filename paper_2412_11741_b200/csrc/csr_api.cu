@@ -5,8 +5,18 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <new>
 
 #include "common.cuh"
+
+struct csr_dict {
+    uint32_t magic;
+    int device;
+    const void* D;
+    int N, d;
+    void* raw;      // cudaMalloc'ed block
+    void* bf16;     // 1024-byte aligned copy inside it
+};
 
 namespace csr {
 
@@ -36,6 +46,7 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kStatusBytes = 256;
+constexpr uint32_t kDictMagic = 0x43535244u;   // "CSRD"
 
 // Library-owned, grow-only device buffers of one device.
 struct DeviceBuffers {
@@ -256,6 +267,17 @@ int encode_device(const csr_encode_params_t* p) {
         return launch_encode_exact(a);
     }
 
+    if (p->dict) {
+        const csr_dict* dc = static_cast<const csr_dict*>(p->dict);
+        int dev = -1;
+        if (int rc = current_device(&dev)) return rc;
+        if (dc->magic != kDictMagic) return fail(CSR_ERR_INVALID_ARG, "dict is not a live csr_dict_t handle");
+        if (dc->device != dev || dc->D != p->D || dc->N != p->N || dc->d != p->d)
+            return fail(CSR_ERR_INVALID_ARG, "dict was created for another device, D, N or d");
+        void* wbase = nullptr;
+        if (int rc = ensure_work(0, &wbase)) return rc;           // only the status word is used
+        return launch_encode_fast_prepared(a, dc->bf16, static_cast<uint32_t*>(wbase));
+    }
     void* base = nullptr;
     if (p->workspace) {
         const int64_t need = workspace_bytes(p->mode, p->d, p->N);
@@ -335,6 +357,46 @@ int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_
     p.s = s;
     p.X_hat = X_hat;
     return csr_reconstruct_ex(&p);
+}
+
+int csr_dict_create(const void* D, int N, int d, void* stream, csr_dict_t** out) {
+    if (!out) return fail(CSR_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (int rc = check_dims(d, N, 1, 0)) return rc;
+    if (!D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
+    if (!aligned16(D)) return fail(CSR_ERR_ALIGNMENT, "D must be 16-byte aligned");
+    int dev = -1;
+    if (int rc = current_device(&dev)) return rc;
+    csr_dict* dc = new (std::nothrow) csr_dict();
+    if (!dc) return fail(CSR_ERR_CUDA, "out of host memory");
+    cudaError_t e = cudaMalloc(&dc->raw, encode_fast_workspace_bytes(d, N) + 1024);
+    if (e != cudaSuccess) {
+        delete dc;
+        return fail(CSR_ERR_CUDA, "cudaMalloc: %s", cudaGetErrorString(e));
+    }
+    dc->bf16 = align_up(dc->raw, 1024);
+    dc->device = dev;
+    dc->D = D;
+    dc->N = N;
+    dc->d = d;
+    if (int rc = prepare_fast_dictionary(static_cast<const float*>(D), N, d, dc->bf16, static_cast<cudaStream_t>(stream))) {
+        cudaFree(dc->raw);
+        delete dc;
+        return rc;
+    }
+    dc->magic = kDictMagic;
+    *out = dc;
+    return CSR_OK;
+}
+
+int csr_dict_destroy(csr_dict_t* dict) {
+    if (!dict) return CSR_OK;
+    if (dict->magic != kDictMagic) return fail(CSR_ERR_INVALID_ARG, "dict is not a live csr_dict_t handle");
+    dict->magic = 0;
+    cudaDeviceSynchronize();
+    cudaFree(dict->raw);
+    delete dict;
+    return CSR_OK;
 }
 
 int csr_encode_grouped(const csr_encode_params_t* problems, int count) {

@@ -743,27 +743,38 @@ int launch_d(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, u
 static int padded_atoms(int N) { return (N + 7) / 8 * 8; }
 size_t encode_fast_workspace_bytes(int d, int N) { return (size_t)padded_atoms(N) * (size_t)d * 2; }
 
+int prepare_fast_dictionary(const float* D, int N, int d, void* workspace, cudaStream_t stream) {
+    if ((reinterpret_cast<uintptr_t>(workspace) & 1023u) != 0)
+        return fail(CSR_ERR_ALIGNMENT, "internal: dictionary scratch not 1024-byte aligned");
+    const int64_t n_vec4 = (int64_t)N * d / 4;
+    int blocks = (int)((n_vec4 + 255) / 256);
+    if (blocks > 4 * sm_count()) blocks = 4 * sm_count();
+    dict_to_bf16_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const float4*>(D), reinterpret_cast<uint2*>(workspace),
+                                                    n_vec4);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "dict_to_bf16 launch: %s", cudaGetErrorString(e));
+    const int n_pad = padded_atoms(N);
+    if (n_pad > N) {
+        e = cudaMemsetAsync(static_cast<char*>(workspace) + (size_t)N * d * 2, 0, (size_t)(n_pad - N) * d * 2, stream);
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    }
+    return CSR_OK;
+}
+
 int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status) {
     if (a.M == 0) return CSR_OK;
+    if (int rc = prepare_fast_dictionary(a.D, a.N, a.d, workspace, a.stream)) return rc;
+    return launch_encode_fast_prepared(a, workspace, status);
+}
+
+int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint32_t* status) {
+    if (a.M == 0) return CSR_OK;
+    void* workspace = const_cast<void*>(dict_bf16);
     if ((reinterpret_cast<uintptr_t>(workspace) & 1023u) != 0)
         return fail(CSR_ERR_ALIGNMENT, "internal: dictionary scratch not 1024-byte aligned");
     EncodeTiledFn encode = get_encode_tiled();
     if (!encode) return fail(CSR_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-
-    // bf16 copy of the dictionary
-    const int64_t n_vec4 = (int64_t)a.N * a.d / 4;
-    int blocks = (int)((n_vec4 + 255) / 256);
-    if (blocks > 4 * sm_count()) blocks = 4 * sm_count();
-    dict_to_bf16_kernel<<<blocks, 256, 0, a.stream>>>(reinterpret_cast<const float4*>(a.D),
-                                                      reinterpret_cast<uint2*>(workspace), n_vec4);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "dict_to_bf16 launch: %s", cudaGetErrorString(e));
     const int n_pad = padded_atoms(a.N);
-    if (n_pad > a.N) {
-        e = cudaMemsetAsync(static_cast<char*>(workspace) + (size_t)a.N * a.d * 2, 0, (size_t)(n_pad - a.N) * a.d * 2,
-                            a.stream);
-        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
-    }
 
     // rows past the padded copy (the rest of the last 256-atom tile) are filled with zeros by TMA
     CUtensorMap tmap;

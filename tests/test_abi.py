@@ -35,7 +35,7 @@ def test_exports_match_header(lib):
 def test_version_and_struct_sizes(lib):
     from paper_2412_11741_b200 import binding
     assert binding.csr_version() == 100
-    assert ctypes.sizeof(binding.csr_encode_params_t) == 112
+    assert ctypes.sizeof(binding.csr_encode_params_t) == 120
     assert ctypes.sizeof(binding.csr_reconstruct_params_t) == 96
 
 
@@ -101,6 +101,15 @@ def test_stride_and_group_argument_errors(lib):
     assert f(0x1000, 0, 16, 128, 0x2000, 2, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_INVALID_ARG     # fp16 X
     assert f(0x1000, 0, 16, 128, 0x2004, 0, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_ALIGNMENT
     assert f(0x1000, 0, 16, 128, 0x2000, 0, 100, 0, 0x3000, 0, None) == binding.CSR_OK                  # nothing to add
+
+
+def test_dict_handle_argument_errors(lib):
+    from paper_2412_11741_b200 import binding
+    h = ctypes.c_void_p()
+    assert lib.csr_dict_create(0x1000, 1024, 96, None, ctypes.byref(h)) == binding.CSR_ERR_UNSUPPORTED
+    assert lib.csr_dict_create(0, 1024, 128, None, ctypes.byref(h)) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_dict_create(0x1000, 1024, 128, None, None) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_dict_destroy(None) == binding.CSR_OK
 
 
 def test_workspace_query(lib):

@@ -269,6 +269,29 @@ def test_fast_zero_rows_and_eight_arg_form(csr):
         csr.csr_encode_ex(D, Xd, w.s, workspace=ws[:1024])
 
 
+def test_prepared_dictionary_handle(csr):
+    """A handle encodes exactly as the plain call does, keeps its snapshot when D changes
+    afterwards, and refuses a call made for another dictionary."""
+    w = wl.llama2_layer(tokens=8, N=1000)                # N not a multiple of 8 * 128 either
+    D = torch.from_numpy(w.D).to(DEV)
+    X = torch.from_numpy(w.X).to(DEV).to(torch.bfloat16)
+    i0, c0 = csr.csr_encode_ex(D, X, w.s)
+    h = csr.csr_dict_create(D)
+    try:
+        i1, c1 = csr.csr_encode_ex(D, X, w.s, dict=h)
+        assert csr.csr_device_status() == csr.CSR_OK
+        assert np.array_equal(_np_idx(i1), _np_idx(i0)) and torch.equal(c1.cpu(), c0.cpu())
+        D.mul_(-1.0)                                     # the copy is a snapshot: same codes as before
+        i2, c2 = csr.csr_encode_ex(D, X, w.s, dict=h)
+        assert np.array_equal(_np_idx(i2), _np_idx(i0)) and torch.equal(c2.cpu(), c0.cpu())
+        i3, c3 = csr.csr_encode_ex(D, X, w.s)            # the plain call sees the negated atoms
+        assert np.array_equal(_np_idx(i3), _np_idx(i0)) and torch.equal(c3.cpu(), -c0.cpu())
+        with pytest.raises(csr.CsrError):
+            csr.csr_encode_ex(D[:512].contiguous(), X, w.s, dict=h)
+    finally:
+        csr.csr_dict_destroy(h)
+
+
 def test_fast_full_size_llama2_layer_sampled(csr):
     """Config 2 at full size in the launch configuration the benchmark times; the oracle
     checks a stratified sample of the outputs."""
