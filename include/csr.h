@@ -48,7 +48,7 @@ extern "C" {
 #define CSR_ERR_TIMEOUT (-5)
 #define CSR_ERR_WORKSPACE (-6)
 
-/* element types of X, X_hat and coef */
+/* element types of X and X_hat (any of the three) and of coef (F32 or F16) */
 #define CSR_DTYPE_F32 0
 #define CSR_DTYPE_BF16 1
 #define CSR_DTYPE_F16 2
@@ -83,7 +83,7 @@ typedef struct csr_encode_params {
     uint32_t struct_size;   /* sizeof(csr_encode_params_t), for versioning */
     int32_t mode;           /* CSR_MODE_* */
     const void* D;          /* [N][d] fp32 */
-    const void* X;          /* [M][d], x_dtype (F32 or BF16) */
+    const void* X;          /* [M][d], x_dtype (F32, BF16 or F16; the fast mode rounds to bf16) */
     int32_t x_dtype;
     int32_t coef_dtype;     /* F16 (the paper's stored form) or F32 */
     int64_t M;
@@ -108,7 +108,7 @@ typedef struct csr_reconstruct_params {
     const uint16_t* idx;    /* [M][s] */
     const void* coef;       /* [M][s], coef_dtype */
     int32_t coef_dtype;     /* F16 or F32 */
-    int32_t out_dtype;      /* BF16 or F32 */
+    int32_t out_dtype;      /* BF16, F16 or F32 */
     int64_t M;
     int32_t d, N, s;
     int32_t reserved1;
@@ -194,7 +194,7 @@ int csr_reconstruct_grouped(const csr_reconstruct_params_t* problems, int count)
  * non-zero residual).  Which rows are sampled is the caller's choice: `rows` is a DEVICE
  * array of n_rows row numbers in [0, M).  D is the caller's [N_cap][d] fp32 device array of
  * which rows [0, N_cur) are in use; N_cur + n_rows <= N_cap is required.  X is [M][d] with
- * x_dtype F32 or BF16 and row stride ldx (0 = d).  Asynchronous on `stream`.
+ * x_dtype F32, BF16 or F16 and row stride ldx (0 = d).  Asynchronous on `stream`.
  */
 int csr_dict_append(void* D, int N_cur, int N_cap, int d, const void* X, int x_dtype, int64_t M, int64_t ldx,
                     const int64_t* rows, int n_rows, void* stream);
@@ -208,7 +208,7 @@ int csr_dict_append(void* D, int N_cur, int N_cap, int d, const void* X, int x_d
  *
  * csr_key_scores:  scores[b][h][t] = scale * Q[b][h][:] . X~_K[b][t][:]
  *                                  = sum_g coef[b][t][g] * (scale * D[idx[b][t][g]][:] . Q[b][h][:]),
- *     terms added in stored order g = 0 .. s-1 in fp32.  Q is [B][H][d], q_dtype F32 or BF16;
+ *     terms added in stored order g = 0 .. s-1 in fp32.  Q is [B][H][d], q_dtype F32, BF16 or F16;
  *     scores is [B][H][T] fp32 (before softmax).
  * csr_value_mix:   out[b][h][:] = sum_t W[b][h][t] * X~_V[b][t][:],
  *     W is [B][H][T] fp32 (attention weights), out is [B][H][d] fp32.  Accumulated with
@@ -247,7 +247,7 @@ typedef struct csr_train_params {
     uint32_t struct_size;   /* sizeof(csr_train_params_t) */
     int32_t mode;           /* CSR_MODE_* of the matching-pursuit forward pass */
     void* D;                /* [N][d] fp32, updated in place */
-    const void* X;          /* [M][d], x_dtype (F32 or BF16), dense */
+    const void* X;          /* [M][d], x_dtype (F32, BF16 or F16), dense */
     int32_t x_dtype;
     int32_t d, N, s;
     int64_t M;

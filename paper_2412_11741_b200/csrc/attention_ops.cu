@@ -29,10 +29,7 @@ __device__ __forceinline__ float load_coef(const void* coef, int coef_dtype, int
     return coef_dtype == CSR_DTYPE_F16 ? __half2float(reinterpret_cast<const __half*>(coef)[off])
                                        : reinterpret_cast<const float*>(coef)[off];
 }
-__device__ __forceinline__ float load_q(const void* Q, int q_dtype, int64_t off) {
-    return q_dtype == CSR_DTYPE_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(Q)[off])
-                                     : reinterpret_cast<const float*>(Q)[off];
-}
+__device__ __forceinline__ float load_q(const void* Q, int q_dtype, int64_t off) { return load_elem(Q, q_dtype, off); }
 
 // ---- P[r][n] = scale * Q[r][:] . D[n][:]  (r = b*H + h) -----------------------------------
 // CTA = 64 atoms x 64 rows; thread = 4 rows x 4 atoms; channels staged 32 at a time,

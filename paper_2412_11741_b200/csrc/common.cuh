@@ -108,6 +108,15 @@ struct TrainArgs {
 };
 int launch_dict_train(const TrainArgs& a);
 
+// Element `off` of an array of dtype F32, BF16 or F16, widened exactly to fp32.
+__device__ __forceinline__ float load_elem(const void* p, int dtype, int64_t off) {
+    if (dtype == CSR_DTYPE_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[off]);
+    if (dtype == CSR_DTYPE_F16) return __half2float(reinterpret_cast<const __half*>(p)[off]);
+    return reinterpret_cast<const float*>(p)[off];
+}
+inline bool valid_x_dtype(int t) { return t == CSR_DTYPE_F32 || t == CSR_DTYPE_BF16 || t == CSR_DTYPE_F16; }
+inline size_t dtype_size(int t) { return t == CSR_DTYPE_F32 ? 4 : 2; }
+
 int sm_count();
 
 }  // namespace csr

@@ -115,8 +115,7 @@ int check_encode(const csr_encode_params_t* p, bool host_io) {
     if (p->mode != CSR_MODE_FP32_EXACT && p->mode != CSR_MODE_BF16_FAST)
         return fail(CSR_ERR_INVALID_ARG, "unknown mode %d", p->mode);
     if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
-    if (p->x_dtype != CSR_DTYPE_F32 && p->x_dtype != CSR_DTYPE_BF16)
-        return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32 or BF16");
+    if (!valid_x_dtype(p->x_dtype)) return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32, BF16 or F16");
     if (p->coef_dtype != CSR_DTYPE_F32 && p->coef_dtype != CSR_DTYPE_F16)
         return fail(CSR_ERR_INVALID_ARG, "coef_dtype must be F32 or F16");
     if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
@@ -128,7 +127,7 @@ int check_encode(const csr_encode_params_t* p, bool host_io) {
     if (host_io && (p->ldx || p->ld_code)) return fail(CSR_ERR_UNSUPPORTED, "the host entry points take dense arrays");
     if (!aligned16(p->D)) return fail(CSR_ERR_ALIGNMENT, "D must be 16-byte aligned");
     if (!host_io) {
-        const size_t xe = p->x_dtype == CSR_DTYPE_BF16 ? 2 : 4, ce = p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4;
+        const size_t xe = dtype_size(p->x_dtype), ce = p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4;
         if (!aligned16(p->X) || (p->ldx && (p->ldx * xe) % 16 != 0))
             return fail(CSR_ERR_ALIGNMENT, "every row of X must start on a 16-byte boundary");
         if (p->ld_code == 0) {
@@ -193,8 +192,7 @@ int check_reconstruct(const csr_reconstruct_params_t* p, bool host_io) {
     if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
     if (p->coef_dtype != CSR_DTYPE_F32 && p->coef_dtype != CSR_DTYPE_F16)
         return fail(CSR_ERR_INVALID_ARG, "coef_dtype must be F32 or F16");
-    if (p->out_dtype != CSR_DTYPE_F32 && p->out_dtype != CSR_DTYPE_BF16)
-        return fail(CSR_ERR_INVALID_ARG, "out_dtype must be F32 or BF16");
+    if (!valid_x_dtype(p->out_dtype)) return fail(CSR_ERR_INVALID_ARG, "out_dtype must be F32, BF16 or F16");
     if (!p->D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
     if (p->M > 0 && (!p->idx || !p->coef || !p->X_hat)) return fail(CSR_ERR_INVALID_ARG, "idx, coef or X_hat is NULL");
     if (p->ld_code < 0 || p->ld_xhat < 0 || (p->ld_code && p->ld_code < p->s) || (p->ld_xhat && p->ld_xhat < p->d))
@@ -203,7 +201,7 @@ int check_reconstruct(const csr_reconstruct_params_t* p, bool host_io) {
     if (host_io && (p->ld_code || p->ld_xhat)) return fail(CSR_ERR_UNSUPPORTED, "the host entry points take dense arrays");
     if (!aligned16(p->D)) return fail(CSR_ERR_ALIGNMENT, "D must be 16-byte aligned");
     if (!host_io) {
-        const size_t xe = p->out_dtype == CSR_DTYPE_BF16 ? 2 : 4, ce = p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4;
+        const size_t xe = dtype_size(p->out_dtype), ce = p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4;
         if (!aligned16(p->X_hat) || (p->ld_xhat && (p->ld_xhat * xe) % 16 != 0))
             return fail(CSR_ERR_ALIGNMENT, "every row of X_hat must start on a 16-byte boundary");
         if (p->ld_code == 0) {
@@ -422,12 +420,12 @@ int csr_dict_append(void* D, int N_cur, int N_cap, int d, const void* X, int x_d
     if (d != 64 && d != 128) return fail(CSR_ERR_UNSUPPORTED, "d = %d: only 64 and 128 are supported", d);
     if (N_cap < 1 || N_cap > 65536 || N_cur < 0 || n_rows < 0 || (int64_t)N_cur + n_rows > N_cap)
         return fail(CSR_ERR_INVALID_ARG, "N_cur = %d, n_rows = %d do not fit N_cap = %d (<= 65536)", N_cur, n_rows, N_cap);
-    if (x_dtype != CSR_DTYPE_F32 && x_dtype != CSR_DTYPE_BF16) return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32 or BF16");
+    if (!valid_x_dtype(x_dtype)) return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32, BF16 or F16");
     if (M < 0 || ldx < 0 || (ldx && ldx < d)) return fail(CSR_ERR_INVALID_ARG, "M < 0 or ldx not 0 or >= d");
     if (n_rows == 0) return CSR_OK;
     if (!D || !X || !rows) return fail(CSR_ERR_INVALID_ARG, "D, X or rows is NULL");
     if (M == 0) return fail(CSR_ERR_INVALID_ARG, "rows given but X is empty");
-    const size_t xe = x_dtype == CSR_DTYPE_BF16 ? 2 : 4;
+    const size_t xe = dtype_size(x_dtype);
     if (!aligned16(D) || !aligned16(X) || (ldx && (ldx * xe) % 16 != 0) || (reinterpret_cast<uintptr_t>(rows) % 8))
         return fail(CSR_ERR_ALIGNMENT, "D and every row of X must be 16-byte aligned, rows 8-byte aligned");
     return launch_dict_append(static_cast<float*>(D) + (size_t)N_cur * d, d, X, x_dtype, M, ldx ? ldx : d, rows, n_rows,
@@ -454,7 +452,7 @@ static int check_attn(const void* D, int N, int d, const void* Q, int B, int H, 
 int csr_key_scores(const void* D, int N, int d, const void* Q, int q_dtype, int B, int H, const uint16_t* idx,
                    const void* coef, int coef_dtype, int64_t T, int s, float scale, float* scores, void* stream) {
     if (int rc = check_attn(D, N, d, Q, B, H, idx, coef, coef_dtype, T, s, scores)) return rc;
-    if (q_dtype != CSR_DTYPE_F32 && q_dtype != CSR_DTYPE_BF16) return fail(CSR_ERR_INVALID_ARG, "q_dtype must be F32 or BF16");
+    if (!valid_x_dtype(q_dtype)) return fail(CSR_ERR_INVALID_ARG, "q_dtype must be F32, BF16 or F16");
     AttnArgs a{static_cast<const float*>(D), N, d, Q, q_dtype, B, H, idx, coef, coef_dtype, T, s, scale, scores,
                static_cast<cudaStream_t>(stream)};
     if (B == 0 || T == 0) return CSR_OK;
@@ -482,8 +480,7 @@ int csr_dict_train_step(const csr_train_params_t* p) {
     if (p->mode != CSR_MODE_FP32_EXACT && p->mode != CSR_MODE_BF16_FAST)
         return fail(CSR_ERR_INVALID_ARG, "unknown mode %d", p->mode);
     if (int rc = check_dims(p->d, p->N, p->s, p->M)) return rc;
-    if (p->x_dtype != CSR_DTYPE_F32 && p->x_dtype != CSR_DTYPE_BF16)
-        return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32 or BF16");
+    if (!valid_x_dtype(p->x_dtype)) return fail(CSR_ERR_INVALID_ARG, "x_dtype must be F32, BF16 or F16");
     if (!p->D || !p->losses || (p->M > 0 && !p->X)) return fail(CSR_ERR_INVALID_ARG, "D, losses or X is NULL");
     if (!aligned16(p->D) || !aligned16(p->X) || (reinterpret_cast<uintptr_t>(p->losses) % 8))
         return fail(CSR_ERR_ALIGNMENT, "D and X must be 16-byte aligned, losses 8-byte aligned");
@@ -543,7 +540,7 @@ int csr_encode_host(const csr_encode_params_t* p) {
     if (p->M == 0) return CSR_OK;
     int dev;
     if (int rc = current_device(&dev)) return rc;
-    const size_t xb = (p->x_dtype == CSR_DTYPE_BF16 ? 2 : 4) * (size_t)p->d;
+    const size_t xb = dtype_size(p->x_dtype) * (size_t)p->d;
     const size_t cb = (p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4) * (size_t)p->s;
     const size_t ib = 2 * (size_t)p->s;
     const int64_t chunk = host_chunk_rows(p->M);
@@ -593,7 +590,7 @@ int csr_reconstruct_host(const csr_reconstruct_params_t* p) {
     if (p->M == 0) return CSR_OK;
     int dev;
     if (int rc = current_device(&dev)) return rc;
-    const size_t xb = (p->out_dtype == CSR_DTYPE_BF16 ? 2 : 4) * (size_t)p->d;
+    const size_t xb = dtype_size(p->out_dtype) * (size_t)p->d;
     const size_t cb = (p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4) * (size_t)p->s;
     const size_t ib = 2 * (size_t)p->s;
     const int64_t chunk = host_chunk_rows(p->M);

@@ -24,8 +24,7 @@ __global__ void dict_append_kernel(float* __restrict__ D_new, const void* __rest
 #pragma unroll
     for (int k = 0; k < PER; ++k) {
         const int64_t off = r * ldx + lane * PER + k;
-        v[k] = (x_dtype == CSR_DTYPE_BF16) ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(X)[off])
-                                           : reinterpret_cast<const float*>(X)[off];
+        v[k] = load_elem(X, x_dtype, off);
         ss = fmaf(v[k], v[k], ss);
     }
     for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);

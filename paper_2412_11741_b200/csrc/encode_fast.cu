@@ -550,6 +550,22 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     if (valid) v = __ldg(src + c);
                     *reinterpret_cast<uint4*>(Atile + swz_off(r, c)) = v;
                 }
+            } else if (x_dtype == CSR_DTYPE_F16) {
+                const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(X) + m * ldx);
+#pragma unroll
+                for (int c = 0; c < CHUNKS; ++c) {
+                    uint4 h = make_uint4(0u, 0u, 0u, 0u);
+                    if (valid) h = __ldg(src + c);
+                    const __half2* hp = reinterpret_cast<const __half2*>(&h);
+                    const float2 f0 = __half22float2(hp[0]), f1 = __half22float2(hp[1]);
+                    const float2 f2 = __half22float2(hp[2]), f3 = __half22float2(hp[3]);
+                    uint4 v;
+                    v.x = pack_bf16(f0.x, f0.y);
+                    v.y = pack_bf16(f1.x, f1.y);
+                    v.z = pack_bf16(f2.x, f2.y);
+                    v.w = pack_bf16(f3.x, f3.y);
+                    *reinterpret_cast<uint4*>(Atile + swz_off(r, c)) = v;
+                }
             } else {
                 const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X) + m * ldx);
 #pragma unroll

@@ -18,10 +18,7 @@ constexpr int BS_LD = BN + 4;
 // the rounding of R itself; two candidates can therefore swap when closer than twice that.
 constexpr float kBandRel = 1.6e-5f;
 
-__device__ __forceinline__ float load_x(const void* X, int x_dtype, int64_t off) {
-    if (x_dtype == CSR_DTYPE_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(X)[off]);
-    return reinterpret_cast<const float*>(X)[off];
-}
+__device__ __forceinline__ float load_x(const void* X, int x_dtype, int64_t off) { return load_elem(X, x_dtype, off); }
 
 struct Top2 {
     float best, second;

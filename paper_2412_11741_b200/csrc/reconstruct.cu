@@ -44,6 +44,12 @@ __device__ __forceinline__ void store_out(void* out, int out_dtype, int64_t off,
         u.x = *reinterpret_cast<uint32_t*>(&lo);
         u.y = *reinterpret_cast<uint32_t*>(&hi);
         reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + off)[lane] = u;
+    } else if (out_dtype == CSR_DTYPE_F16) {
+        __half2 lo = __floats2half2_rn(a.x, a.y), hi = __floats2half2_rn(a.z, a.w);
+        uint2 u;
+        u.x = *reinterpret_cast<uint32_t*>(&lo);
+        u.y = *reinterpret_cast<uint32_t*>(&hi);
+        reinterpret_cast<uint2*>(reinterpret_cast<__half*>(out) + off)[lane] = u;
     } else {
         reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + off)[lane] = a;
     }
@@ -52,6 +58,9 @@ __device__ __forceinline__ void store_out(void* out, int out_dtype, int64_t off,
     if (out_dtype == CSR_DTYPE_BF16) {
         __nv_bfloat162 v = __floats2bfloat162_rn(a.x, a.y);
         reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(out) + off)[lane] = *reinterpret_cast<uint32_t*>(&v);
+    } else if (out_dtype == CSR_DTYPE_F16) {
+        __half2 v = __floats2half2_rn(a.x, a.y);
+        reinterpret_cast<uint32_t*>(reinterpret_cast<__half*>(out) + off)[lane] = *reinterpret_cast<uint32_t*>(&v);
     } else {
         reinterpret_cast<float2*>(reinterpret_cast<float*>(out) + off)[lane] = a;
     }

@@ -21,10 +21,7 @@
 namespace csr {
 namespace {
 
-__device__ __forceinline__ float load_x(const void* X, int x_dtype, int64_t off) {
-    if (x_dtype == CSR_DTYPE_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(X)[off]);
-    return reinterpret_cast<const float*>(X)[off];
-}
+__device__ __forceinline__ float load_x(const void* X, int x_dtype, int64_t off) { return load_elem(X, x_dtype, off); }
 
 template <int D_>
 __global__ void __launch_bounds__(256)

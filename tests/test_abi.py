@@ -54,7 +54,7 @@ def _params(binding, **kw):
 @pytest.mark.parametrize("kw,code", [
     (dict(d=96), -2), (dict(N=0), -1), (dict(N=70000), -1), (dict(s=0), -1), (dict(s=65), -1), (dict(M=-1), -1),
     (dict(D=0), -1), (dict(X=0), -1), (dict(out_idx=0), -1), (dict(D=0x1008), -3),
-    (dict(X=0x2004), -3), (dict(mode=7), -1), (dict(x_dtype=2), -1), (dict(coef_dtype=1), -1),
+    (dict(X=0x2004), -3), (dict(mode=7), -1), (dict(x_dtype=3), -1), (dict(coef_dtype=1), -1),
     (dict(struct_size=8), -1), (dict(workspace=0x5008), -3),
 ])
 def test_encode_argument_errors(lib, kw, code):
@@ -98,7 +98,7 @@ def test_stride_and_group_argument_errors(lib):
     f = lib.csr_dict_append
     assert f(0x1000, 10, 16, 128, 0x2000, 0, 100, 0, 0x3000, 7, None) == binding.CSR_ERR_INVALID_ARG    # 10 + 7 > 16
     assert f(0x1000, 0, 16, 96, 0x2000, 0, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_UNSUPPORTED
-    assert f(0x1000, 0, 16, 128, 0x2000, 2, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_INVALID_ARG     # fp16 X
+    assert f(0x1000, 0, 16, 128, 0x2000, 7, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_INVALID_ARG     # unknown dtype
     assert f(0x1000, 0, 16, 128, 0x2004, 0, 100, 0, 0x3000, 4, None) == binding.CSR_ERR_ALIGNMENT
     assert f(0x1000, 0, 16, 128, 0x2000, 0, 100, 0, 0x3000, 0, None) == binding.CSR_OK                  # nothing to add
 

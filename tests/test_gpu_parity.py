@@ -247,6 +247,28 @@ def test_fast_fp32_input_and_odd_s(csr):
         assert np.array_equal(coef16, coef.astype(np.float16).astype(np.float32))
 
 
+def test_fp16_inputs_and_outputs(csr):
+    """fp16 is the paper's model precision: X may be fp16 (read exactly by the exact mode,
+    rounded to bf16 by the fast mode) and X_hat may be written as fp16."""
+    rng = np.random.default_rng(16)
+    D = wl.normalise_rows(rng.standard_normal((1024, 128)).astype(np.float32))
+    X = (rng.standard_normal((900, 128)) * 3).astype(np.float16).astype(np.float32)
+    Dd = torch.from_numpy(D).to(DEV)
+    Xh = torch.from_numpy(X).to(DEV).to(torch.float16)
+    s = 6
+    idx, coef = csr.csr_encode_ex(Dd, Xh, s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
+    rep = parity.compare_exact(D, X, s, _np_idx(idx), coef.cpu().numpy())
+    assert rep.ok, rep.detail
+    idx, coef = csr.csr_encode_ex(Dd, Xh, s, coef_dtype=torch.float32)
+    i2, c2 = csr.csr_encode_ex(Dd, Xh.to(torch.bfloat16), s, coef_dtype=torch.float32)   # = rounding to bf16 first
+    assert np.array_equal(_np_idx(idx), _np_idx(i2)) and torch.equal(coef, c2)
+    rep = parity.compare_fast(D, X, s, _np_idx(idx), coef.cpu().numpy())
+    assert rep.ok, rep.detail
+    x32 = csr.csr_reconstruct_ex(Dd, idx, coef, out_dtype=torch.float32)
+    x16 = csr.csr_reconstruct_ex(Dd, idx, coef, out_dtype=torch.float16)
+    assert torch.equal(x16, x32.to(torch.float16))
+
+
 def test_fast_zero_rows_and_eight_arg_form(csr):
     w = wl.llama2_layer(tokens=8, N=1024)
     X = w.X.copy()
