@@ -150,6 +150,15 @@ int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_
 int csr_reconstruct_ex(const csr_reconstruct_params_t* p);
 
 /*
+ * Packs fp32 coefficients into the stored form of "Analysis for CSR" (fp16, round to
+ * nearest even): for codes that were produced with coef_dtype F32, e.g. by the exact mode
+ * for verification, and are now to be kept.  The indices are stored as produced.  n values,
+ * dense; both device pointers 16-byte aligned; asynchronous on `stream`.  A pure streaming
+ * kernel: 4 bytes read and 2 written per value.
+ */
+int csr_pack_coefficients(const float* coef32, int64_t n, void* coef16, void* stream);
+
+/*
  * Prepared dictionary.  The fast mode works on a bf16 copy of D which the encode calls
  * otherwise rebuild in scratch memory on every call (one extra launch of a few
  * microseconds: measured 83 -> 80 us on a 4160-row call, nothing on large ones).  A

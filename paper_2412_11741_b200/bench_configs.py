@@ -1,6 +1,6 @@
 """Throughput and reconstruction error of the codec on every synthetic configuration.
 
-  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5,decode,attention,train] [--reps 30]
+  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5,decode,attention,train,pack] [--reps 30]
 
 One JSON line per case: vectors/s and TFLOP/s of the fast encoder (median of the last two
 thirds of `reps` back-to-back launches, i.e. after the clocks have settled under the power
@@ -142,6 +142,16 @@ def run_train_case(reps):
             "rows_per_s": w.M / (t * 1e-3), "L_MSE": l[0], "L_div": l[1]}
 
 
+def run_pack_case(reps):
+    """The stored-form writer alone: 2^28 fp32 coefficients -> fp16 (1 GiB in, 0.5 GiB out)."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    n = 1 << 28
+    c32 = torch.randn(n, device=dev)
+    c16 = torch.empty(n, dtype=torch.float16, device=dev)
+    t = _time(lambda: csr.csr_pack_coefficients(c32, c16), reps)
+    return {"case": "pack_coefficients", "n": n, "ms": round(t, 4), "hbm_gbs": 6.0 * n / (t * 1e-3) / 1e9}
+
+
 def cases(names):
     for n in names:
         if n == "c1":
@@ -163,14 +173,14 @@ def cases(names):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--configs", default="c1,c2,c3,c4,c5,decode,attention,train")
+    ap.add_argument("--configs", default="c1,c2,c3,c4,c5,decode,attention,train,pack")
     ap.add_argument("--reps", type=int, default=30)
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device (there is no CPU fallback)")
     build.build()
     names = args.configs.split(",")
-    for w in cases([n for n in names if n not in ("decode", "attention", "train")]):
+    for w in cases([n for n in names if n not in ("decode", "attention", "train", "pack")]):
         print(json.dumps(run_case(w, args.reps)), flush=True)
     if "decode" in names:
         for seqs, kv_heads in ((1, 8), (8, 8), (64, 8)):
@@ -179,6 +189,8 @@ def main():
         print(json.dumps(run_attention_case(args.reps)), flush=True)
     if "train" in names:
         print(json.dumps(run_train_case(args.reps)), flush=True)
+    if "pack" in names:
+        print(json.dumps(run_pack_case(args.reps)), flush=True)
 
 
 if __name__ == "__main__":

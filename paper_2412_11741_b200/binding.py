@@ -33,7 +33,7 @@ CSR_MODE_BF16_FAST = 1
 
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
-    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append", "csr_dict_create", "csr_dict_destroy", "csr_dict_train_step", "csr_key_scores", "csr_value_mix",
+    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append", "csr_dict_create", "csr_dict_destroy", "csr_dict_train_step", "csr_key_scores", "csr_pack_coefficients", "csr_value_mix",
     "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
@@ -120,6 +120,8 @@ def lib() -> ctypes.CDLL:
         L.csr_key_scores.restype = i32
         L.csr_value_mix.argtypes = [vp, i32, i32, vp, i32, i32, vp, vp, i32, i64, i32, vp, vp]
         L.csr_value_mix.restype = i32
+        L.csr_pack_coefficients.argtypes = [vp, i64, vp, vp]
+        L.csr_pack_coefficients.restype = i32
         L.csr_dict_create.argtypes = [vp, i32, i32, vp, ctypes.POINTER(vp)]
         L.csr_dict_create.restype = i32
         L.csr_dict_destroy.argtypes = [vp]
@@ -163,6 +165,17 @@ def csr_encode_workspace_bytes(mode: int, d: int, N: int) -> int:
     if n < 0:
         raise CsrError(n, csr_last_error_string())
     return n
+
+
+def csr_pack_coefficients(coef32: torch.Tensor, coef16: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """csr_pack_coefficients: fp32 coefficients -> the stored fp16 form (round to nearest even)."""
+    assert coef32.is_cuda and coef32.is_contiguous() and coef32.dtype == torch.float32
+    if coef16 is None:
+        coef16 = torch.empty(coef32.shape, dtype=torch.float16, device=coef32.device)
+    assert coef16.is_contiguous() and coef16.dtype == torch.float16 and coef16.numel() == coef32.numel()
+    with torch.cuda.device(coef32.device):
+        _check(lib().csr_pack_coefficients(coef32.data_ptr(), coef32.numel(), coef16.data_ptr(), _stream_ptr(coef32)))
+    return coef16
 
 
 def csr_dict_create(D: torch.Tensor) -> int:

@@ -117,6 +117,9 @@ __device__ __forceinline__ float load_elem(const void* p, int dtype, int64_t off
 inline bool valid_x_dtype(int t) { return t == CSR_DTYPE_F32 || t == CSR_DTYPE_BF16 || t == CSR_DTYPE_F16; }
 inline size_t dtype_size(int t) { return t == CSR_DTYPE_F32 ? 4 : 2; }
 
+// fp32 coefficients -> stored fp16 form (round to nearest even), n values.
+int launch_pack_coef(const float* coef32, int64_t n, void* coef16, cudaStream_t stream);
+
 int sm_count();
 
 }  // namespace csr

@@ -357,6 +357,13 @@ int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_
     return csr_reconstruct_ex(&p);
 }
 
+int csr_pack_coefficients(const float* coef32, int64_t n, void* coef16, void* stream) {
+    if (n < 0) return fail(CSR_ERR_INVALID_ARG, "n is negative");
+    if (n > 0 && (!coef32 || !coef16)) return fail(CSR_ERR_INVALID_ARG, "coef32 or coef16 is NULL");
+    if (!aligned16(coef32) || !aligned16(coef16)) return fail(CSR_ERR_ALIGNMENT, "coef32 and coef16 must be 16-byte aligned");
+    return launch_pack_coef(coef32, n, coef16, static_cast<cudaStream_t>(stream));
+}
+
 int csr_dict_create(const void* D, int N, int d, void* stream, csr_dict_t** out) {
     if (!out) return fail(CSR_ERR_INVALID_ARG, "out is NULL");
     *out = nullptr;

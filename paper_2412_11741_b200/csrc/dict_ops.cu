@@ -33,7 +33,41 @@ __global__ void dict_append_kernel(float* __restrict__ D_new, const void* __rest
     for (int k = 0; k < PER; ++k) D_new[(int64_t)i * D_ + lane * PER + k] = v[k] * inv;
 }
 
+// Stored form of the coefficients ("Analysis for CSR": fp16 beside the 16-bit index): fp32 ->
+// fp16, round to nearest even, eight values per thread (two 16-byte loads, one 16-byte store).
+__global__ void pack_coef_kernel(const float4* __restrict__ src, uint4* __restrict__ dst, int64_t n8, const float* tail_src,
+                                 __half* tail_dst, int tail) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
+        const float4 a = src[2 * i], b = src[2 * i + 1];
+        __half2 h0 = __floats2half2_rn(a.x, a.y), h1 = __floats2half2_rn(a.z, a.w);
+        __half2 h2 = __floats2half2_rn(b.x, b.y), h3 = __floats2half2_rn(b.z, b.w);
+        uint4 u;
+        u.x = *reinterpret_cast<uint32_t*>(&h0);
+        u.y = *reinterpret_cast<uint32_t*>(&h1);
+        u.z = *reinterpret_cast<uint32_t*>(&h2);
+        u.w = *reinterpret_cast<uint32_t*>(&h3);
+        dst[i] = u;
+    }
+    if (blockIdx.x == 0 && (int)threadIdx.x < tail) tail_dst[threadIdx.x] = __float2half_rn(tail_src[threadIdx.x]);
+}
+
 }  // namespace
+
+int launch_pack_coef(const float* coef32, int64_t n, void* coef16, cudaStream_t stream) {
+    if (n == 0) return CSR_OK;
+    const int64_t n8 = n / 8;
+    const int tail = (int)(n - 8 * n8);
+    int64_t blocks = (n8 + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    pack_coef_kernel<<<(int)blocks, 256, 0, stream>>>(reinterpret_cast<const float4*>(coef32), reinterpret_cast<uint4*>(coef16),
+                                                     n8, coef32 + 8 * n8, reinterpret_cast<__half*>(coef16) + 8 * n8, tail);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "pack_coef launch: %s", cudaGetErrorString(e));
+    return CSR_OK;
+}
 
 int launch_dict_append(float* D_new, int d, const void* X, int x_dtype, int64_t M, int64_t ldx, const int64_t* rows,
                        int n_rows, cudaStream_t stream) {

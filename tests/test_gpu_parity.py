@@ -247,6 +247,17 @@ def test_fast_fp32_input_and_odd_s(csr):
         assert np.array_equal(coef16, coef.astype(np.float16).astype(np.float32))
 
 
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 1000003])
+def test_pack_coefficients_is_round_to_nearest_even(csr, n):
+    rng = np.random.default_rng(n)
+    c = (rng.standard_normal(n) * np.exp(rng.uniform(-12, 8, n))).astype(np.float32)
+    if n > 5:
+        c[:5] = [0.0, -0.0, 65504.0, 1e-8, -70000.0]      # signed zero, largest, subnormal underflow, overflow
+    _, want = orc.pack_codes(np.zeros(n, np.int32), c.astype(np.float64))
+    got = csr.csr_pack_coefficients(torch.from_numpy(c).to(DEV)).cpu().numpy()
+    assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
+
+
 def test_fp16_inputs_and_outputs(csr):
     """fp16 is the paper's model precision: X may be fp16 (read exactly by the exact mode,
     rounded to bf16 by the fast mode) and X_hat may be written as fp16."""
