@@ -497,3 +497,49 @@ def test_host_entry_point(csr):
     xh32 = torch.empty((w.M, w.d), dtype=torch.float32)          # pageable memory and fp32 output work too
     csr.csr_reconstruct_host(D, oi, oc, xh32)
     assert torch.equal(xh32, csr.csr_reconstruct_ex(D, idx, coef, out_dtype=torch.float32).cpu())
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_both_modes(csr, seed):
+    """Seeded random (M, N, d, s, input type) combinations, ragged in every dimension, through
+    both encoders and the de-sparse kernel against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    d = int(rng.choice([64, 128]))
+    N = int(rng.choice([1, 2, 17, 100, 255, 256, 257, 600, 1023, 3000, 5000]))
+    M = int(rng.choice([1, 3, 100, 255, 257, 700, 1500, 5000]))
+    s = int(rng.integers(1, 20))
+    kind = str(rng.choice(["f32", "bf16", "f16"]))
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    if N > 2 and seed % 3 == 0:
+        D[N // 2] = D[0]                                  # a duplicated atom
+    X = (rng.standard_normal((M, d)) * rng.choice([0.01, 1.0, 30.0])).astype(np.float32)
+    if kind == "bf16":
+        X = wl.round_to_bf16(X)
+    elif kind == "f16":
+        X = X.astype(np.float16).astype(np.float32)
+    if M > 2:
+        X[M // 2] = 0.0
+    Dd = torch.from_numpy(D).to(DEV)
+    Xd = torch.from_numpy(X).to(DEV).to({"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[kind])
+    res = orc.mp_encode(D, X, s)
+    idx, coef = csr.csr_encode_ex(Dd, Xd, s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
+    rep = parity.compare_exact(D, X, s, _np_idx(idx), coef.cpu().numpy(), res)
+    assert rep.ok, (d, N, M, s, kind, rep.detail)
+    xh = csr.csr_reconstruct_ex(Dd, idx, coef, out_dtype=torch.float32).cpu().numpy()
+    ref = orc.reconstruct(D, _np_idx(idx).astype(np.int32), coef.cpu().numpy().astype(np.float64))
+    scale = np.abs(coef.cpu().numpy()).sum(1, keepdims=True) + 1e-30
+    assert np.all(np.abs(xh - ref) <= 2e-6 * scale)
+    idx, coef = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float32)
+    assert csr.csr_device_status() == csr.CSR_OK
+    gi, gc = _np_idx(idx), coef.cpu().numpy()
+    assert int(gi.max()) < N
+    if M > 2:
+        assert gi[M // 2].tolist() == [0] * s and np.all(gc[M // 2] == 0)
+    if N >= 100 and M >= 100:
+        Xb = wl.round_to_bf16(X)                          # what the fast mode encodes
+        rep = parity.compare_fast(D, Xb, s, gi, gc, max_gap=2.0 ** -3)
+        assert rep.ok, (d, N, M, s, kind, rep.detail)
+    else:                                                 # tiny problems: the codes must at least describe x
+        e_gpu = orc.relative_error(X, orc.reconstruct(D, gi.astype(np.int32), gc.astype(np.float64)))
+        e_or = res.resnorm[:, -1] / np.maximum(np.linalg.norm(X.astype(np.float64), axis=1), 1e-300)
+        assert np.all(e_gpu <= 1.3 * e_or + 2.0 ** -6), (d, N, M, s, kind)
