@@ -3,7 +3,8 @@
 Every input vector is encoded independently and the dictionary is a few MB, so the path
 shards by rows with no exchange step: each rank owns a contiguous block of rows, keeps
 its own copy of the dictionary and writes its own block of codes.  The only
-communication is the bookkeeping below (who owns which rows; the job-wide rate).
+communication is the bookkeeping below (who owns which rows; the job-wide rate) and one
+broadcast when a dictionary is installed or replaced.
 """
 from __future__ import annotations
 
@@ -37,3 +38,12 @@ def job_rate(units_local: int, seconds_local: float, device: torch.device | str 
         dist.all_reduce(secs, op=dist.ReduceOp.MAX)
         return float(units.item() / secs.item())
     return float(t[0].item() / t[1].item())
+
+
+def install_dictionary(D: torch.Tensor, src: int = 0) -> torch.Tensor:
+    """Every rank ends up with rank `src`'s dictionary: one broadcast at install time (a new
+    prompt's online atoms, a newly trained dictionary), never on the encode path.  D must have
+    the same shape and dtype on every rank and is overwritten in place on the others."""
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.broadcast(D, src=src)
+    return D

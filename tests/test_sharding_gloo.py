@@ -40,6 +40,9 @@ def _worker(rank, world, port, M, out):
     w = wl.llama2_layer(tokens=4, N=128)
     b, e = sharding.shard_rows(M, rank, world)
     res = orc.mp_encode(w.D, w.X[b:e], 4)          # each rank encodes only its rows
+    Dl = torch.from_numpy(w.D.copy()) if rank == 0 else torch.zeros(w.D.shape)
+    sharding.install_dictionary(Dl, src=0)         # rank 1 starts without the dictionary
+    assert np.array_equal(Dl.numpy(), w.D)
     rate = sharding.job_rate(e - b, 1.0 + rank)    # rank 1 is "slower"
     np.save(os.path.join(out, f"idx{rank}.npy"), res.idx)
     np.save(os.path.join(out, f"meta{rank}.npy"), np.array([b, e, rate]))
