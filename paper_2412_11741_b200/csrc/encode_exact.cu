@@ -34,7 +34,7 @@ struct Smem {
 };
 
 template <int D_>
-__global__ void __launch_bounds__(NT, 1)
+__global__ void __launch_bounds__(NT, 2)
 encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int x_dtype, int64_t ldx, int64_t M, int N,
                     int s, uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype, int64_t ldc) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -141,7 +141,8 @@ encode_exact_kernel(const float* __restrict__ D, const void* __restrict__ X, int
 int launch_encode_exact(const EncodeArgs& a) {
     const int64_t n_tiles = (a.M + BM - 1) / BM;
     if (n_tiles == 0) return CSR_OK;
-    const int grid = (int)(n_tiles < (int64_t)sm_count() ? n_tiles : (int64_t)sm_count());
+    const int64_t resident = 2 * (int64_t)sm_count();   // two CTAs per SM
+    const int grid = (int)(n_tiles < resident ? n_tiles : resident);
     cudaError_t e;
     if (a.d == 128) {
         const size_t smem = sizeof(Smem<128>);

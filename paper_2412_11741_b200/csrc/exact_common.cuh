@@ -10,7 +10,7 @@ namespace exact {
 
 constexpr int BM = 64;        // rows per CTA
 constexpr int BN = 128;       // atoms per dictionary tile
-constexpr int BK = 16;        // channels per staged chunk
+constexpr int BK = 8;         // channels per staged chunk (small: two CTAs of the row-tile encoder fit one SM)
 constexpr int NT = 256;       // threads per CTA
 constexpr int AS_LD = BM + 4; // leading dimension of the transposed fp32 residual
 constexpr int BS_LD = BN + 4;
@@ -59,13 +59,15 @@ __device__ __forceinline__ void sweep_tiles(const float* __restrict__ D, int N, 
     const int ty = tid >> 4;   // row group: rows ty*4 .. ty*4+3
     const int total_chunks = (bt1 - bt0) * KCH;
     if (total_chunks <= 0) return;
-    float4 stage[2];
+    constexpr int KQ = BK / 4;                            // float4 per atom per chunk
+    constexpr int FPT = BN * KQ / NT;                     // float4 staged per thread
+    float4 stage[FPT];
     auto gload = [&](int chunk) {
         const int bt = bt0 + chunk / KCH, kc = chunk % KCH;
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < FPT; ++i) {
             const int f = tid + i * NT;
-            const int atom = f >> 2, kq = f & 3;
+            const int atom = f / KQ, kq = f % KQ;
             const int n = bt * BN + atom;
             stage[i] = (n < N) ? *reinterpret_cast<const float4*>(D + (int64_t)n * D_ + kc * BK + kq * 4)
                                : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -73,9 +75,9 @@ __device__ __forceinline__ void sweep_tiles(const float* __restrict__ D, int N, 
     };
     auto sstore = [&](int buf) {
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < FPT; ++i) {
             const int f = tid + i * NT;
-            const int atom = f >> 2, kq = f & 3;
+            const int atom = f / KQ, kq = f % KQ;
             Bs[buf][kq * 4 + 0][atom] = stage[i].x;
             Bs[buf][kq * 4 + 1][atom] = stage[i].y;
             Bs[buf][kq * 4 + 2][atom] = stage[i].z;
