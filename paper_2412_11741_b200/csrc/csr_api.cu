@@ -265,6 +265,11 @@ int encode_device(const csr_encode_params_t* p) {
         return launch_encode_exact(a);
     }
 
+    // few rows: library-owned scratch lets the dictionary be split across the SMs (a caller
+    // workspace is sized for the bf16 copy only, so with one the whole-job kernel runs)
+    const bool split = !p->workspace && encode_fast_split_applies(p->M, p->N) && !getenv("CSR_FAST_NO_SPLIT");
+    const size_t dict_b = (encode_fast_workspace_bytes(p->d, p->N) + 1023) / 1024 * 1024;
+    const size_t split_b = split ? encode_fast_split_scratch_bytes(p->M, p->d, p->N) : 0;
     if (p->dict) {
         const csr_dict* dc = static_cast<const csr_dict*>(p->dict);
         int dev = -1;
@@ -273,8 +278,9 @@ int encode_device(const csr_encode_params_t* p) {
         if (dc->device != dev || dc->D != p->D || dc->N != p->N || dc->d != p->d)
             return fail(CSR_ERR_INVALID_ARG, "dict was created for another device, D, N or d");
         void* wbase = nullptr;
-        if (int rc = ensure_work(0, &wbase)) return rc;           // only the status word is used
-        return launch_encode_fast_prepared(a, dc->bf16, static_cast<uint32_t*>(wbase));
+        if (int rc = ensure_work(split_b, &wbase)) return rc;     // status word (+ split scratch)
+        void* sp = split ? align_up(static_cast<char*>(wbase) + kStatusBytes, 1024) : nullptr;
+        return launch_encode_fast_prepared(a, dc->bf16, static_cast<uint32_t*>(wbase), sp);
     }
     void* base = nullptr;
     if (p->workspace) {
@@ -286,11 +292,12 @@ int encode_device(const csr_encode_params_t* p) {
         cudaError_t e = cudaMemsetAsync(base, 0, kStatusBytes, a.stream);
         if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
     } else {
-        if (int rc = ensure_work(encode_fast_workspace_bytes(p->d, p->N), &base)) return rc;
+        if (int rc = ensure_work(dict_b + split_b, &base)) return rc;
     }
     uint32_t* status = static_cast<uint32_t*>(base);
-    void* scratch = align_up(static_cast<char*>(base) + kStatusBytes, 1024);
-    return launch_encode_fast(a, scratch, status);
+    char* scratch = static_cast<char*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024));
+    if (int rc = prepare_fast_dictionary(a.D, a.N, a.d, scratch, a.stream)) return rc;
+    return launch_encode_fast_prepared(a, scratch, status, split ? scratch + dict_b : nullptr);
 }
 
 }  // namespace
@@ -493,7 +500,8 @@ int csr_dict_train_step(const csr_train_params_t* p) {
         return fail(CSR_ERR_ALIGNMENT, "D and X must be 16-byte aligned, losses 8-byte aligned");
     if (!(p->lr >= 0.f) || !(p->beta >= 0.f)) return fail(CSR_ERR_INVALID_ARG, "lr and beta must be >= 0");
     // scratch layout: [encoder's own region][idx][coef][grad_mse][grad_div]
-    size_t enc = encode_fast_workspace_bytes(p->d, p->N);
+    size_t enc = (encode_fast_workspace_bytes(p->d, p->N) + 1023) / 1024 * 1024;
+    if (p->M > 0 && encode_fast_split_applies(p->M, p->N)) enc += encode_fast_split_scratch_bytes(p->M, p->d, p->N);
     if (p->M > 0 && encode_exact_split_applies(p->M, p->N)) {
         const size_t sp = encode_exact_split_scratch_bytes(p->M, p->d, p->N);
         if (sp > enc) enc = sp;

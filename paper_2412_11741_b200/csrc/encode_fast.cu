@@ -398,6 +398,115 @@ __global__ void dict_to_bf16_kernel(const float4* __restrict__ src, uint2* __res
 }
 
 // ---------------------------------------------------------------------------------------
+// few rows: the dictionary is split across CTAs, one iteration per launch
+// ---------------------------------------------------------------------------------------
+// R_0 = x rounded to bf16, dense [M][d]; one thread per 16-byte chunk of eight channels.
+template <int D_>
+__global__ void rows_to_bf16_kernel(const void* __restrict__ X, int x_dtype, int64_t ldx, int64_t M, uint4* __restrict__ Rb) {
+    constexpr int CHUNKS = D_ / 8;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M * CHUNKS) return;
+    const int64_t m = i / CHUNKS;
+    const int c = (int)(i % CHUNKS);
+    uint4 v;
+    if (x_dtype == CSR_DTYPE_BF16) {
+        v = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(X) + m * ldx + 8 * c);
+    } else {
+        float f[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) f[k] = load_elem(X, x_dtype, m * ldx + 8 * c + k);
+        v.x = pack_bf16(f[0], f[1]);
+        v.y = pack_bf16(f[2], f[3]);
+        v.z = pack_bf16(f[4], f[5]);
+        v.w = pack_bf16(f[6], f[7]);
+    }
+    Rb[i] = v;
+}
+
+// Pick of one iteration for the split sweep: merges a row's per-CTA (key, tile) pairs (largest
+// key, lowest tile among equal keys: the order in which one CTA would have met them), then
+// does exactly what pick_and_update does, on the residual rows kept in global memory.
+// Eight lanes per row, four rows per warp.
+template <int D_, int G>
+__global__ void __launch_bounds__(128)
+split_pick_kernel(const uint16_t* __restrict__ Db, uint4* __restrict__ Rb, const uint2* __restrict__ partial, int n_splits,
+                  int64_t M, int g, int update, uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype,
+                  int64_t ldc) {
+    constexpr int CH = D_ / 64;
+    constexpr int APR = D_ / 8;
+    constexpr int NG = TILE_N / G;
+    const int lane = threadIdx.x & 31, sub = lane >> 3, l8 = lane & 7;
+    const int64_t m = ((int64_t)blockIdx.x * 4 + (threadIdx.x >> 5)) * 4 + sub;
+    const bool valid = m < M;
+    uint32_t key = 0, t = 0;
+    if (valid) {
+        for (int j = l8; j < n_splits; j += 8) {
+            const uint2 pr = partial[m * n_splits + j];
+            if (pr.x > key || (pr.x == key && pr.y < t)) {
+                key = pr.x;
+                t = pr.y;
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) {
+        const uint32_t ok = __shfl_xor_sync(0xffffffffu, key, o), ot = __shfl_xor_sync(0xffffffffu, t, o);
+        if (ok > key || (ok == key && ot < t)) {
+            key = ok;
+            t = ot;
+        }
+    }
+    const int n0 = static_cast<int>(t) * TILE_N + (NG - 1 - static_cast<int>(key & static_cast<uint32_t>(NG - 1))) * G;
+    const int64_t mr = valid ? m : 0;
+    uint4 atom[G][CH], rv[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+        rv[c] = Rb[mr * APR + l8 * CH + c];
+#pragma unroll
+        for (int j = 0; j < G; ++j)
+            atom[j][c] = __ldg(reinterpret_cast<const uint4*>(Db + static_cast<size_t>(n0) * D_) + j * APR + l8 * CH + c);
+    }
+    float dot[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) {
+        float ev = 0.f, od = 0.f;
+#pragma unroll
+        for (int c = 0; c < CH; ++c) dot8(rv[c], atom[j][c], ev, od);
+        dot[j] = ev + od;
+    }
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1)
+#pragma unroll
+        for (int j = 0; j < G; ++j) dot[j] += __shfl_xor_sync(0xffffffffu, dot[j], o);
+    if (!valid) return;
+    float coef = dot[0];
+    int jb = 0;
+#pragma unroll
+    for (int j = 1; j < G; ++j)
+        if (fabsf(dot[j]) > fabsf(coef)) {
+            coef = dot[j];
+            jb = j;
+        }
+    if (update) {
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            uint4 av = atom[0][c];
+#pragma unroll
+            for (int j = 1; j < G; ++j)
+                if (jb == j) av = atom[j][c];
+            Rb[m * APR + l8 * CH + c] = axpy8(rv[c], av, coef);
+        }
+    }
+    if (l8 == 0) {
+        out_idx[m * ldc + g] = static_cast<uint16_t>(n0 + jb);
+        if (coef_dtype == CSR_DTYPE_F16)
+            reinterpret_cast<__half*>(out_coef)[m * ldc + g] = __float2half_rn(coef);
+        else
+            reinterpret_cast<float*>(out_coef)[m * ldc + g] = coef;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
 // the encoder
 // ---------------------------------------------------------------------------------------
 template <int D_, int G>
@@ -405,7 +514,7 @@ __global__ void __launch_bounds__(NT, 1)
 encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* __restrict__ Db,
                    const void* __restrict__ X, int x_dtype, int64_t ldx, int64_t M, int N, int s,
                    uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype, int64_t ldc, int vec_codes,
-                   uint32_t key_mask, uint32_t* status) {
+                   uint32_t key_mask, uint32_t* status, int n_splits, uint2* __restrict__ partial) {
     using S = FastSmem<D_>;
     extern __shared__ uint8_t smem_raw[];
     S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -414,6 +523,13 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
     const int lane = threadIdx.x & 31;
     const int T = (N + TILE_N - 1) / TILE_N;                // dictionary tiles per sweep (the last may be half)
     const int64_t n_pairs = (M + 2 * TILE_M - 1) / (2 * TILE_M);
+    // Few rows (n_splits > 1): n_splits CTAs share one pair of row tiles, CTA j sweeping the
+    // dictionary tiles j, j + n_splits, ... of ONE iteration (s == 1 is passed) and leaving each
+    // row's best (key, tile) in `partial` for the pick kernel instead of picking itself.
+    const int t_begin = n_splits > 1 ? (int)(blockIdx.x % n_splits) : 0;
+    const int t_step = n_splits > 1 ? n_splits : 1;
+    const int64_t pair_first = n_splits > 1 ? blockIdx.x / n_splits : blockIdx.x;
+    const int64_t pair_step = n_splits > 1 ? gridDim.x / n_splits : gridDim.x;
     constexpr int KH = D_ / STAGE_CH;                       // stages per dictionary tile
     constexpr int KSTEPS = STAGE_CH / UMMA_K;               // MMAs per stage
     constexpr int CHUNKS = D_ / 8;                          // 16-byte chunks per row
@@ -449,9 +565,9 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_d)) : "memory");
             uint32_t p = 0;
             bool ok = true;
-            for (int64_t pair = blockIdx.x; pair < n_pairs && ok; pair += gridDim.x) {
+            for (int64_t pair = pair_first; pair < n_pairs && ok; pair += pair_step) {
                 for (int g = 0; g < s && ok; ++g) {
-                    for (int t = 0; t < T && ok; ++t) {
+                    for (int t = t_begin; t < T && ok; t += t_step) {
                         for (int h = 0; h < KH; ++h, ++p) {
                             const int stage = p % STAGES;
                             if (!wait_bounded(&sm.empty_b[stage], ((p / STAGES) & 1) ^ 1, wc)) {
@@ -480,11 +596,11 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         if (lane == 0) {
             uint32_t p = 0, accn = 0, steps = 0;
             bool ok = true;
-            for (int64_t pair = blockIdx.x; pair < n_pairs && ok; pair += gridDim.x) {
+            for (int64_t pair = pair_first; pair < n_pairs && ok; pair += pair_step) {
                 for (int g = 0; g < s && ok; ++g, ++steps) {
-                    for (int t = 0; t < T && ok; ++t, p += KH, ++accn) {
+                    for (int t = t_begin; t < T && ok; t += t_step, p += KH, ++accn) {
                         for (int tile = 0; tile < 2 && ok; ++tile) {
-                            if (t == 0 && !wait_bounded(&sm.res_ready[tile], steps & 1, wc)) {
+                            if (t == t_begin && !wait_bounded(&sm.res_ready[tile], steps & 1, wc)) {
                                 ok = false;
                                 break;
                             }
@@ -538,7 +654,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + tile * TILE_N;
         uint32_t accn = 0;
         bool ok = true;
-        for (int64_t pair = blockIdx.x; pair < n_pairs && ok; pair += gridDim.x) {
+        for (int64_t pair = pair_first; pair < n_pairs && ok; pair += pair_step) {
             const int64_t m = pair * (2 * TILE_M) + slot;
             const bool valid = m < M;
             // ---- R_0 = x, rounded to bf16, into the operand tile ----
@@ -589,7 +705,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             for (int g = 0; g < s && ok; ++g) {
                 // ---- sweep: running arg-max of |correlation| over all atom tiles ----
                 uint32_t best_key = 0, best_t = 0;
-                for (int t = 0; t < T; ++t, ++accn) {
+                for (int t = t_begin; t < T; t += t_step, ++accn) {
                     bool got = wait_bounded(&sm.acc_full[tile], accn & 1, wc);
                     got = __all_sync(0xffffffffu, got);
                     if (!got) {
@@ -634,6 +750,10 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     }
                 }
                 if (!ok) break;
+                if (partial) {                              // split sweep: the pick kernel takes over
+                    if (valid) partial[m * n_splits + t_begin] = make_uint2(best_key, best_t);
+                    continue;
+                }
                 // ---- pick, signed coefficient, residual update ----
                 const int gi = g & (CODE_BLOCK - 1);
                 const int n0 = static_cast<int>(best_t) * TILE_N +
@@ -707,13 +827,15 @@ EncodeTiledFn get_encode_tiled() {
 }
 
 template <int D_, int G>
-int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status) {
+int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, int n_splits,
+           uint2* partial) {
     const size_t smem = sizeof(FastSmem<D_>) + 1024;
     cudaError_t e =
         cudaFuncSetAttribute(encode_fast_kernel<D_, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     const int64_t n_pairs = (a.M + 2 * TILE_M - 1) / (2 * TILE_M);
-    const int grid = (int)(n_pairs < (int64_t)sm_count() ? n_pairs : (int64_t)sm_count());
+    const int grid = n_splits > 1 ? (int)(n_pairs * n_splits)
+                                  : (int)(n_pairs < (int64_t)sm_count() ? n_pairs : (int64_t)sm_count());
     // keys keep the magnitude bits above the group tag; with G == 1 the key is built from the
     // raw value, so the mask clears the sign bit as well
     const uint32_t key_mask = (G == 1 ? 0x7FFFFFFFu : 0xFFFFFFFFu) & ~static_cast<uint32_t>(TILE_N / G - 1);
@@ -722,7 +844,7 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
     const int vec_codes = (a.s % 8 == 0) && (a.ld_code % 8 == 0) && (ci % 16 == 0) && (cc % 16 == 0);
     encode_fast_kernel<D_, G><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
                                                            a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask,
-                                                           status);
+                                                           status, n_splits, partial);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "encode_fast launch: %s", cudaGetErrorString(e));
     return CSR_OK;
@@ -745,14 +867,66 @@ int group_size(int d, int N) {
 template <int D_>
 int launch_d(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status) {
     switch (group_size(D_, a.N)) {
-        case 1: return launch<D_, 1>(a, tmap, Db, status);
-        case 2: return launch<D_, 2>(a, tmap, Db, status);
-        case 8: return launch<D_, 8>(a, tmap, Db, status);
-        default: return launch<D_, 4>(a, tmap, Db, status);
+        case 1: return launch<D_, 1>(a, tmap, Db, status, 0, nullptr);
+        case 2: return launch<D_, 2>(a, tmap, Db, status, 0, nullptr);
+        case 8: return launch<D_, 8>(a, tmap, Db, status, 0, nullptr);
+        default: return launch<D_, 4>(a, tmap, Db, status, 0, nullptr);
+    }
+}
+
+// Few rows: how many CTAs share a pair of row tiles (1 = the whole dictionary per CTA).
+int split_count(int64_t M, int N) {
+    const int64_t n_pairs = (M + 2 * TILE_M - 1) / (2 * TILE_M);
+    const int T = (N + TILE_N - 1) / TILE_N;
+    if (n_pairs < 1 || n_pairs * 2 > sm_count() || T < 2) return 1;
+    int ns = (int)(sm_count() / n_pairs);
+    if (ns > T) ns = T;
+    if (ns > 32) ns = 32;
+    return ns;
+}
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+// One launch of the sweep (every CTA a slice of the dictionary, s = 1) and one of the pick
+// per iteration; the residual rows live in global memory as bf16 in between.
+template <int D_, int G>
+int run_split_g(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, void* scratch) {
+    const int ns = split_count(a.M, a.N);
+    uint4* Rb = static_cast<uint4*>(scratch);
+    uint2* partial = reinterpret_cast<uint2*>(static_cast<char*>(scratch) + align256((size_t)a.M * D_ * 2));
+    const int64_t chunks = a.M * (D_ / 8);
+    rows_to_bf16_kernel<D_><<<(unsigned)((chunks + 255) / 256), 256, 0, a.stream>>>(a.X, a.x_dtype, a.ldx, a.M, Rb);
+    EncodeArgs b = a;
+    b.X = Rb;
+    b.x_dtype = CSR_DTYPE_BF16;
+    b.ldx = D_;
+    b.s = 1;
+    const unsigned pick_blocks = (unsigned)((a.M + 15) / 16);
+    for (int g = 0; g < a.s; ++g) {
+        if (int rc = launch<D_, G>(b, tmap, Db, status, ns, partial)) return rc;
+        split_pick_kernel<D_, G><<<pick_blocks, 128, 0, a.stream>>>(Db, Rb, partial, ns, a.M, g, g + 1 < a.s, a.out_idx, a.out_coef,
+                                                                a.coef_dtype, a.ld_code);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "encode_fast split launch: %s", cudaGetErrorString(e));
+    return CSR_OK;
+}
+
+template <int D_>
+int run_split(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, void* scratch) {
+    switch (group_size(D_, a.N)) {
+        case 1: return run_split_g<D_, 1>(a, tmap, Db, status, scratch);
+        case 2: return run_split_g<D_, 2>(a, tmap, Db, status, scratch);
+        case 8: return run_split_g<D_, 8>(a, tmap, Db, status, scratch);
+        default: return run_split_g<D_, 4>(a, tmap, Db, status, scratch);
     }
 }
 
 }  // namespace
+
+bool encode_fast_split_applies(int64_t M, int N) { return M > 0 && split_count(M, N) > 1; }
+size_t encode_fast_split_scratch_bytes(int64_t M, int d, int N) {
+    return align256((size_t)M * d * 2) + align256((size_t)M * split_count(M, N) * sizeof(uint2));
+}
 
 // The bf16 copy holds N rounded up to a multiple of 8 atoms; the extra rows are zero, so a
 // group of up to 8 candidate atoms never reaches past the copy.
@@ -780,10 +954,10 @@ int prepare_fast_dictionary(const float* D, int N, int d, void* workspace, cudaS
 int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status) {
     if (a.M == 0) return CSR_OK;
     if (int rc = prepare_fast_dictionary(a.D, a.N, a.d, workspace, a.stream)) return rc;
-    return launch_encode_fast_prepared(a, workspace, status);
+    return launch_encode_fast_prepared(a, workspace, status, nullptr);
 }
 
-int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint32_t* status) {
+int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint32_t* status, void* split_scratch) {
     if (a.M == 0) return CSR_OK;
     void* workspace = const_cast<void*>(dict_bf16);
     if ((reinterpret_cast<uintptr_t>(workspace) & 1023u) != 0)
@@ -804,6 +978,10 @@ int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint
     if (r != CUDA_SUCCESS) return fail(CSR_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
 
     const uint16_t* Db = static_cast<const uint16_t*>(workspace);
+    if (split_scratch) {
+        if (a.d == 128) return run_split<128>(a, tmap, Db, status, split_scratch);
+        return run_split<64>(a, tmap, Db, status, split_scratch);
+    }
     if (a.d == 128) return launch_d<128>(a, tmap, Db, status);
     return launch_d<64>(a, tmap, Db, status);
 }

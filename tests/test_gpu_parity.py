@@ -233,6 +233,34 @@ def test_fast_any_dictionary_size(csr, N, G, monkeypatch):
         assert np.array_equal(idx, res.idx) and np.all(np.abs(coef[:, 0] - res.coef[:, 0]) <= 2.0 ** -8 * xn)   # bf16 atom
 
 
+@pytest.mark.parametrize("M,N,d,s,kind", [(1, 8192, 128, 16, "bf16"), (128, 8192, 128, 16, "bf16"), (300, 1000, 128, 5, "f32"),
+                                          (2000, 4096, 64, 8, "f16"), (9000, 2048, 128, 4, "bf16"), (16, 65536, 64, 3, "bf16")])
+def test_fast_few_rows_split_dictionary_path(csr, M, N, d, s, kind, monkeypatch):
+    """Few rows: the dictionary is split across CTAs, one sweep and one pick launch per
+    iteration.  The codes must be those of the one-launch kernel bit for bit."""
+    rng = np.random.default_rng(M * 7 + N)
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    X = rng.standard_normal((M, d)).astype(np.float32)
+    X = wl.round_to_bf16(X) if kind == "bf16" else X.astype(np.float16).astype(np.float32) if kind == "f16" else X
+    if M > 2:
+        X[1] = 0.0
+    Dd = torch.from_numpy(D).to(DEV)
+    Xd = torch.from_numpy(X).to(DEV).to({"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[kind])
+    i1, c1 = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float32)
+    assert csr.csr_device_status() == csr.CSR_OK
+    h = csr.csr_dict_create(Dd)
+    i3, c3 = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float16, dict=h)       # handle + packed coefficients
+    csr.csr_dict_destroy(h)
+    monkeypatch.setenv("CSR_FAST_NO_SPLIT", "1")
+    i2, c2 = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float32)
+    monkeypatch.delenv("CSR_FAST_NO_SPLIT")
+    assert np.array_equal(_np_idx(i1), _np_idx(i2)) and torch.equal(c1, c2)
+    assert np.array_equal(_np_idx(i3), _np_idx(i2)) and torch.equal(c3, c2.to(torch.float16))
+    if N >= 1000 and M >= 100:
+        rep = parity.compare_fast(D, wl.round_to_bf16(X), s, _np_idx(i1), c1.cpu().numpy())
+        assert rep.ok, rep.detail
+
+
 def test_fast_fp32_input_and_odd_s(csr):
     rng = np.random.default_rng(13)
     D = wl.normalise_rows(rng.standard_normal((1024, 128)).astype(np.float32))
