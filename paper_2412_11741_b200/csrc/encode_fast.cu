@@ -882,7 +882,10 @@ int split_count(int64_t M, int N) {
     int ns = (int)(sm_count() / n_pairs);
     if (ns > T) ns = T;
     if (ns > 32) ns = 32;
-    return ns;
+    // Worth it only if an iteration's sweep over all T tiles by one CTA (about 1.55 us per
+    // tile, measured) outlasts two launches (about 12 us) plus the sweep of a slice.
+    const float whole = 1.55f * T, sliced = 1.2f * (12.f + 1.6f * ((T + ns - 1) / ns));
+    return whole > sliced ? ns : 1;
 }
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
