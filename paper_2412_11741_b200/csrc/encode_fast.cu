@@ -429,8 +429,8 @@ __global__ void rows_to_bf16_kernel(const void* __restrict__ X, int x_dtype, int
 // Eight lanes per row, four rows per warp.
 template <int D_, int G>
 __global__ void __launch_bounds__(128)
-split_pick_kernel(const uint16_t* __restrict__ Db, uint4* __restrict__ Rb, const uint2* __restrict__ partial, int n_splits,
-                  int64_t M, int g, int update, uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype,
+split_pick_kernel(const uint16_t* __restrict__ Db, int N, uint4* __restrict__ Rb, const uint2* __restrict__ partial,
+                  int n_splits, int64_t M, int g, int update, uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype,
                   int64_t ldc) {
     constexpr int CH = D_ / 64;
     constexpr int APR = D_ / 8;
@@ -456,7 +456,8 @@ split_pick_kernel(const uint16_t* __restrict__ Db, uint4* __restrict__ Rb, const
             t = ot;
         }
     }
-    const int n0 = static_cast<int>(t) * TILE_N + (NG - 1 - static_cast<int>(key & static_cast<uint32_t>(NG - 1))) * G;
+    const int n0 = min(static_cast<int>(t) * TILE_N + (NG - 1 - static_cast<int>(key & static_cast<uint32_t>(NG - 1))) * G,
+                       ((N + 7) / 8) * 8 - G);     // as in the one-launch kernel: never past the padded copy
     const int64_t mr = valid ? m : 0;
     uint4 atom[G][CH], rv[CH];
 #pragma unroll
@@ -756,8 +757,11 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 }
                 // ---- pick, signed coefficient, residual update ----
                 const int gi = g & (CODE_BLOCK - 1);
-                const int n0 = static_cast<int>(best_t) * TILE_N +
-                               (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G;
+                // (NaN correlations can make a zero-filled column past the dictionary win: keep the
+                // gather inside the padded bf16 copy whatever the keys say)
+                const int n0 = min(static_cast<int>(best_t) * TILE_N +
+                                       (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G,
+                                   ((N + 7) / 8) * 8 - G);
                 pick_and_update<D_, G>(Atile, q, lane, Db, n0, g + 1 < s, code_idx, code_coef, gi);
                 if (g + 1 < s) {
                     fence_proxy_async_smem();
@@ -906,7 +910,7 @@ int run_split_g(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db
     const unsigned pick_blocks = (unsigned)((a.M + 15) / 16);
     for (int g = 0; g < a.s; ++g) {
         if (int rc = launch<D_, G>(b, tmap, Db, status, ns, partial)) return rc;
-        split_pick_kernel<D_, G><<<pick_blocks, 128, 0, a.stream>>>(Db, Rb, partial, ns, a.M, g, g + 1 < a.s, a.out_idx, a.out_coef,
+        split_pick_kernel<D_, G><<<pick_blocks, 128, 0, a.stream>>>(Db, a.N, Rb, partial, ns, a.M, g, g + 1 < a.s, a.out_idx, a.out_coef,
                                                                 a.coef_dtype, a.ld_code);
     }
     cudaError_t e = cudaGetLastError();

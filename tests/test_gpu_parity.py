@@ -571,3 +571,28 @@ def test_random_shapes_both_modes(csr, seed):
         e_gpu = orc.relative_error(X, orc.reconstruct(D, gi.astype(np.int32), gc.astype(np.float64)))
         e_or = res.resnorm[:, -1] / np.maximum(np.linalg.norm(X.astype(np.float64), axis=1), 1e-300)
         assert np.all(e_gpu <= 1.3 * e_or + 2.0 ** -6), (d, N, M, s, kind)
+
+
+@pytest.mark.parametrize("M,N", [(700, 1000), (64, 8192)])
+def test_nan_and_inf_rows_do_no_harm(csr, M, N):
+    """NaN or Inf in X: those rows' codes are unspecified, but the calls return, no device-side
+    wait expires, every index stays below 65536 and inside what the de-sparse kernel accepts,
+    and the other rows get exactly the codes they get without the bad rows."""
+    rng = np.random.default_rng(M)
+    D = wl.normalise_rows(rng.standard_normal((N, 128)).astype(np.float32))
+    X = wl.round_to_bf16(rng.standard_normal((M, 128)).astype(np.float32))
+    bad = X.copy()
+    bad[5, 3] = np.nan
+    bad[9] = np.inf
+    bad[17, 100] = -np.inf
+    good = np.ones(M, bool)
+    good[[5, 9, 17]] = False
+    Dd = torch.from_numpy(D).to(DEV)
+    for mode, dt in ((csr.CSR_MODE_BF16_FAST, torch.bfloat16), (csr.CSR_MODE_FP32_EXACT, torch.float32)):
+        i0, c0 = csr.csr_encode_ex(Dd, torch.from_numpy(X).to(DEV).to(dt), 6, mode=mode, coef_dtype=torch.float32)
+        i1, c1 = csr.csr_encode_ex(Dd, torch.from_numpy(bad).to(DEV).to(dt), 6, mode=mode, coef_dtype=torch.float32)
+        assert csr.csr_device_status() == csr.CSR_OK
+        g = torch.from_numpy(good).to(DEV)
+        assert torch.equal(i0.view(torch.int16)[g], i1.view(torch.int16)[g]) and torch.equal(c0[g], c1[g])
+        xh = csr.csr_reconstruct_ex(Dd, i1, c1, out_dtype=torch.float32)       # clamps whatever the bad rows hold
+        assert bool(torch.isfinite(xh[g]).all())
