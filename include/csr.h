@@ -154,6 +154,21 @@ int csr_reconstruct(const void* D, const uint16_t* idx, const void* coef, int64_
 int csr_reconstruct_ex(const csr_reconstruct_params_t* p);
 
 /*
+ * One decoding step's attention over a cache kept as codes ("De-Sparse to restore" followed by
+ * the attention it feeds, with nothing restored): for every stream b and query head h
+ *     weights[b][h][:] = softmax_t( scale * Q[b][h] . X~_K[b][t] )          (csr_key_scores + softmax)
+ *     out[b][h][:]     = sum_t weights[b][h][t] * X~_V[b][t]                 (csr_value_mix)
+ * Keys and values have their own dictionaries (Dk [Nk][d], Dv [Nv][d]) and code arrays
+ * ([B][T][sk] and [B][T][sv], one coef_dtype).  `weights` is a caller buffer [B][H][T] fp32 that
+ * receives the attention weights; out is [B][H][d] fp32.  T >= 1.  Limits, alignment and
+ * reproducibility as for csr_key_scores / csr_value_mix; no causal mask is applied (a
+ * decoding step attends to the whole cache).
+ */
+int csr_decode_attention(const void* Dk, int Nk, const void* Dv, int Nv, int d, const void* Q, int q_dtype, int B, int H,
+                         const uint16_t* k_idx, const void* k_coef, int sk, const uint16_t* v_idx, const void* v_coef,
+                         int sv, int coef_dtype, int64_t T, float scale, float* weights, float* out, void* stream);
+
+/*
  * Packs fp32 coefficients into the stored form of "Analysis for CSR" (fp16, round to
  * nearest even): for codes that were produced with coef_dtype F32, e.g. by the exact mode
  * for verification, and are now to be kept.  The indices are stored as produced.  n values,

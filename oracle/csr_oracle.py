@@ -161,6 +161,16 @@ def value_mix(D: np.ndarray, W: np.ndarray, idx: np.ndarray, coef: np.ndarray) -
     return out
 
 
+def decode_attention(Dk, Dv, Q, k_idx, k_coef, v_idx, v_coef, scale: float):
+    """softmax_t(scale * Q . X~_K[t]) applied to X~_V, both tensors restored by Eq. 12; returns
+    (out [B][H][d], weights [B][H][T]) in fp64."""
+    sc = key_scores(Dk, Q, k_idx, k_coef, scale)
+    sc = sc - sc.max(axis=2, keepdims=True)
+    w = np.exp(sc)
+    w /= w.sum(axis=2, keepdims=True)
+    return value_mix(Dv, w, v_idx, v_coef), w
+
+
 # --- one training step of the offline dictionary ("NeuralDict") -----------------------------
 
 def mse_loss_and_grad(D: np.ndarray, X: np.ndarray, idx: np.ndarray, coef: np.ndarray):

@@ -33,7 +33,7 @@ CSR_MODE_BF16_FAST = 1
 
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
-    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_dict_append", "csr_dict_create", "csr_dict_destroy", "csr_dict_train_step", "csr_key_scores", "csr_pack_coefficients", "csr_value_mix",
+    "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_decode_attention", "csr_dict_append", "csr_dict_create", "csr_dict_destroy", "csr_dict_train_step", "csr_key_scores", "csr_pack_coefficients", "csr_value_mix",
     "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
@@ -120,6 +120,9 @@ def lib() -> ctypes.CDLL:
         L.csr_key_scores.restype = i32
         L.csr_value_mix.argtypes = [vp, i32, i32, vp, i32, i32, vp, vp, i32, i64, i32, vp, vp]
         L.csr_value_mix.restype = i32
+        L.csr_decode_attention.argtypes = [vp, i32, vp, i32, i32, vp, i32, i32, i32, vp, vp, i32, vp, vp, i32, i32, i64, f32,
+                                           vp, vp, vp]
+        L.csr_decode_attention.restype = i32
         L.csr_pack_coefficients.argtypes = [vp, i64, vp, vp]
         L.csr_pack_coefficients.restype = i32
         L.csr_dict_create.argtypes = [vp, i32, i32, vp, ctypes.POINTER(vp)]
@@ -410,6 +413,33 @@ def csr_dict_train_step(D: torch.Tensor, X: torch.Tensor, s: int, lr: float, bet
     with torch.cuda.device(D.device):
         _check(lib().csr_dict_train_step(ctypes.byref(p)))
     return losses
+
+
+def csr_decode_attention(Dk: torch.Tensor, Dv: torch.Tensor, Q: torch.Tensor, k_idx: torch.Tensor, k_coef: torch.Tensor,
+                         v_idx: torch.Tensor, v_coef: torch.Tensor, scale: float,
+                         weights: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None):
+    """csr_decode_attention: softmax(scale * Q K~^T) V~ straight from the codes.  Q [B][H][d]; key
+    codes [B][T][sk], value codes [B][T][sv]; returns (out [B][H][d], weights [B][H][T]), fp32."""
+    _check_codes(Dk, k_idx, k_coef)
+    _check_codes(Dv, v_idx, v_coef)
+    B, T, sk = k_idx.shape
+    sv = v_idx.shape[2]
+    d = Dk.shape[1]
+    assert v_idx.shape[:2] == (B, T) and Dv.shape[1] == d and k_coef.dtype == v_coef.dtype
+    assert Q.is_cuda and Q.is_contiguous() and Q.dim() == 3 and Q.shape[0] == B and Q.shape[2] == d
+    H = Q.shape[1]
+    if weights is None:
+        weights = torch.empty((B, H, T), dtype=torch.float32, device=Dk.device)
+    if out is None:
+        out = torch.empty((B, H, d), dtype=torch.float32, device=Dk.device)
+    assert weights.is_contiguous() and weights.dtype == torch.float32 and tuple(weights.shape) == (B, H, T)
+    assert out.is_contiguous() and out.dtype == torch.float32 and tuple(out.shape) == (B, H, d)
+    with torch.cuda.device(Dk.device):
+        _check(lib().csr_decode_attention(Dk.data_ptr(), Dk.shape[0], Dv.data_ptr(), Dv.shape[0], d, Q.data_ptr(),
+                                          _TORCH_DTYPE[Q.dtype], B, H, k_idx.data_ptr(), k_coef.data_ptr(), sk,
+                                          v_idx.data_ptr(), v_coef.data_ptr(), sv, _TORCH_DTYPE[k_coef.dtype], T,
+                                          float(scale), weights.data_ptr(), out.data_ptr(), _stream_ptr(Dk)))
+    return out, weights
 
 
 def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *,

@@ -293,6 +293,47 @@ value_scatter_kernel(int N, const float* __restrict__ W, int B, int H, const uin
     }
 }
 
+// Softmax over the T scores of one (stream, head) row, in place; one CTA per row, fp32, the
+// maximum subtracted first.  Rows are a few tens of KB and were just written: they come
+// from L2.
+__global__ void __launch_bounds__(NT)
+softmax_rows_kernel(float* __restrict__ S, int64_t T) {
+    __shared__ float red[NT / 32];
+    __shared__ float bcast;
+    float* row = S + (int64_t)blockIdx.x * T;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float mx = -INFINITY;
+    for (int64_t t = threadIdx.x; t < T; t += NT) mx = fmaxf(mx, row[t]);
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float m = red[0];
+        for (int j = 1; j < NT / 32; ++j) m = fmaxf(m, red[j]);
+        bcast = m;
+    }
+    __syncthreads();
+    mx = bcast;
+    float sum = 0.f;
+    for (int64_t t = threadIdx.x; t < T; t += NT) {
+        const float e = __expf(row[t] - mx);
+        row[t] = e;
+        sum += e;
+    }
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    __syncthreads();
+    if (lane == 0) red[warp] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int j = 0; j < NT / 32; ++j) t += red[j];
+        bcast = 1.0f / t;
+    }
+    __syncthreads();
+    const float inv = bcast;
+    for (int64_t t = threadIdx.x; t < T; t += NT) row[t] *= inv;
+}
+
 // Query heads whose N-vectors fit in shared memory side by side: 8, 4, 2 or 1 (0 = none fits).
 int head_group(int N, int H) {
     int hgp = 8;
@@ -343,6 +384,14 @@ int launch_key_scores(const AttnArgs& a, float* P) {
     cudaError_t e = hg == 8 ? run_key_scores<8>(a, P) : hg == 4 ? run_key_scores<4>(a, P)
                     : hg == 2 ? run_key_scores<2>(a, P) : run_key_scores<1>(a, P);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "key_scores launch: %s", cudaGetErrorString(e));
+    return CSR_OK;
+}
+
+int launch_softmax_rows(float* S, int64_t rows, int64_t T, cudaStream_t stream) {
+    if (rows == 0 || T == 0) return CSR_OK;
+    softmax_rows_kernel<<<(unsigned)rows, NT, 0, stream>>>(S, T);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "softmax launch: %s", cudaGetErrorString(e));
     return CSR_OK;
 }
 

@@ -93,6 +93,7 @@ struct AttnArgs {
 size_t attn_scratch_bytes(int B, int H, int N);
 int launch_key_scores(const AttnArgs& a, float* scratch);
 int launch_value_mix(const AttnArgs& a, float* scratch);
+int launch_softmax_rows(float* S, int64_t rows, int64_t T, cudaStream_t stream);   // in place, fp32
 
 // Gradient step of the dictionary on one batch whose codes (idx, fp32 coef, dense [M][s])
 // are given; losses[0] = L_MSE, losses[1] = L_div of the dictionary before the update.

@@ -487,6 +487,18 @@ int csr_value_mix(const void* D, int N, int d, const float* W, int B, int H, con
     return launch_value_mix(a, static_cast<float*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)));
 }
 
+int csr_decode_attention(const void* Dk, int Nk, const void* Dv, int Nv, int d, const void* Q, int q_dtype, int B, int H,
+                         const uint16_t* k_idx, const void* k_coef, int sk, const uint16_t* v_idx, const void* v_coef,
+                         int sv, int coef_dtype, int64_t T, float scale, float* weights, float* out, void* stream) {
+    if (T == 0 && B > 0) return fail(CSR_ERR_INVALID_ARG, "attention over an empty cache (T = 0) is undefined");
+    if (int rc = check_attn(Dv, Nv, d, weights, B, H, v_idx, v_coef, coef_dtype, T, sv, out)) return rc;
+    if (int rc = csr_key_scores(Dk, Nk, d, Q, q_dtype, B, H, k_idx, k_coef, coef_dtype, T, sk, scale, weights, stream))
+        return rc;
+    if (B == 0) return CSR_OK;
+    if (int rc = launch_softmax_rows(weights, (int64_t)B * H, T, static_cast<cudaStream_t>(stream))) return rc;
+    return csr_value_mix(Dv, Nv, d, weights, B, H, v_idx, v_coef, coef_dtype, T, sv, out, stream);
+}
+
 int csr_dict_train_step(const csr_train_params_t* p) {
     if (!p) return fail(CSR_ERR_INVALID_ARG, "params is NULL");
     if (p->struct_size != sizeof(csr_train_params_t))

@@ -197,3 +197,30 @@ def test_dictionary_training_step_matches_oracle(csr, N, d, M, s):
         losses = csr.csr_dict_train_step(Dd, Xd, s, 2e-3, beta, mode=mode).cpu().numpy()
     assert csr.csr_device_status() == csr.CSR_OK
     assert losses[0] < first and np.isfinite(losses).all()
+
+
+def test_decode_attention_over_encoded_cache(csr):
+    """A decoding step end to end: keys and values of 12 streams are encoded (separate
+    dictionaries, s = 8 for keys and 4 for values), then softmax(q K~^T / sqrt(d)) V~ is taken
+    straight from the codes and compared with the oracle, which restores both tensors."""
+    rng = np.random.default_rng(77)
+    B, H, T, d, Nk, Nv = 12, 4, 700, 128, 1024, 512
+    Dk = wl.normalise_rows(rng.standard_normal((Nk, d)).astype(np.float32))
+    Dv = wl.normalise_rows(rng.standard_normal((Nv, d)).astype(np.float32))
+    K = wl.round_to_bf16(rng.standard_normal((B * T, d)).astype(np.float32))
+    V = wl.round_to_bf16(rng.standard_normal((B * T, d)).astype(np.float32))
+    Q = (rng.standard_normal((B, H, d)) * 2).astype(np.float32)
+    Dkd, Dvd = torch.from_numpy(Dk).to(DEV), torch.from_numpy(Dv).to(DEV)
+    ki, kc = csr.csr_encode(Dkd, torch.from_numpy(K).to(DEV).to(torch.bfloat16), 8)
+    vi, vc = csr.csr_encode(Dvd, torch.from_numpy(V).to(DEV).to(torch.bfloat16), 4)
+    scale = 1.0 / np.sqrt(d)
+    out, w = csr.csr_decode_attention(Dkd, Dvd, torch.from_numpy(Q).to(DEV), ki.view(B, T, 8), kc.view(B, T, 8),
+                                      vi.view(B, T, 4), vc.view(B, T, 4), scale)
+    want_out, want_w = orc.decode_attention(Dk, Dv, Q, _np_idx(ki).astype(np.int32).reshape(B, T, 8),
+                                            kc.float().cpu().numpy().astype(np.float64).reshape(B, T, 8),
+                                            _np_idx(vi).astype(np.int32).reshape(B, T, 4),
+                                            vc.float().cpu().numpy().astype(np.float64).reshape(B, T, 4), scale)
+    w, out = w.cpu().numpy(), out.cpu().numpy()
+    assert np.allclose(w.sum(-1), 1.0, atol=1e-5)
+    assert np.all(np.abs(w - want_w) <= 1e-4 * want_w + 1e-9)             # exp of scores good to ~1e-5
+    assert np.all(np.abs(out - want_out) <= 2e-4 * np.abs(vc.float().cpu().numpy()).max())
