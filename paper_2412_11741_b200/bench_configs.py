@@ -120,11 +120,12 @@ def run_attention_case(reps):
     t_sc = _time(lambda: csr.csr_key_scores(D, Q, idx, coef, 1.0, scores=sc), reps)
     t_mx = _time(lambda: csr.csr_value_mix(D, W, idx, coef, out=out), reps)
     t_rc = _time(lambda: csr.csr_reconstruct_ex(D, idx.view(B * T, s), coef.view(B * T, s), X_hat=xh), reps)
+    t_da = _time(lambda: csr.csr_decode_attention(D, D, Q, idx, coef, idx, coef, 1.0 / d ** 0.5, weights=sc, out=out), reps)
     code_b, sw_b = B * T * s * 4.0, B * H * T * 4.0
     return {"case": "attention_from_codes", "B": B, "H": H, "T": T, "N": N, "d": d, "s": s,
             "key_scores_ms": round(t_sc, 4), "key_scores_hbm_gbs": (code_b + sw_b) / (t_sc * 1e-3) / 1e9,
             "value_mix_ms": round(t_mx, 4), "value_mix_hbm_gbs": (code_b + sw_b) / (t_mx * 1e-3) / 1e9,
-            "restore_to_bf16_ms": round(t_rc, 4), "restored_bytes": B * T * d * 2.0, "code_bytes": code_b}
+            "decode_attention_ms": round(t_da, 4), "restore_to_bf16_ms": round(t_rc, 4), "restored_bytes": B * T * d * 2.0, "code_bytes": code_b}
 
 
 def run_train_case(reps):
