@@ -93,7 +93,10 @@ def run_decode_case(seqs, kv_heads, N, s, reps):
     os.environ["CSR_EXACT_NO_SPLIT"] = "1"
     out["exact_row_tile_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, X, s, mode=csr.CSR_MODE_FP32_EXACT, out_idx=idx, out_coef=coef), 3)
     del os.environ["CSR_EXACT_NO_SPLIT"]
+    out["fast_cluster_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, Xb, s, out_idx=idx, out_coef=coef), reps)
+    os.environ["CSR_FAST_NO_CLUSTER"] = "1"
     out["fast_split_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, Xb, s, out_idx=idx, out_coef=coef), reps)
+    del os.environ["CSR_FAST_NO_CLUSTER"]
     os.environ["CSR_FAST_NO_SPLIT"] = "1"
     out["fast_one_launch_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, Xb, s, out_idx=idx, out_coef=coef), reps)
     del os.environ["CSR_FAST_NO_SPLIT"]

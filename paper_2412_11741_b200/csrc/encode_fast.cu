@@ -101,6 +101,37 @@ __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.p
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// ---- thread-block cluster: peers' shared memory and barriers ----
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t cta_rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(cta_rank));
+    return r;
+}
+// Eight bytes into a peer's shared memory; the peer's barrier is credited with them when they
+// have landed, so the reader needs nothing but to wait for its barrier.
+__device__ __forceinline__ void st_async_u64(uint32_t raddr, unsigned long long v, uint32_t rbar) {
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];" ::"r"(raddr), "l"(v),
+                 "r"(rbar)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Every thread of every CTA of the cluster (a lone CTA is a cluster of one).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
@@ -200,6 +231,9 @@ struct FastSmem {
     uint64_t acc_empty[2];
     uint64_t res_ready[2];
     uint64_t drained;
+    uint64_t xbar[2];                                  // cluster exchange: gathered / merged, one phase per iteration each
+    unsigned long long xin[2 * TILE_M];                // cluster exchange: (key, ~tile) of the rows this CTA merges, per source CTA
+    unsigned long long xout[2 * TILE_M];               // cluster exchange: merged (key, ~tile) of every row
     uint32_t tmem_base;
     volatile uint32_t abort;
 };
@@ -216,6 +250,22 @@ __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, con
     const unsigned long long t0 = globaltimer_ns();
     for (uint32_t it = 1; it < (1u << 28); ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0) {
+            if (*w.abort) return false;
+            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) break;
+        }
+    }
+    *w.abort = 1;
+    atomicOr(w.status, kStatusTimeout);
+    return false;
+}
+
+// The same wait on a barrier that other CTAs of the cluster arrive on.
+__device__ __forceinline__ bool wait_bounded_cluster(uint64_t* bar, uint32_t parity, const WaitCtx& w) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    for (uint32_t it = 1; it < (1u << 28); ++it) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
         if ((it & 63u) == 0) {
             if (*w.abort) return false;
             if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) break;
@@ -510,7 +560,7 @@ split_pick_kernel(const uint16_t* __restrict__ Db, int N, uint4* __restrict__ Rb
 // ---------------------------------------------------------------------------------------
 // the encoder
 // ---------------------------------------------------------------------------------------
-template <int D_, int G>
+template <int D_, int G, bool CL>
 __global__ void __launch_bounds__(NT, 1)
 encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* __restrict__ Db,
                    const void* __restrict__ X, int x_dtype, int64_t ldx, int64_t M, int N, int s,
@@ -525,8 +575,13 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
     const int T = (N + TILE_N - 1) / TILE_N;                // dictionary tiles per sweep (the last may be half)
     const int64_t n_pairs = (M + 2 * TILE_M - 1) / (2 * TILE_M);
     // Few rows (n_splits > 1): n_splits CTAs share one pair of row tiles, CTA j sweeping the
-    // dictionary tiles j, j + n_splits, ... of ONE iteration (s == 1 is passed) and leaving each
-    // row's best (key, tile) in `partial` for the pick kernel instead of picking itself.
+    // dictionary tiles j, j + n_splits, ...
+    //  - CL: the n_splits CTAs are one thread-block cluster and run all s iterations.
+    //    After each sweep every row's best (key, tile) is max-reduced into every CTA's shared
+    //    memory, every CTA then makes the same pick and the same residual update on its own
+    //    copy of the rows, and CTA 0 of the cluster writes the codes.
+    //  - otherwise ONE iteration per launch (s == 1 is passed): each row's best (key, tile) goes
+    //    to `partial` and the pick kernel takes over.
     const int t_begin = n_splits > 1 ? (int)(blockIdx.x % n_splits) : 0;
     const int t_step = n_splits > 1 ? n_splits : 1;
     const int64_t pair_first = n_splits > 1 ? blockIdx.x / n_splits : blockIdx.x;
@@ -548,6 +603,13 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             mbar_init(&sm.res_ready[t], TILE_M);
         }
         mbar_init(&sm.drained, 1);
+        if constexpr (CL) {
+            // one phase per iteration: this thread arms it with the bytes the peers will send
+            mbar_init(&sm.xbar[0], 1);
+            mbar_init(&sm.xbar[1], 1);
+            mbar_expect_tx(&sm.xbar[0], 2 * TILE_M * 8);
+            mbar_expect_tx(&sm.xbar[1], 2 * TILE_M * 8);
+        }
         sm.abort = 0;
         fence_barrier_init();
     }
@@ -559,6 +621,8 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sm.tmem_base;
+    // no CTA touches a peer's barrier or words before every peer has set them up
+    if constexpr (CL) cluster_sync_all();
 
     if (warp == PRODUCER_WARP) {
         // ------------------------------ TMA producer ------------------------------
@@ -654,7 +718,9 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         float (*code_coef)[CODE_BLOCK] = &sm.code_coef[tile * TILE_M];
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + tile * TILE_N;
         uint32_t accn = 0;
+        [[maybe_unused]] uint32_t xn = 0;
         bool ok = true;
+        const bool writes_codes = !CL || t_begin == 0;
         for (int64_t pair = pair_first; pair < n_pairs && ok; pair += pair_step) {
             const int64_t m = pair * (2 * TILE_M) + slot;
             const bool valid = m < M;
@@ -751,9 +817,53 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     }
                 }
                 if (!ok) break;
-                if (partial) {                              // split sweep: the pick kernel takes over
+                if (!CL && partial) {                       // split sweep: the pick kernel takes over
                     if (valid) partial[m * n_splits + t_begin] = make_uint2(best_key, best_t);
                     continue;
+                }
+                if constexpr (CL) {
+                    // ---- every CTA of the cluster learns the row's best over the whole dictionary:
+                    // the highest key and, among equal keys, the lowest tile.  Row i of the pair is
+                    // merged by CTA i % n_splits: gather there, merge, send the result to everyone.
+                    // Both buffers are single.  An entry of xin is overwritten by a peer that has
+                    // seen this iteration's merged rows from all of this CTA's merging threads,
+                    // each of which read its entries first; an entry of xout is overwritten by a
+                    // peer that has received the next iteration's key from the one thread that
+                    // reads it. ----
+                    const unsigned long long mine =
+                        (static_cast<unsigned long long>(best_key) << 32) | (0xFFFFFFFFu - best_t);
+                    const int per_cta = 2 * TILE_M / n_splits;        // rows merged by one CTA
+                    {
+                        const uint32_t o = static_cast<uint32_t>(slot % n_splits);
+                        st_async_u64(map_to_cta(smem_u32(&sm.xin[t_begin * per_cta + slot / n_splits]), o), mine,
+                                     map_to_cta(smem_u32(&sm.xbar[0]), o));
+                    }
+                    bool got = true;
+                    if (slot < per_cta) {
+                        got = wait_bounded_cluster(&sm.xbar[0], xn & 1, wc);
+                        if (got) {
+                            if (slot == 0) mbar_expect_tx(&sm.xbar[0], 2 * TILE_M * 8);       // the next iteration's
+                            unsigned long long top = 0ull;
+                            for (int c = 0; c < n_splits; ++c) {
+                                const unsigned long long v =
+                                    *reinterpret_cast<volatile unsigned long long*>(&sm.xin[c * per_cta + slot]);
+                                top = v > top ? v : top;
+                            }
+                            const uint32_t dst = smem_u32(&sm.xout[slot * n_splits + t_begin]), bar = smem_u32(&sm.xbar[1]);
+                            for (int c = 0; c < n_splits; ++c) st_async_u64(map_to_cta(dst, c), top, map_to_cta(bar, c));
+                        }
+                    }
+                    if (got) got = wait_bounded_cluster(&sm.xbar[1], xn & 1, wc);
+                    got = __all_sync(0xffffffffu, got);
+                    if (!got) {
+                        ok = false;
+                        break;
+                    }
+                    if (slot == 0) mbar_expect_tx(&sm.xbar[1], 2 * TILE_M * 8);               // the next iteration's
+                    const unsigned long long all = *reinterpret_cast<volatile unsigned long long*>(&sm.xout[slot]);
+                    ++xn;
+                    best_key = static_cast<uint32_t>(all >> 32);
+                    best_t = 0xFFFFFFFFu - static_cast<uint32_t>(all);
                 }
                 // ---- pick, signed coefficient, residual update ----
                 const int gi = g & (CODE_BLOCK - 1);
@@ -769,7 +879,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 }
                 __syncwarp();
                 // ---- flush the collected codes eight at a time ----
-                if ((gi == CODE_BLOCK - 1 || g == s - 1) && valid) {
+                if ((gi == CODE_BLOCK - 1 || g == s - 1) && valid && writes_codes) {
                     const int g0 = g - gi;
                     const int64_t o = m * ldc + g0;
                     if (gi == CODE_BLOCK - 1 && vec_codes) {
@@ -812,6 +922,8 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+    // a CTA's shared memory must outlive its peers' last writes to it
+    if constexpr (CL) cluster_sync_all();
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -831,11 +943,57 @@ EncodeTiledFn get_encode_tiled() {
 }
 
 template <int D_, int G>
+void cluster_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int cluster_ctas, int grid, size_t smem,
+                    cudaStream_t stream) {
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(NT, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster_ctas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+}
+
+// How many clusters of `cluster_ctas` CTAs of the encoder the device holds at once (0: none,
+// or clusters of that size cannot be launched here).  Asked once per size.
+template <int D_, int G>
+int max_clusters(int cluster_ctas) {
+    static int cached[17] = {0};                       // 0 = not asked yet, -1 = none
+    if (cluster_ctas < 2 || cluster_ctas > 16) return 0;
+    if (cached[cluster_ctas] == 0) {
+        const size_t smem = sizeof(FastSmem<D_>) + 1024;
+        int n = 0;
+        bool good = cudaFuncSetAttribute(encode_fast_kernel<D_, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem) == cudaSuccess;
+        if (good && cluster_ctas > 8)
+            good = cudaFuncSetAttribute(encode_fast_kernel<D_, G, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
+                   cudaSuccess;
+        if (good) {
+            cudaLaunchConfig_t cfg = {};
+            cudaLaunchAttribute attr[1];
+            cluster_config<D_, G>(cfg, attr, cluster_ctas, cluster_ctas, smem, 0);
+            good = cudaOccupancyMaxActiveClusters(&n, encode_fast_kernel<D_, G, true>, &cfg) == cudaSuccess;
+        }
+        if (!good) {
+            cudaGetLastError();                        // a refusal is an answer, not a failure of the call
+            n = 0;
+        }
+        cached[cluster_ctas] = n > 0 ? n : -1;
+    }
+    return cached[cluster_ctas] > 0 ? cached[cluster_ctas] : 0;
+}
+
+template <int D_, int G>
 int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, int n_splits,
-           uint2* partial) {
+           uint2* partial, int cluster_grid = 0) {
     const size_t smem = sizeof(FastSmem<D_>) + 1024;
     cudaError_t e =
-        cudaFuncSetAttribute(encode_fast_kernel<D_, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cluster_grid > 0
+            ? cudaFuncSetAttribute(encode_fast_kernel<D_, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+            : cudaFuncSetAttribute(encode_fast_kernel<D_, G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     const int64_t n_pairs = (a.M + 2 * TILE_M - 1) / (2 * TILE_M);
     const int grid = n_splits > 1 ? (int)(n_pairs * n_splits)
@@ -846,7 +1004,18 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
     // 16-byte code stores need eight codes per flush and 16-byte aligned rows in both arrays
     const uintptr_t ci = reinterpret_cast<uintptr_t>(a.out_idx), cc = reinterpret_cast<uintptr_t>(a.out_coef);
     const int vec_codes = (a.s % 8 == 0) && (a.ld_code % 8 == 0) && (ci % 16 == 0) && (cc % 16 == 0);
-    encode_fast_kernel<D_, G><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
+    if (cluster_grid > 0) {
+        // n_splits CTAs per cluster, cluster_grid CTAs in all
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        cluster_config<D_, G>(cfg, attr, n_splits, cluster_grid, smem, a.stream);
+        e = cudaLaunchKernelEx(&cfg, encode_fast_kernel<D_, G, true>, tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
+                               a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask, status, n_splits,
+                               static_cast<uint2*>(nullptr));
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "encode_fast cluster launch: %s", cudaGetErrorString(e));
+        return CSR_OK;
+    }
+    encode_fast_kernel<D_, G, false><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
                                                            a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask,
                                                            status, n_splits, partial);
     e = cudaGetLastError();
@@ -875,6 +1044,59 @@ int launch_d(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, u
         case 2: return launch<D_, 2>(a, tmap, Db, status, 0, nullptr);
         case 8: return launch<D_, 8>(a, tmap, Db, status, 0, nullptr);
         default: return launch<D_, 4>(a, tmap, Db, status, 0, nullptr);
+    }
+}
+
+// Few rows, one launch: clusters of CTAs share a pair of row tiles.  Picks the cluster size
+// whose modelled time per iteration (about 1.6 us per 256-atom tile swept plus about 3.5 us
+// for the exchange and the pick, over as many rounds as the device needs to hold all pairs)
+// is lowest, and returns 0 when one CTA per pair over the whole dictionary (about 1.55 us
+// per tile, measured) is no slower.  *grid gets the CTAs to launch.
+template <int D_, int G>
+int cluster_split(int64_t M, int N, int* grid) {
+    const int64_t n_pairs = (M + 2 * TILE_M - 1) / (2 * TILE_M);
+    const int T = (N + TILE_N - 1) / TILE_N;
+    if (n_pairs < 1 || T < 2) return 0;
+    float best = 0.f;
+    int best_ns = 0;
+    for (int ns = 16; ns >= 2; ns >>= 1) {
+        if (ns > T) continue;
+        const int nc = max_clusters<D_, G>(ns);
+        if (nc < 1) continue;
+        const int64_t rounds = (n_pairs + nc - 1) / nc;
+        const float est = (float)rounds * (1.6f * ((T + ns - 1) / ns) + 3.5f);
+        if (best_ns == 0 || est < best) {
+            best = est;
+            best_ns = ns;
+            *grid = (int)(n_pairs < nc ? n_pairs : nc) * ns;
+        }
+    }
+    if (best_ns == 0) return 0;
+    const int64_t whole_rounds = (n_pairs + sm_count() - 1) / sm_count();
+    return (float)whole_rounds * 1.55f * T > 1.15f * best ? best_ns : 0;
+}
+
+template <int D_>
+int launch_clustered(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, bool* done) {
+    int grid = 0, ns = 0;
+    *done = false;
+    switch (group_size(D_, a.N)) {
+        case 1:
+            if ((ns = cluster_split<D_, 1>(a.M, a.N, &grid)) == 0) return CSR_OK;
+            *done = true;
+            return launch<D_, 1>(a, tmap, Db, status, ns, nullptr, grid);
+        case 2:
+            if ((ns = cluster_split<D_, 2>(a.M, a.N, &grid)) == 0) return CSR_OK;
+            *done = true;
+            return launch<D_, 2>(a, tmap, Db, status, ns, nullptr, grid);
+        case 8:
+            if ((ns = cluster_split<D_, 8>(a.M, a.N, &grid)) == 0) return CSR_OK;
+            *done = true;
+            return launch<D_, 8>(a, tmap, Db, status, ns, nullptr, grid);
+        default:
+            if ((ns = cluster_split<D_, 4>(a.M, a.N, &grid)) == 0) return CSR_OK;
+            *done = true;
+            return launch<D_, 4>(a, tmap, Db, status, ns, nullptr, grid);
     }
 }
 
@@ -985,6 +1207,14 @@ int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint
     if (r != CUDA_SUCCESS) return fail(CSR_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
 
     const uint16_t* Db = static_cast<const uint16_t*>(workspace);
+    // few rows: one launch of CTA clusters that share the dictionary (needs no scratch) ...
+    if (!getenv("CSR_FAST_NO_SPLIT") && !getenv("CSR_FAST_NO_CLUSTER")) {
+        bool done = false;
+        const int rc = a.d == 128 ? launch_clustered<128>(a, tmap, Db, status, &done)
+                                  : launch_clustered<64>(a, tmap, Db, status, &done);
+        if (rc != CSR_OK || done) return rc;
+    }
+    // ... else, with scratch, a sweep launch and a pick launch per iteration
     if (split_scratch) {
         if (a.d == 128) return run_split<128>(a, tmap, Db, status, split_scratch);
         return run_split<64>(a, tmap, Db, status, split_scratch);

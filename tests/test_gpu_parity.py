@@ -236,11 +236,15 @@ def test_fast_any_dictionary_size(csr, N, G, monkeypatch):
 @pytest.mark.parametrize("M,N,d,s,kind", [(1, 8192, 128, 16, "bf16"), (128, 8192, 128, 16, "bf16"), (300, 1000, 128, 5, "f32"),
                                           (2000, 4096, 64, 8, "f16"), (9000, 2048, 128, 4, "bf16"), (16, 65536, 64, 3, "bf16")])
 def test_fast_few_rows_split_dictionary_path(csr, M, N, d, s, kind, monkeypatch):
-    """Few rows: the dictionary is split across CTAs, one sweep and one pick launch per
-    iteration.  The codes must be those of the one-launch kernel bit for bit."""
+    """Few rows: the dictionary is split across the CTAs of a cluster (one launch) or, without
+    clusters, across CTAs with one sweep and one pick launch per iteration.  Both must return
+    the codes of the one-CTA-per-row-pair kernel bit for bit."""
     rng = np.random.default_rng(M * 7 + N)
     D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
     X = rng.standard_normal((M, d)).astype(np.float32)
+    if N >= 1024:
+        D[512 + 3] = D[3]                # the same atom at the same place of two 256-atom tiles: equal keys,
+        X[0] = 3.0 * D[3] + 0.05 * X[0]  # and a row whose first pick it is: the lower index must win
     X = wl.round_to_bf16(X) if kind == "bf16" else X.astype(np.float16).astype(np.float32) if kind == "f16" else X
     if M > 2:
         X[1] = 0.0
@@ -248,13 +252,20 @@ def test_fast_few_rows_split_dictionary_path(csr, M, N, d, s, kind, monkeypatch)
     Xd = torch.from_numpy(X).to(DEV).to({"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[kind])
     i1, c1 = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float32)
     assert csr.csr_device_status() == csr.CSR_OK
+    if N >= 1024:
+        assert int(_np_idx(i1)[0, 0]) == 3
     h = csr.csr_dict_create(Dd)
     i3, c3 = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float16, dict=h)       # handle + packed coefficients
     csr.csr_dict_destroy(h)
+    monkeypatch.setenv("CSR_FAST_NO_CLUSTER", "1")                # the launch-per-iteration split
+    i4, c4 = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float32)
+    monkeypatch.delenv("CSR_FAST_NO_CLUSTER")
+    assert csr.csr_device_status() == csr.CSR_OK
     monkeypatch.setenv("CSR_FAST_NO_SPLIT", "1")
     i2, c2 = csr.csr_encode_ex(Dd, Xd, s, coef_dtype=torch.float32)
     monkeypatch.delenv("CSR_FAST_NO_SPLIT")
     assert np.array_equal(_np_idx(i1), _np_idx(i2)) and torch.equal(c1, c2)
+    assert np.array_equal(_np_idx(i4), _np_idx(i2)) and torch.equal(c4, c2)
     assert np.array_equal(_np_idx(i3), _np_idx(i2)) and torch.equal(c3, c2.to(torch.float16))
     if N >= 1000 and M >= 100:
         rep = parity.compare_fast(D, wl.round_to_bf16(X), s, _np_idx(i1), c1.cpu().numpy())
