@@ -73,10 +73,13 @@ extern "C" {
  *                        reconstruction error does not, down to a floor of about
  *                        2^-8 * ||x|| (the residual is carried in bf16); use the exact
  *                        mode for errors below 1e-2 * ||x||.  With few rows (at most half
- *                        as many pairs of 128-row tiles as SMs) and the library-owned
- *                        scratch, the dictionary is split across the SMs, one sweep and
- *                        one pick launch per iteration, with identical codes (off when
- *                        the environment variable CSR_FAST_NO_SPLIT is set).  The variable
+ *                        as many pairs of 128-row tiles as SMs) the dictionary is split
+ *                        across the CTAs of thread-block clusters that share the rows,
+ *                        still one launch, with identical codes; where clusters cannot be
+ *                        launched (or CSR_FAST_NO_CLUSTER is set) and the library-owned
+ *                        scratch is in use, across CTAs with one sweep and one pick launch
+ *                        per iteration (both off when the environment variable
+ *                        CSR_FAST_NO_SPLIT is set).  The variable
  *                        CSR_FAST_GROUP (1, 2, 4 or 8) overrides the arg-max group size
  *                        the kernel would choose; every setting meets the same gates.
  */

@@ -46,9 +46,11 @@ int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status);
 size_t encode_fast_workspace_bytes(int d, int N);
 // The two halves of launch_encode_fast: build the bf16 copy once, encode against it many times.
 int prepare_fast_dictionary(const float* D, int N, int d, void* workspace, cudaStream_t stream);
-// With `split_scratch` (encode_fast_split_scratch_bytes(), 256-byte aligned) and few rows the
-// dictionary is split across CTAs, one sweep launch and one pick launch per iteration, with
-// identical codes; NULL = one launch for the whole job.
+// With few rows the dictionary is split across the CTAs of thread-block clusters (one launch,
+// no scratch).  Where clusters cannot be launched, `split_scratch`
+// (encode_fast_split_scratch_bytes(), 256-byte aligned) lets it be split across CTAs with one
+// sweep launch and one pick launch per iteration; NULL = one CTA per pair of row tiles over
+// the whole dictionary.  Identical codes in all three.
 int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint32_t* status, void* split_scratch);
 bool encode_fast_split_applies(int64_t M, int N);
 size_t encode_fast_split_scratch_bytes(int64_t M, int d, int N);

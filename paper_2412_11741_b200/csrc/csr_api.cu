@@ -265,8 +265,9 @@ int encode_device(const csr_encode_params_t* p) {
         return launch_encode_exact(a);
     }
 
-    // few rows: library-owned scratch lets the dictionary be split across the SMs (a caller
-    // workspace is sized for the bf16 copy only, so with one the whole-job kernel runs)
+    // few rows: the cluster path needs no scratch; its fallback (a launch pair per iteration)
+    // does, and gets it from the library-owned buffer only (a caller workspace is sized for
+    // the bf16 copy)
     const bool split = !p->workspace && encode_fast_split_applies(p->M, p->N) && !getenv("CSR_FAST_NO_SPLIT");
     const size_t dict_b = (encode_fast_workspace_bytes(p->d, p->N) + 1023) / 1024 * 1024;
     const size_t split_b = split ? encode_fast_split_scratch_bytes(p->M, p->d, p->N) : 0;

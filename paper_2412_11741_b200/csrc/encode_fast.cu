@@ -367,17 +367,22 @@ __device__ __forceinline__ uint4 axpy8(const uint4& rv, const uint4& av, float c
 // in magnitude (lowest atom on ties) gives the index and the coefficient, and, unless
 // this was the last iteration, the residual row in the operand tile becomes
 // R - coef * atom.  The code goes to the row's slot in the shared-memory staging arrays.
-template <int D_, int G>
+// With SKIP, groups of (at most four) passes none of whose rows is set in `row_mask` (bit i =
+// row i of the warp's 32 is a row of X) are left out: with few rows the pick is on the
+// critical path of every iteration.
+template <int D_, int G, bool SKIP = false>
 __device__ __forceinline__ void pick_and_update(uint8_t* Atile, int q, int lane, const uint16_t* __restrict__ Db,
                                                 int n0, bool update, uint16_t (*code_idx)[CODE_BLOCK],
-                                                float (*code_coef)[CODE_BLOCK], int gi) {
+                                                float (*code_coef)[CODE_BLOCK], int gi, uint32_t row_mask = 0xffffffffu) {
     constexpr int CH = D_ / 64;                           // 16-byte chunks per lane per atom
     constexpr int APR = D_ / 8;                           // 16-byte chunks per atom row
     constexpr int LPP = G * CH;                           // gathered chunks per lane per pass
-    constexpr int WAVE = (32 / LPP) < 8 ? (32 / LPP) : 8; // passes whose gathers are in flight together
+    constexpr int WAVE0 = (32 / LPP) < 8 ? (32 / LPP) : 8;
+    constexpr int WAVE = SKIP && WAVE0 > 4 ? 4 : WAVE0;   // passes whose gathers are in flight together
     const int sub = lane >> 3, l8 = lane & 7;
 #pragma unroll
     for (int w0 = 0; w0 < 8; w0 += WAVE) {
+        if (SKIP && ((row_mask >> (w0 * 4)) & ((1ull << (4 * WAVE)) - 1)) == 0) continue;
         uint4 atom[WAVE][G][CH];
         int base[WAVE];
 #pragma unroll
@@ -724,6 +729,8 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         for (int64_t pair = pair_first; pair < n_pairs && ok; pair += pair_step) {
             const int64_t m = pair * (2 * TILE_M) + slot;
             const bool valid = m < M;
+            uint32_t row_mask = 0xffffffffu;
+            if constexpr (CL) row_mask = __ballot_sync(0xffffffffu, valid);
             // ---- R_0 = x, rounded to bf16, into the operand tile ----
             if (x_dtype == CSR_DTYPE_BF16) {
                 const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(X) + m * ldx);
@@ -872,7 +879,10 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 const int n0 = min(static_cast<int>(best_t) * TILE_N +
                                        (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G,
                                    ((N + 7) / 8) * 8 - G);
-                pick_and_update<D_, G>(Atile, q, lane, Db, n0, g + 1 < s, code_idx, code_coef, gi);
+                if constexpr (CL)
+                    pick_and_update<D_, G, true>(Atile, q, lane, Db, n0, g + 1 < s, code_idx, code_coef, gi, row_mask);
+                else
+                    pick_and_update<D_, G>(Atile, q, lane, Db, n0, g + 1 < s, code_idx, code_coef, gi);
                 if (g + 1 < s) {
                     fence_proxy_async_smem();
                     mbar_arrive(&sm.res_ready[tile]);
