@@ -1061,9 +1061,10 @@ int launch_d(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, u
 // whose modelled time per iteration (about 1.6 us per 256-atom tile swept plus about 3.5 us
 // for the exchange and the pick, over as many rounds as the device needs to hold all pairs)
 // is lowest, and returns 0 when one CTA per pair over the whole dictionary (about 1.55 us
-// per tile, measured) is no slower.  *grid gets the CTAs to launch.
+// per tile, measured) is no slower, or when the estimate exceeds `budget_us` (what another
+// path is expected to take).  *grid gets the CTAs to launch.
 template <int D_, int G>
-int cluster_split(int64_t M, int N, int* grid) {
+int cluster_split(int64_t M, int N, float budget_us, int* grid) {
     const int64_t n_pairs = (M + 2 * TILE_M - 1) / (2 * TILE_M);
     const int T = (N + TILE_N - 1) / TILE_N;
     if (n_pairs < 1 || T < 2) return 0;
@@ -1081,37 +1082,39 @@ int cluster_split(int64_t M, int N, int* grid) {
             *grid = (int)(n_pairs < nc ? n_pairs : nc) * ns;
         }
     }
-    if (best_ns == 0) return 0;
+    if (best_ns == 0 || best > budget_us) return 0;
     const int64_t whole_rounds = (n_pairs + sm_count() - 1) / sm_count();
     return (float)whole_rounds * 1.55f * T > 1.15f * best ? best_ns : 0;
 }
 
 template <int D_>
-int launch_clustered(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, bool* done) {
+int launch_clustered(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, float budget_us,
+                     bool* done) {
     int grid = 0, ns = 0;
     *done = false;
     switch (group_size(D_, a.N)) {
         case 1:
-            if ((ns = cluster_split<D_, 1>(a.M, a.N, &grid)) == 0) return CSR_OK;
+            if ((ns = cluster_split<D_, 1>(a.M, a.N, budget_us, &grid)) == 0) return CSR_OK;
             *done = true;
             return launch<D_, 1>(a, tmap, Db, status, ns, nullptr, grid);
         case 2:
-            if ((ns = cluster_split<D_, 2>(a.M, a.N, &grid)) == 0) return CSR_OK;
+            if ((ns = cluster_split<D_, 2>(a.M, a.N, budget_us, &grid)) == 0) return CSR_OK;
             *done = true;
             return launch<D_, 2>(a, tmap, Db, status, ns, nullptr, grid);
         case 8:
-            if ((ns = cluster_split<D_, 8>(a.M, a.N, &grid)) == 0) return CSR_OK;
+            if ((ns = cluster_split<D_, 8>(a.M, a.N, budget_us, &grid)) == 0) return CSR_OK;
             *done = true;
             return launch<D_, 8>(a, tmap, Db, status, ns, nullptr, grid);
         default:
-            if ((ns = cluster_split<D_, 4>(a.M, a.N, &grid)) == 0) return CSR_OK;
+            if ((ns = cluster_split<D_, 4>(a.M, a.N, budget_us, &grid)) == 0) return CSR_OK;
             *done = true;
             return launch<D_, 4>(a, tmap, Db, status, ns, nullptr, grid);
     }
 }
 
-// Few rows: how many CTAs share a pair of row tiles (1 = the whole dictionary per CTA).
-int split_count(int64_t M, int N) {
+// Few rows: how many CTAs share a pair of row tiles (1 = the whole dictionary per CTA);
+// *per_iter_us gets the modelled time of one iteration.
+int split_count(int64_t M, int N, float* per_iter_us = nullptr) {
     const int64_t n_pairs = (M + 2 * TILE_M - 1) / (2 * TILE_M);
     const int T = (N + TILE_N - 1) / TILE_N;
     if (n_pairs < 1 || n_pairs * 2 > sm_count() || T < 2) return 1;
@@ -1120,8 +1123,9 @@ int split_count(int64_t M, int N) {
     if (ns > 32) ns = 32;
     // Worth it only if an iteration's sweep over all T tiles by one CTA (about 1.55 us per
     // tile, measured) outlasts two launches (about 12 us) plus the sweep of a slice.
-    const float whole = 1.55f * T, sliced = 1.2f * (12.f + 1.6f * ((T + ns - 1) / ns));
-    return whole > sliced ? ns : 1;
+    const float whole = 1.55f * T, sliced = 12.f + 1.6f * ((T + ns - 1) / ns);
+    if (per_iter_us) *per_iter_us = sliced;
+    return whole > 1.2f * sliced ? ns : 1;
 }
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
@@ -1218,10 +1222,14 @@ int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint
 
     const uint16_t* Db = static_cast<const uint16_t*>(workspace);
     // few rows: one launch of CTA clusters that share the dictionary (needs no scratch) ...
+    // (unless the launch-per-iteration split below, which can spread a pair of row tiles over more
+    // than 16 CTAs, is expected to be faster: very large dictionaries)
     if (!getenv("CSR_FAST_NO_SPLIT") && !getenv("CSR_FAST_NO_CLUSTER")) {
+        float budget = 3.0e38f;
+        if (split_scratch && split_count(a.M, a.N, &budget) <= 1) budget = 3.0e38f;
         bool done = false;
-        const int rc = a.d == 128 ? launch_clustered<128>(a, tmap, Db, status, &done)
-                                  : launch_clustered<64>(a, tmap, Db, status, &done);
+        const int rc = a.d == 128 ? launch_clustered<128>(a, tmap, Db, status, budget, &done)
+                                  : launch_clustered<64>(a, tmap, Db, status, budget, &done);
         if (rc != CSR_OK || done) return rc;
     }
     // ... else, with scratch, a sweep launch and a pick launch per iteration
