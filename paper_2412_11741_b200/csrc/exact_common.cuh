@@ -46,63 +46,47 @@ __device__ __forceinline__ void top2_merge(Top2& t, float ob, float os, int oi) 
     t.second = sec;
 }
 
+// The same bookkeeping without branches (NaN values count as ties and send the row to the
+// fp64 re-scoring instead of being skipped).
+__device__ __forceinline__ void top2_push_fast(Top2& t, float a, int n) {
+    t.second = fmaxf(t.second, fminf(a, t.best));
+    const bool p = a > t.best;
+    t.best = fmaxf(a, t.best);
+    t.idx = p ? n : t.idx;
+}
+
 // Sweep of dictionary tiles [bt0, bt1) (128 atoms each) for the 64 rows whose fp32 residual
 // sits transposed in As (Eq. 2-3): fp32 register-tiled products, each thread 4 rows x 8
 // atoms, k ascending; every thread keeps the two largest |correlations| of its rows.
-// Bs is the double-buffered staging area of dictionary chunks.  Ends with a __syncthreads.
+// Bs is the double-buffered staging area of dictionary chunks (8 channels each; the next
+// chunk waits in registers while the current one is used).  Ends with a __syncthreads.
 template <int D_>
 __device__ __forceinline__ void sweep_tiles(const float* __restrict__ D, int N, int bt0, int bt1,
                                             const float (*As)[AS_LD], float (*Bs)[BK][BS_LD], Top2 (&top)[4]) {
-    constexpr int KCH = D_ / BK;
+    static_assert(BK == 8 && NT == 2 * BN, "two threads stage one atom's eight channels");
+    constexpr int KCH = D_ / BK;                          // chunks per tile (even)
     const int tid = threadIdx.x;
     const int tx = tid & 15;   // atom group
     const int ty = tid >> 4;   // row group: rows ty*4 .. ty*4+3
-    const int total_chunks = (bt1 - bt0) * KCH;
-    if (total_chunks <= 0) return;
-    constexpr int KQ = BK / 4;                            // float4 per atom per chunk
-    constexpr int FPT = BN * KQ / NT;                     // float4 staged per thread
-    float4 stage[FPT];
-    auto gload = [&](int chunk) {
-        const int bt = bt0 + chunk / KCH, kc = chunk % KCH;
-#pragma unroll
-        for (int i = 0; i < FPT; ++i) {
-            const int f = tid + i * NT;
-            const int atom = f / KQ, kq = f % KQ;
-            const int n = bt * BN + atom;
-            stage[i] = (n < N) ? *reinterpret_cast<const float4*>(D + (int64_t)n * D_ + kc * BK + kq * 4)
-                               : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+    if (bt1 <= bt0) return;
+    const int satom = tid >> 1, skq = (tid & 1) * 4;       // staged: channels skq .. skq+3 of atom satom
+    float4 stage;
+    auto gload = [&](const float* src, bool in_range) {
+        stage = in_range ? *reinterpret_cast<const float4*>(src) : make_float4(0.f, 0.f, 0.f, 0.f);
     };
-    auto sstore = [&](int buf) {
-#pragma unroll
-        for (int i = 0; i < FPT; ++i) {
-            const int f = tid + i * NT;
-            const int atom = f / KQ, kq = f % KQ;
-            Bs[buf][kq * 4 + 0][atom] = stage[i].x;
-            Bs[buf][kq * 4 + 1][atom] = stage[i].y;
-            Bs[buf][kq * 4 + 2][atom] = stage[i].z;
-            Bs[buf][kq * 4 + 3][atom] = stage[i].w;
-        }
+    auto sstore = [&](float (*B)[BS_LD]) {
+        B[skq + 0][satom] = stage.x;
+        B[skq + 1][satom] = stage.y;
+        B[skq + 2][satom] = stage.z;
+        B[skq + 3][satom] = stage.w;
     };
-    gload(0);
-    sstore(0);
-    __syncthreads();
     float acc[4][8];
-    for (int chunk = 0; chunk < total_chunks; ++chunk) {
-        const int buf = chunk & 1;
-        const int kc = chunk % KCH;
-        if (kc == 0) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
-        }
-        if (chunk + 1 < total_chunks) gload(chunk + 1);
+    auto compute8 = [&](const float (*B)[BS_LD], const float (*A)[AS_LD]) {
 #pragma unroll
         for (int k = 0; k < BK; ++k) {
-            const float4 a4 = *reinterpret_cast<const float4*>(&As[kc * BK + k][ty * 4]);
-            const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
-            const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][k][64 + tx * 4]);
+            const float4 a4 = *reinterpret_cast<const float4*>(&A[k][ty * 4]);
+            const float4 b0 = *reinterpret_cast<const float4*>(&B[k][tx * 4]);
+            const float4 b1 = *reinterpret_cast<const float4*>(&B[k][64 + tx * 4]);
             const float a[4] = {a4.x, a4.y, a4.z, a4.w};
             const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
@@ -110,19 +94,56 @@ __device__ __forceinline__ void sweep_tiles(const float* __restrict__ D, int N, 
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
         }
-        if (kc == KCH - 1) {
-            const int nb = (bt0 + chunk / KCH) * BN;
+    };
+    const float* src = D + ((int64_t)bt0 * BN + satom) * D_ + skq;
+    bool in_range = bt0 * BN + satom < N;
+    gload(src, in_range);
+    sstore(Bs[0]);
+    __syncthreads();
+    for (int bt = bt0; bt < bt1; ++bt) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+        const bool last_tile = bt + 1 == bt1;
+#pragma unroll 1
+        for (int c = 0; c < KCH; c += 2) {
+            // here: Bs[0] holds chunk c of the tile
+            src += BK;
+            gload(src, in_range);                         // chunk c + 1 (KCH is even)
+            compute8(Bs[0], As + c * BK);
+            sstore(Bs[1]);
+            __syncthreads();
+            const bool more = !(last_tile && c + 2 == KCH);
+            if (more) {                                   // chunk c + 2, or the next tile's first
+                if (c + 2 == KCH) {
+                    src += (int64_t)BN * D_ - (KCH - 1) * BK;
+                    in_range = (bt + 1) * BN + satom < N;
+                } else {
+                    src += BK;
+                }
+                gload(src, in_range);
+            }
+            compute8(Bs[1], As + (c + 1) * BK);
+            if (more) sstore(Bs[0]);
+            __syncthreads();
+        }
+        const int nb = bt * BN + tx * 4;
+        if ((bt + 1) * BN <= N) {                         // a whole tile: no atom to leave out
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) top2_push_fast(top[i], fabsf(acc[i][j]), nb + (j >> 2) * 64 + (j & 3));
+        } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const int n = nb + (j < 4 ? tx * 4 + j : 64 + tx * 4 + (j - 4));
+                const int n = nb + (j >> 2) * 64 + (j & 3);
                 if (n < N) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) top2_push(top[i], fabsf(acc[i][j]), n);
+                    for (int i = 0; i < 4; ++i) top2_push_fast(top[i], fabsf(acc[i][j]), n);
                 }
             }
         }
-        if (chunk + 1 < total_chunks) sstore(buf ^ 1);
-        __syncthreads();
     }
 }
 
