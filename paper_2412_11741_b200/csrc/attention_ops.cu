@@ -9,14 +9,17 @@
 // or weight) instead of the 2*d bytes of a restored bf16 row written and read again.
 //
 // key_scores: (1) p = scale * Q D^T for all B*H query heads, a small fp32 GEMM written to a
-// scratch array [B*H][N] (channels summed in ascending order); (2) one CTA per (code stream,
-// token range) copies its heads' rows of p into shared memory, streams the codes, one
-// thread per token, and sums the s terms in stored order.
-// value_mix: (1) one CTA per (code stream, token range) scatters w * coef into a[head][N] in
-// shared memory with atomic adds while it streams the codes and then adds its a to the
-// scratch array [B*H][N] with global atomic adds; (2) out = a D, a small fp32 GEMM (split
-// over atoms with atomic adds when there are few heads).  Atomic fp32 adds make value_mix
-// reproducible only to rounding.
+// scratch array [B][N][H] (a stream's heads side by side per atom; channels summed in
+// ascending order); (2) one CTA per (code stream, token range) copies its heads' part of p
+// into shared memory, streams the codes, one thread per token, and sums the s terms in
+// stored order.
+// value_mix: (1) every code stream is cut into `pieces` token ranges, one CTA each, which
+// scatters w * coef into a[head][N] in shared memory with atomic adds while it streams the
+// codes and then stores its a to the scratch array [B][pieces][H][N]; (2) out = a D with the
+// pieces summed in order on the way in, a small fp32 GEMM (split over atoms with atomic
+// adds when there are few heads).  The tables are accumulated in fixed point (see
+// value_scatter_kernel) and are the same on every run; the split over atoms of step (2),
+// when it is used, still adds in an order that varies.
 #include "common.cuh"
 
 namespace csr {
@@ -31,7 +34,7 @@ __device__ __forceinline__ float load_coef(const void* coef, int coef_dtype, int
 }
 __device__ __forceinline__ float load_q(const void* Q, int q_dtype, int64_t off) { return load_elem(Q, q_dtype, off); }
 
-// ---- P[r][n] = scale * Q[r][:] . D[n][:]  (r = b*H + h) -----------------------------------
+// ---- P[b][n][h] = scale * Q[r][:] . D[n][:]  (r = b*H + h) --------------------------------
 // CTA = 64 atoms x 64 rows; thread = 4 rows x 4 atoms; channels staged 32 at a time,
 // transposed, and summed in ascending order.
 constexpr int PA = 64;    // atoms per CTA
@@ -39,7 +42,7 @@ constexpr int QROWS = 64; // rows per CTA (grid.y)
 constexpr int PK = 32;    // channels per staged block
 template <int D_>
 __global__ void __launch_bounds__(NT)
-qd_kernel(const float* __restrict__ D, int N, const void* __restrict__ Q, int q_dtype, int R, float scale,
+qd_kernel(const float* __restrict__ D, int N, const void* __restrict__ Q, int q_dtype, int R, int H, float scale,
           float* __restrict__ P) {
     __shared__ __align__(16) float Ds[PK][PA + 4];         // Ds[k][atom]
     __shared__ __align__(16) float Qs[PK][QROWS + 4];      // Qs[k][row]
@@ -79,19 +82,19 @@ qd_kernel(const float* __restrict__ D, int N, const void* __restrict__ Q, int q_
         if (r < R) {
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (n0 + ta + j < N) P[(int64_t)r * N + n0 + ta + j] = scale * acc[i][j];
+                if (n0 + ta + j < N) P[((int64_t)(r / H) * N + n0 + ta + j) * H + r % H] = scale * acc[i][j];
         }
     }
 }
 
-// ---- out[r][:] (+)= sum_{n in slice} A[r][n] * D[n][:] ------------------------------------
+// ---- out[r][:] (+)= sum_{n in slice} (sum_pieces A[b][piece][h][n]) * D[n][:] ---------------
 // CTA = 16 rows x one atom slice; thread = (channel, group of rows).
 constexpr int OR = 16;    // rows per CTA
 constexpr int OA = 64;    // atoms per staged block
 template <int D_>
 __global__ void __launch_bounds__(NT)
-ad_kernel(const float* __restrict__ D, int N, const float* __restrict__ A, int R, int atoms_per_slice, int use_atomics,
-          float* __restrict__ out) {
+ad_kernel(const float* __restrict__ D, int N, const float* __restrict__ A, int R, int H, int pieces, int atoms_per_slice,
+          int use_atomics, float* __restrict__ out) {
     __shared__ float Ds[OA][D_];
     __shared__ __align__(16) float As[OR][OA];
     constexpr int RG = NT / D_;            // row groups (2 or 4)
@@ -111,7 +114,12 @@ ad_kernel(const float* __restrict__ D, int N, const float* __restrict__ A, int R
         }
         for (int f = threadIdx.x; f < OR * OA; f += NT) {
             const int r = f / OA, a = f % OA;
-            As[r][a] = (r0 + r < R && n0 + a < ne) ? A[(int64_t)(r0 + r) * N + n0 + a] : 0.f;
+            float v = 0.f;
+            if (r0 + r < R && n0 + a < ne) {                // row (b, h): the stream's pieces in order
+                const int64_t bb = (r0 + r) / H, hh = (r0 + r) % H;
+                for (int pc = 0; pc < pieces; ++pc) v += A[((bb * pieces + pc) * H + hh) * N + n0 + a];
+            }
+            As[r][a] = v;
         }
         __syncthreads();
         for (int a = 0; a < OA; a += 4) {
@@ -226,8 +234,19 @@ key_scores_kernel(const float* __restrict__ P, int N, int B, int H, const uint16
             const int b = (int)(w / chunks_per_b);
             if (b != cur_b) {
                 __syncthreads();
-                const float* src = P + ((int64_t)b * H + h0) * N;
-                for (int j = threadIdx.x; j < hg * N; j += NTS) tab[(j % N) * HGP + j / N] = src[j];
+                const float* src = P + (int64_t)b * N * H;           // [N][H]
+                if (HGP == H && HGP >= 4) {                          // the whole stream's table, as it lies
+                    const float4* s4 = reinterpret_cast<const float4*>(src);
+                    float4* t4 = reinterpret_cast<float4*>(tab);
+                    const int n4 = N * HGP / 4;
+#pragma unroll 8
+                    for (int j = threadIdx.x; j < n4; j += NTS) t4[j] = s4[j];
+                } else {
+                    for (int j = threadIdx.x; j < N * HGP; j += NTS) {
+                        const int n = j / HGP, h = j % HGP;
+                        tab[j] = h < hg ? src[(int64_t)n * H + h0 + h] : 0.f;
+                    }
+                }
                 __syncthreads();
                 cur_b = b;
             }
@@ -248,48 +267,119 @@ key_scores_kernel(const float* __restrict__ P, int N, int B, int H, const uint16
     }
 }
 
+// Block-wide maximum / sum of one value per thread (NTS threads), returned to every thread;
+// the order of the additions is fixed.
+__device__ __forceinline__ float block_max(float v, float* red) {
+    for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = red[0];
+    for (int j = 1; j < NTS / 32; ++j) r = fmaxf(r, red[j]);
+    return r;
+}
+__device__ __forceinline__ float block_sum(float v, float* red) {
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = 0.f;
+    for (int j = 0; j < NTS / 32; ++j) r += red[j];
+    return r;
+}
+
+// Unit of work = (code stream, piece): a contiguous range of the stream's token chunks.  The
+// CTA owns the unit's table, so its result is stored, not added.
+//
+// The table is accumulated in 32-bit fixed point: integer shared-memory atomics run at more
+// than twice the rate of fp32 ones (measured 17.5 against 7.7 per ns per SM), and integer
+// addition does not depend on the order, so the table is the same on every run.  A first
+// pass over the unit's weights and coefficients gives, per head, S = sum |w_t| and
+// U = max |coef|; no table entry can exceed S * U in magnitude, and the scale is the power
+// of two that maps S * U to at most 2^29, which leaves the rounding of the individual terms
+// (half a unit each) far inside the 32-bit range.  Each term w * coef is rounded once to
+// fp32, as a floating-point accumulation would, and once to the grid, whose step is
+// 2^-29 * S * U or finer.  A unit whose S or U is not finite falls back to fp32 atomics, so
+// that NaN and Inf still reach the output.
 template <int HGP>
 __global__ void __launch_bounds__(NTS)
 value_scatter_kernel(int N, const float* __restrict__ W, int B, int H, const uint16_t* __restrict__ idx,
-                     const void* __restrict__ coef, int coef_dtype, int64_t T, int s, int vec, float* __restrict__ A) {
+                     const void* __restrict__ coef, int coef_dtype, int64_t T, int s, int vec, int pieces,
+                     float* __restrict__ A) {
     extern __shared__ __align__(16) float tab[];           // [HGP][N]: scalar atomics want the heads apart
+    __shared__ float red[NTS / 32];
+    int* itab = reinterpret_cast<int*>(tab);
     const int64_t chunks_per_b = (T + CHUNK_T - 1) / CHUNK_T;
-    const int64_t total = (int64_t)B * chunks_per_b;
-    const int64_t w0 = total * blockIdx.x / gridDim.x, w1 = total * (blockIdx.x + 1) / gridDim.x;
-    for (int h0 = 0; h0 < H; h0 += HGP) {
-        const int hg = H - h0 < HGP ? H - h0 : HGP;
-        int cur_b = -1;
-        auto flush = [&]() {                               // add this CTA's table to the stream's rows of A
+    const int64_t units = (int64_t)B * pieces;
+    for (int64_t unit = blockIdx.x; unit < units; unit += gridDim.x) {
+        const int b = (int)(unit / pieces), piece = (int)(unit % pieces);
+        const int64_t c0 = chunks_per_b * piece / pieces, c1 = chunks_per_b * (piece + 1) / pieces;
+        for (int h0 = 0; h0 < H; h0 += HGP) {
+            const int hg = H - h0 < HGP ? H - h0 : HGP;
             __syncthreads();
-            if (cur_b >= 0) {
-                float* dst = A + ((int64_t)cur_b * H + h0) * N;
-                for (int j = threadIdx.x; j < hg * N; j += NTS) {
-                    const float v = tab[j];
-                    if (v != 0.f) atomicAdd(&dst[j], v);
+            for (int j = threadIdx.x; j < N * HGP; j += NTS) tab[j] = 0.f;    // +0.0f and integer 0 share their bits
+            // ---- pass 1: bounds ----
+            float umax = 0.f, sw[HGP];
+#pragma unroll
+            for (int h = 0; h < HGP; ++h) sw[h] = 0.f;
+            for (int64_t c = c0; c < c1; ++c) {
+                const int64_t t = c * CHUNK_T + threadIdx.x;
+                if (t >= T) continue;
+#pragma unroll
+                for (int h = 0; h < HGP; ++h)
+                    if (h < hg) sw[h] += fabsf(W[((int64_t)b * H + h0 + h) * T + t]);
+                for_each_code(idx, coef, coef_dtype, ((int64_t)b * T + t) * s, s, N, vec,
+                              [&](int, float cf) { umax = fmaxf(umax, fabsf(cf)); if (cf != cf) umax = INFINITY; });
+            }
+            umax = block_max(umax, red);
+            float scale[HGP], inv_scale[HGP];
+            bool fixed_point = umax < INFINITY;
+#pragma unroll
+            for (int h = 0; h < HGP; ++h) {
+                const float S = block_sum(sw[h], red);
+                const float bound = S * umax;
+                if (!(bound < INFINITY)) fixed_point = false;                 // Inf or NaN
+                int e = 0;
+                if (bound > 0.f) e = 29 - (ilogbf(bound) + 1);                // 2^e * bound <= 2^29
+                e = e > 96 ? 96 : e < -96 ? -96 : e;
+                scale[h] = ldexpf(1.f, e);
+                inv_scale[h] = ldexpf(1.f, -e);
+            }
+            __syncthreads();
+            // ---- pass 2: scatter ----
+            for (int64_t c = c0; c < c1; ++c) {
+                const int64_t t = c * CHUNK_T + threadIdx.x;
+                if (t >= T) continue;
+                float wv[HGP];
+#pragma unroll
+                for (int h = 0; h < HGP; ++h) wv[h] = h < hg ? W[((int64_t)b * H + h0 + h) * T + t] : 0.f;
+                if (fixed_point) {
+#pragma unroll
+                    for (int h = 0; h < HGP; ++h) wv[h] *= scale[h];          // exact: a power of two
+                    for_each_code(idx, coef, coef_dtype, ((int64_t)b * T + t) * s, s, N, vec, [&](int i, float cf) {
+#pragma unroll
+                        for (int h = 0; h < HGP; ++h)
+                            if (h < hg) atomicAdd(&itab[h * N + i], __float2int_rn(wv[h] * cf));
+                    });
+                } else {
+                    for_each_code(idx, coef, coef_dtype, ((int64_t)b * T + t) * s, s, N, vec, [&](int i, float cf) {
+#pragma unroll
+                        for (int h = 0; h < HGP; ++h)
+                            if (h < hg) atomicAdd(&tab[h * N + i], wv[h] * cf);
+                    });
                 }
             }
             __syncthreads();
-        };
-        for (int64_t w = w0; w < w1; ++w) {
-            const int b = (int)(w / chunks_per_b);
-            if (b != cur_b) {
-                flush();
-                for (int j = threadIdx.x; j < N * HGP; j += NTS) tab[j] = 0.f;
-                __syncthreads();
-                cur_b = b;
-            }
-            const int64_t t = (w % chunks_per_b) * CHUNK_T + threadIdx.x;
-            if (t >= T) continue;
-            float wv[HGP];
-#pragma unroll
-            for (int h = 0; h < HGP; ++h) wv[h] = h < hg ? W[((int64_t)b * H + h0 + h) * T + t] : 0.f;
-            for_each_code(idx, coef, coef_dtype, ((int64_t)b * T + t) * s, s, N, vec, [&](int i, float c) {
+            float* dst = A + ((unit * H) + h0) * N;         // rows h0 .. h0+hg-1 of this unit, [H][N]
+            if (fixed_point) {
 #pragma unroll
                 for (int h = 0; h < HGP; ++h)
-                    if (h < hg) atomicAdd(&tab[h * N + i], wv[h] * c);
-            });
+                    if (h < hg)
+                        for (int j = threadIdx.x; j < N; j += NTS) dst[h * N + j] = static_cast<float>(itab[h * N + j]) * inv_scale[h];
+            } else {
+                for (int j = threadIdx.x; j < hg * N; j += NTS) dst[j] = tab[j];
+            }
         }
-        flush();
     }
 }
 
@@ -356,20 +446,32 @@ cudaError_t run_key_scores(const AttnArgs& a, const float* P) {
     return cudaGetLastError();
 }
 
+// Token ranges a code stream is cut into for value_mix: enough to give every SM a unit, no
+// more than there are chunks.
+int value_pieces(int B, int64_t T) {
+    const int64_t chunks_per_b = (T + CHUNK_T - 1) / CHUNK_T;
+    int64_t k = B > 0 ? sm_count() / B : 1;
+    if (k > chunks_per_b) k = chunks_per_b;
+    return k < 1 ? 1 : (int)k;
+}
+
 template <int HGP>
-cudaError_t run_value_scatter(const AttnArgs& a, float* A) {
+cudaError_t run_value_scatter(const AttnArgs& a, float* A, int pieces) {
     const size_t smem = (size_t)HGP * a.N * 4;
     cudaError_t e = cudaFuncSetAttribute(value_scatter_kernel<HGP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    value_scatter_kernel<HGP><<<stream_grid(a.B, a.T), NTS, smem, a.stream>>>(a.N, static_cast<const float*>(a.Q), a.B, a.H,
-                                                                             a.idx, a.coef, a.coef_dtype, a.T, a.s,
-                                                                             a.s % 8 == 0, A);
+    const int64_t units = (int64_t)a.B * pieces;
+    const int grid = (int)(units < (int64_t)sm_count() ? units : (int64_t)sm_count());
+    value_scatter_kernel<HGP><<<grid, NTS, smem, a.stream>>>(a.N, static_cast<const float*>(a.Q), a.B, a.H, a.idx, a.coef,
+                                                            a.coef_dtype, a.T, a.s, a.s % 8 == 0, pieces, A);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-size_t attn_scratch_bytes(int B, int H, int N) { return (size_t)B * H * N * sizeof(float); }
+size_t attn_scratch_bytes(int B, int H, int N, int64_t T) {
+    return (size_t)B * value_pieces(B, T) * H * N * sizeof(float);
+}
 
 int launch_key_scores(const AttnArgs& a, float* P) {
     if (a.B == 0 || a.T == 0 || a.H == 0) return CSR_OK;
@@ -378,9 +480,9 @@ int launch_key_scores(const AttnArgs& a, float* P) {
     const int R = a.B * a.H;
     const dim3 pgrid((a.N + PA - 1) / PA, (R + QROWS - 1) / QROWS);
     if (a.d == 128)
-        qd_kernel<128><<<pgrid, NT, 0, a.stream>>>(a.D, a.N, a.Q, a.q_dtype, R, a.scale, P);
+        qd_kernel<128><<<pgrid, NT, 0, a.stream>>>(a.D, a.N, a.Q, a.q_dtype, R, a.H, a.scale, P);
     else
-        qd_kernel<64><<<pgrid, NT, 0, a.stream>>>(a.D, a.N, a.Q, a.q_dtype, R, a.scale, P);
+        qd_kernel<64><<<pgrid, NT, 0, a.stream>>>(a.D, a.N, a.Q, a.q_dtype, R, a.H, a.scale, P);
     cudaError_t e = hg == 8 ? run_key_scores<8>(a, P) : hg == 4 ? run_key_scores<4>(a, P)
                     : hg == 2 ? run_key_scores<2>(a, P) : run_key_scores<1>(a, P);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "key_scores launch: %s", cudaGetErrorString(e));
@@ -405,10 +507,9 @@ int launch_value_mix(const AttnArgs& a, float* A) {
     }
     const int hg = head_group(a.N, a.H);
     if (hg < 1) return fail(CSR_ERR_UNSUPPORTED, "N = %d: one head's N fp32 values do not fit in shared memory", a.N);
-    cudaError_t e = cudaMemsetAsync(A, 0, attn_scratch_bytes(a.B, a.H, a.N), a.stream);
-    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
-    e = hg == 8 ? run_value_scatter<8>(a, A) : hg == 4 ? run_value_scatter<4>(a, A)
-        : hg == 2 ? run_value_scatter<2>(a, A) : run_value_scatter<1>(a, A);
+    const int pieces = value_pieces(a.B, a.T);
+    cudaError_t e = hg == 8 ? run_value_scatter<8>(a, A, pieces) : hg == 4 ? run_value_scatter<4>(a, A, pieces)
+                    : hg == 2 ? run_value_scatter<2>(a, A, pieces) : run_value_scatter<1>(a, A, pieces);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "value_scatter launch: %s", cudaGetErrorString(e));
     // out = A D: row blocks of 16; with few row blocks the atoms are split over CTAs as well
     const int row_blocks = (R + OR - 1) / OR;
@@ -424,9 +525,9 @@ int launch_value_mix(const AttnArgs& a, float* A) {
     }
     const dim3 ogrid(row_blocks, slices);
     if (a.d == 128)
-        ad_kernel<128><<<ogrid, NT, 0, a.stream>>>(a.D, a.N, A, R, per_slice, slices > 1, a.out);
+        ad_kernel<128><<<ogrid, NT, 0, a.stream>>>(a.D, a.N, A, R, a.H, pieces, per_slice, slices > 1, a.out);
     else
-        ad_kernel<64><<<ogrid, NT, 0, a.stream>>>(a.D, a.N, A, R, per_slice, slices > 1, a.out);
+        ad_kernel<64><<<ogrid, NT, 0, a.stream>>>(a.D, a.N, A, R, a.H, pieces, per_slice, slices > 1, a.out);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "value_mix launch: %s", cudaGetErrorString(e));
     return CSR_OK;

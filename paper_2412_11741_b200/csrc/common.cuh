@@ -91,8 +91,9 @@ struct AttnArgs {
     float* out;
     cudaStream_t stream;
 };
-// `scratch` holds attn_scratch_bytes() bytes: the [B*H][N] fp32 array of partial products.
-size_t attn_scratch_bytes(int B, int H, int N);
+// `scratch` holds attn_scratch_bytes() bytes: the fp32 array of per-atom partial products
+// ([B][N][H] for the scores, [B][pieces][H][N] for the value mix).
+size_t attn_scratch_bytes(int B, int H, int N, int64_t T);
 int launch_key_scores(const AttnArgs& a, float* scratch);
 int launch_value_mix(const AttnArgs& a, float* scratch);
 int launch_softmax_rows(float* S, int64_t rows, int64_t T, cudaStream_t stream);   // in place, fp32

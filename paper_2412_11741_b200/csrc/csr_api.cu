@@ -472,7 +472,7 @@ int csr_key_scores(const void* D, int N, int d, const void* Q, int q_dtype, int 
                static_cast<cudaStream_t>(stream)};
     if (B == 0 || T == 0) return CSR_OK;
     void* base = nullptr;
-    if (int rc = ensure_work(attn_scratch_bytes(B, H, N), &base)) return rc;
+    if (int rc = ensure_work(attn_scratch_bytes(B, H, N, T), &base)) return rc;
     return launch_key_scores(a, static_cast<float*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)));
 }
 
@@ -484,7 +484,7 @@ int csr_value_mix(const void* D, int N, int d, const float* W, int B, int H, con
                static_cast<cudaStream_t>(stream)};
     if (B == 0) return CSR_OK;
     void* base = nullptr;
-    if (int rc = ensure_work(attn_scratch_bytes(B, H, N), &base)) return rc;
+    if (int rc = ensure_work(attn_scratch_bytes(B, H, N, T), &base)) return rc;
     return launch_value_mix(a, static_cast<float*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)));
 }
 
