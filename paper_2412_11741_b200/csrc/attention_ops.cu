@@ -20,7 +20,7 @@
 // adds when there are few heads).  The tables are accumulated in fixed point (see
 // value_scatter_kernel) and are the same on every run; the split over atoms of step (2),
 // when it is used, still adds in an order that varies.
-#include "common.cuh"
+#include "exact_common.cuh"
 
 namespace csr {
 namespace {
@@ -35,112 +35,170 @@ __device__ __forceinline__ float load_coef(const void* coef, int coef_dtype, int
 __device__ __forceinline__ float load_q(const void* Q, int q_dtype, int64_t off) { return load_elem(Q, q_dtype, off); }
 
 // ---- P[b][n][h] = scale * Q[r][:] . D[n][:]  (r = b*H + h) --------------------------------
-// CTA = 64 atoms x 64 rows; thread = 4 rows x 4 atoms; channels staged 32 at a time,
-// transposed, and summed in ascending order.
-constexpr int PA = 64;    // atoms per CTA
-constexpr int QROWS = 64; // rows per CTA (grid.y)
-constexpr int PK = 32;    // channels per staged block
+// CTA = 64 rows x one 128-atom tile of the dictionary, on the register-tiled product the
+// exact encoder sweeps with (thread = 4 rows x 8 atoms, channels summed in ascending order).
 template <int D_>
 __global__ void __launch_bounds__(NT)
 qd_kernel(const float* __restrict__ D, int N, const void* __restrict__ Q, int q_dtype, int R, int H, float scale,
           float* __restrict__ P) {
-    __shared__ __align__(16) float Ds[PK][PA + 4];         // Ds[k][atom]
-    __shared__ __align__(16) float Qs[PK][QROWS + 4];      // Qs[k][row]
-    const int n0 = blockIdx.x * PA, r0 = blockIdx.y * QROWS;
-    const int ta = (threadIdx.x & 15) * 4, tr = (threadIdx.x >> 4) * 4;
-    float acc[4][4];
+    __shared__ __align__(16) float As[D_][exact::AS_LD];              // As[k][row]
+    __shared__ __align__(16) float Bs[2][exact::BK][exact::BS_LD];
+    const int r0 = blockIdx.y * exact::BM;
+    for (int f = threadIdx.x; f < exact::BM * D_; f += NT) {
+        const int r = f / D_, k = f % D_;
+        As[k][r] = (r0 + r < R) ? load_q(Q, q_dtype, (int64_t)(r0 + r) * D_ + k) : 0.f;
+    }
+    __syncthreads();
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    exact::sweep_tiles_fn<D_>(D, N, blockIdx.x, blockIdx.x + 1, As, Bs, [&](int bt, const float (&acc)[4][8]) {
+        const int rr = r0 + ty * 4;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int n = bt * exact::BN + (j >> 2) * 64 + tx * 4 + (j & 3);
+            if (n >= N) continue;
+            if (H == 4 && rr + 3 < R) {                   // the four rows are one stream's four heads
+                float4 v;
+                v.x = scale * acc[0][j];
+                v.y = scale * acc[1][j];
+                v.z = scale * acc[2][j];
+                v.w = scale * acc[3][j];
+                *reinterpret_cast<float4*>(P + ((int64_t)(rr / 4) * N + n) * 4) = v;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int r = rr + i;
+                    if (r < R) P[((int64_t)(r / H) * N + n) * H + r % H] = scale * acc[i][j];
+                }
+            }
+        }
+    });
+}
+
+// ---- part[slice][r][:] = sum_{n in slice} (sum_pieces A[b][piece][h][n]) * D[n][:] ----------
+// CTA = 64 rows x all channels x one slice of the atoms; thread = 4 rows x 8 (d = 128) or 4
+// (d = 64) channels.  The slice is taken 64 atoms at a time: all of a tile's loads are issued
+// together (one memory latency per tile, several CTAs per SM to cover it), then the tile is
+// multiplied out of shared memory, atoms in ascending order.  With more than one slice a
+// second kernel adds the slices in order, so the result does not depend on the schedule.
+constexpr int OR = 64;    // rows per CTA
+constexpr int OA = 64;    // atoms per tile
+template <int D_>
+struct AdSmem {
+    float As[OA][OR + 4];      // As[atom][row]
+    float Bs[OA][D_ + 4];      // Bs[atom][channel]
+};
+template <int D_>
+__global__ void __launch_bounds__(NT, 3)
+ad_kernel(const float* __restrict__ D, int N, const float* __restrict__ A, int R, int H, int pieces, int atoms_per_slice,
+          float* __restrict__ part) {
+    extern __shared__ __align__(16) unsigned char ad_raw[];
+    AdSmem<D_>& sm = *reinterpret_cast<AdSmem<D_>*>(ad_raw);
+    constexpr int CPT = D_ / 16;                          // channels per thread: 8 or 4
+    constexpr int DV = OA * D_ / 4 / NT;                  // float4 of D per thread per tile: 8 or 4
+    constexpr int AV = OA * OR / 4 / NT;                  // float4 of A per thread per tile: 4
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const int r0 = blockIdx.y * OR;
+    const int nb = blockIdx.x * atoms_per_slice;
+    const int ne = min(nb + atoms_per_slice, N);
+    const int64_t piece_stride = (int64_t)H * N;
+    const bool vec_a = (N % 4) == 0;                       // rows of A start on 16-byte boundaries
+    float acc[4][CPT];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-    for (int k0 = 0; k0 < D_; k0 += PK) {
-        __syncthreads();
-        for (int f = threadIdx.x; f < PA * PK; f += NT) {
-            const int a = f / PK, k = f % PK;
-            Ds[k][a] = (n0 + a < N) ? D[(int64_t)(n0 + a) * D_ + k0 + k] : 0.f;
+        for (int j = 0; j < CPT; ++j) acc[i][j] = 0.f;
+    for (int n0 = nb; n0 < ne; n0 += OA) {
+        // ---- stage the tile: A (pieces summed in order, transposed) and D ----
+        float4 av[AV];
+#pragma unroll
+        for (int u = 0; u < AV; ++u) av[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int pc = 0; pc < pieces; ++pc) {
+#pragma unroll
+            for (int u = 0; u < AV; ++u) {
+                const int f = tid + u * NT;               // float4 index: row = f / 16, atoms 4 * (f % 16) ..
+                const int r = r0 + f / (OA / 4), n = n0 + 4 * (f % (OA / 4));
+                if (r >= R || n >= ne) continue;
+                const float* src = A + (((int64_t)(r / H) * pieces + pc) * H + r % H) * N + n;
+                float4 v;
+                if (vec_a && n + 3 < ne) {
+                    v = *reinterpret_cast<const float4*>(src);
+                } else {
+                    v.x = src[0];
+                    v.y = n + 1 < ne ? src[1] : 0.f;
+                    v.z = n + 2 < ne ? src[2] : 0.f;
+                    v.w = n + 3 < ne ? src[3] : 0.f;
+                }
+                av[u].x += v.x;
+                av[u].y += v.y;
+                av[u].z += v.z;
+                av[u].w += v.w;
+            }
         }
-        for (int f = threadIdx.x; f < QROWS * PK; f += NT) {
-            const int r = f / PK, k = f % PK;
-            Qs[k][r] = (r0 + r < R) ? load_q(Q, q_dtype, (int64_t)(r0 + r) * D_ + k0 + k) : 0.f;
+        float4 dv[DV];
+#pragma unroll
+        for (int u = 0; u < DV; ++u) {
+            const int f = tid + u * NT;
+            const int atom = f / (D_ / 4), c4 = f % (D_ / 4);
+            dv[u] = (n0 + atom < ne) ? *reinterpret_cast<const float4*>(D + (int64_t)(n0 + atom) * D_ + c4 * 4)
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        __syncthreads();                                   // the previous tile has been used
+#pragma unroll
+        for (int u = 0; u < AV; ++u) {
+            const int f = tid + u * NT;
+            const int r = f / (OA / 4), a4 = 4 * (f % (OA / 4));
+            sm.As[a4 + 0][r] = av[u].x;
+            sm.As[a4 + 1][r] = av[u].y;
+            sm.As[a4 + 2][r] = av[u].z;
+            sm.As[a4 + 3][r] = av[u].w;
+        }
+#pragma unroll
+        for (int u = 0; u < DV; ++u) {
+            const int f = tid + u * NT;
+            *reinterpret_cast<float4*>(&sm.Bs[f / (D_ / 4)][(f % (D_ / 4)) * 4]) = dv[u];
         }
         __syncthreads();
+        // ---- multiply ----
 #pragma unroll 8
-        for (int k = 0; k < PK; ++k) {
-            const float4 dv = *reinterpret_cast<const float4*>(&Ds[k][ta]);
-            const float4 qv = *reinterpret_cast<const float4*>(&Qs[k][tr]);
-            const float d[4] = {dv.x, dv.y, dv.z, dv.w};
-            const float q[4] = {qv.x, qv.y, qv.z, qv.w};
+        for (int k = 0; k < OA; ++k) {
+            const float4 a4 = *reinterpret_cast<const float4*>(&sm.As[k][ty * 4]);
+            const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+            float bch[CPT];
+#pragma unroll
+            for (int q = 0; q < CPT / 4; ++q) {
+                const float4 b4 = *reinterpret_cast<const float4*>(&sm.Bs[k][q * 64 + tx * 4]);
+                bch[4 * q + 0] = b4.x;
+                bch[4 * q + 1] = b4.y;
+                bch[4 * q + 2] = b4.z;
+                bch[4 * q + 3] = b4.w;
+            }
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(q[i], d[j], acc[i][j]);
+                for (int j = 0; j < CPT; ++j) acc[i][j] = fmaf(a[i], bch[j], acc[i][j]);
         }
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const int r = r0 + tr + i;
-        if (r < R) {
+        const int r = r0 + ty * 4 + i;
+        if (r >= R) continue;
+        float* dst = part + ((int64_t)blockIdx.x * R + r) * D_;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (n0 + ta + j < N) P[((int64_t)(r / H) * N + n0 + ta + j) * H + r % H] = scale * acc[i][j];
-        }
+        for (int q = 0; q < CPT / 4; ++q)
+            *reinterpret_cast<float4*>(dst + q * 64 + tx * 4) =
+                make_float4(acc[i][4 * q + 0], acc[i][4 * q + 1], acc[i][4 * q + 2], acc[i][4 * q + 3]);
     }
 }
 
-// ---- out[r][:] (+)= sum_{n in slice} (sum_pieces A[b][piece][h][n]) * D[n][:] ---------------
-// CTA = 16 rows x one atom slice; thread = (channel, group of rows).
-constexpr int OR = 16;    // rows per CTA
-constexpr int OA = 64;    // atoms per staged block
-template <int D_>
+// out[j] = part[0][j] + part[1][j] + ... in this order
 __global__ void __launch_bounds__(NT)
-ad_kernel(const float* __restrict__ D, int N, const float* __restrict__ A, int R, int H, int pieces, int atoms_per_slice,
-          int use_atomics, float* __restrict__ out) {
-    __shared__ float Ds[OA][D_];
-    __shared__ __align__(16) float As[OR][OA];
-    constexpr int RG = NT / D_;            // row groups (2 or 4)
-    constexpr int RPT = OR / RG;           // rows per thread (8 or 4)
-    const int c = threadIdx.x % D_, rg = threadIdx.x / D_;
-    const int r0 = blockIdx.x * OR;
-    const int nb = blockIdx.y * atoms_per_slice;
-    const int ne = min(nb + atoms_per_slice, N);
-    float acc[RPT];
-#pragma unroll
-    for (int i = 0; i < RPT; ++i) acc[i] = 0.f;
-    for (int n0 = nb; n0 < ne; n0 += OA) {
-        __syncthreads();
-        for (int f = threadIdx.x; f < OA * D_; f += NT) {
-            const int a = f / D_, k = f % D_;
-            Ds[a][k] = (n0 + a < ne) ? D[(int64_t)(n0 + a) * D_ + k] : 0.f;
-        }
-        for (int f = threadIdx.x; f < OR * OA; f += NT) {
-            const int r = f / OA, a = f % OA;
-            float v = 0.f;
-            if (r0 + r < R && n0 + a < ne) {                // row (b, h): the stream's pieces in order
-                const int64_t bb = (r0 + r) / H, hh = (r0 + r) % H;
-                for (int pc = 0; pc < pieces; ++pc) v += A[((bb * pieces + pc) * H + hh) * N + n0 + a];
-            }
-            As[r][a] = v;
-        }
-        __syncthreads();
-        for (int a = 0; a < OA; a += 4) {
-            const float d0 = Ds[a][c], d1 = Ds[a + 1][c], d2 = Ds[a + 2][c], d3 = Ds[a + 3][c];
-#pragma unroll
-            for (int i = 0; i < RPT; ++i) {
-                const float4 w = *reinterpret_cast<const float4*>(&As[rg * RPT + i][a]);
-                acc[i] = fmaf(w.w, d3, fmaf(w.z, d2, fmaf(w.y, d1, fmaf(w.x, d0, acc[i]))));
-            }
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < RPT; ++i) {
-        const int r = r0 + rg * RPT + i;
-        if (r < R) {
-            if (use_atomics)
-                atomicAdd(&out[(int64_t)r * D_ + c], acc[i]);
-            else
-                out[(int64_t)r * D_ + c] = acc[i];
-        }
-    }
+add_slices_kernel(const float* __restrict__ part, int slices, int64_t n, float* __restrict__ out) {
+    const int64_t j = (int64_t)blockIdx.x * NT + threadIdx.x;
+    if (j >= n) return;
+    float v = 0.f;
+    for (int sl = 0; sl < slices; ++sl) v += part[(int64_t)sl * n + j];
+    out[j] = v;
 }
 
 // Eight consecutive codes of one token (16-byte loads; the caller guarantees s % 8 == 0 and
@@ -469,8 +527,10 @@ cudaError_t run_value_scatter(const AttnArgs& a, float* A, int pieces) {
 
 }  // namespace
 
+// tables of the value mix (the larger use) + the per-slice outputs of its second step
 size_t attn_scratch_bytes(int B, int H, int N, int64_t T) {
-    return (size_t)B * value_pieces(B, T) * H * N * sizeof(float);
+    const size_t slices_max = 4 * (size_t)sm_count();
+    return ((size_t)B * value_pieces(B, T) * H * N + 4 + slices_max * (size_t)B * H * 128) * sizeof(float);
 }
 
 int launch_key_scores(const AttnArgs& a, float* P) {
@@ -478,7 +538,7 @@ int launch_key_scores(const AttnArgs& a, float* P) {
     const int hg = head_group(a.N, a.H);
     if (hg < 1) return fail(CSR_ERR_UNSUPPORTED, "N = %d: one head's N fp32 values do not fit in shared memory", a.N);
     const int R = a.B * a.H;
-    const dim3 pgrid((a.N + PA - 1) / PA, (R + QROWS - 1) / QROWS);
+    const dim3 pgrid((a.N + exact::BN - 1) / exact::BN, (R + exact::BM - 1) / exact::BM);
     if (a.d == 128)
         qd_kernel<128><<<pgrid, NT, 0, a.stream>>>(a.D, a.N, a.Q, a.q_dtype, R, a.H, a.scale, P);
     else
@@ -511,23 +571,30 @@ int launch_value_mix(const AttnArgs& a, float* A) {
     cudaError_t e = hg == 8 ? run_value_scatter<8>(a, A, pieces) : hg == 4 ? run_value_scatter<4>(a, A, pieces)
                     : hg == 2 ? run_value_scatter<2>(a, A, pieces) : run_value_scatter<1>(a, A, pieces);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "value_scatter launch: %s", cudaGetErrorString(e));
-    // out = A D: row blocks of 16; with few row blocks the atoms are split over CTAs as well
+    // out = A D: row blocks of 64; the atoms are split over CTAs as well (four CTAs per SM: each
+    // waits for its next chunk of atoms most of the time)
     const int row_blocks = (R + OR - 1) / OR;
     int slices = 4 * sm_count() / row_blocks;
-    const int max_slices = (a.N + 255) / 256;
+    const int max_slices = (a.N + 63) / 64;
     if (slices > max_slices) slices = max_slices;
     if (slices < 1) slices = 1;
-    int per_slice = ((a.N + slices - 1) / slices + OA - 1) / OA * OA;
+    const int per_slice = ((a.N + slices - 1) / slices + OA - 1) / OA * OA;
     slices = (a.N + per_slice - 1) / per_slice;
-    if (slices > 1) {
-        e = cudaMemsetAsync(a.out, 0, (size_t)R * a.d * sizeof(float), a.stream);
-        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    float* part = slices > 1 ? A + ((size_t)a.B * pieces * a.H * a.N + 3) / 4 * 4 : a.out;      // 16-byte aligned
+    const dim3 ogrid(slices, row_blocks);
+    cudaError_t e2;
+    if (a.d == 128) {
+        e2 = cudaFuncSetAttribute(ad_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AdSmem<128>));
+        ad_kernel<128><<<ogrid, NT, sizeof(AdSmem<128>), a.stream>>>(a.D, a.N, A, R, a.H, pieces, per_slice, part);
+    } else {
+        e2 = cudaFuncSetAttribute(ad_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AdSmem<64>));
+        ad_kernel<64><<<ogrid, NT, sizeof(AdSmem<64>), a.stream>>>(a.D, a.N, A, R, a.H, pieces, per_slice, part);
     }
-    const dim3 ogrid(row_blocks, slices);
-    if (a.d == 128)
-        ad_kernel<128><<<ogrid, NT, 0, a.stream>>>(a.D, a.N, A, R, a.H, pieces, per_slice, slices > 1, a.out);
-    else
-        ad_kernel<64><<<ogrid, NT, 0, a.stream>>>(a.D, a.N, A, R, a.H, pieces, per_slice, slices > 1, a.out);
+    if (e2 != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e2));
+    if (slices > 1) {
+        const int64_t n = (int64_t)R * a.d;
+        add_slices_kernel<<<(unsigned)((n + NT - 1) / NT), NT, 0, a.stream>>>(part, slices, n, a.out);
+    }
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "value_mix launch: %s", cudaGetErrorString(e));
     return CSR_OK;

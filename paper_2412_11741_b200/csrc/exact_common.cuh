@@ -55,14 +55,16 @@ __device__ __forceinline__ void top2_push_fast(Top2& t, float a, int n) {
     t.idx = p ? n : t.idx;
 }
 
-// Sweep of dictionary tiles [bt0, bt1) (128 atoms each) for the 64 rows whose fp32 residual
-// sits transposed in As (Eq. 2-3): fp32 register-tiled products, each thread 4 rows x 8
-// atoms, k ascending; every thread keeps the two largest |correlations| of its rows.
-// Bs is the double-buffered staging area of dictionary chunks (8 channels each; the next
-// chunk waits in registers while the current one is used).  Ends with a __syncthreads.
-template <int D_>
-__device__ __forceinline__ void sweep_tiles(const float* __restrict__ D, int N, int bt0, int bt1,
-                                            const float (*As)[AS_LD], float (*Bs)[BK][BS_LD], Top2 (&top)[4]) {
+// Products of the 64 rows whose fp32 values sit transposed in As with the atoms of dictionary
+// tiles [bt0, bt1) (128 atoms each): fp32 register-tiled, each thread 4 rows x 8 atoms, k
+// ascending.  Thread (tx, ty) = (tid & 15, tid >> 4) ends every tile with acc[i][j] = the
+// product of row ty*4 + i with atom bt*128 + (j >> 2)*64 + tx*4 + (j & 3) and hands it to
+// on_tile(bt, acc).  Bs is the double-buffered staging area of dictionary chunks (8 channels
+// each; the next chunk waits in registers while the current one is used).  Ends with a
+// __syncthreads.
+template <int D_, typename TileFn>
+__device__ __forceinline__ void sweep_tiles_fn(const float* __restrict__ D, int N, int bt0, int bt1,
+                                               const float (*As)[AS_LD], float (*Bs)[BK][BS_LD], TileFn&& on_tile) {
     static_assert(BK == 8 && NT == 2 * BN, "two threads stage one atom's eight channels");
     constexpr int KCH = D_ / BK;                          // chunks per tile (even)
     const int tid = threadIdx.x;
@@ -128,6 +130,16 @@ __device__ __forceinline__ void sweep_tiles(const float* __restrict__ D, int N, 
             if (more) sstore(Bs[0]);
             __syncthreads();
         }
+        on_tile(bt, acc);
+    }
+}
+
+// The sweep of Eq. 2-3: every thread keeps the two largest |correlations| of its rows.
+template <int D_>
+__device__ __forceinline__ void sweep_tiles(const float* __restrict__ D, int N, int bt0, int bt1,
+                                            const float (*As)[AS_LD], float (*Bs)[BK][BS_LD], Top2 (&top)[4]) {
+    const int tx = threadIdx.x & 15;
+    sweep_tiles_fn<D_>(D, N, bt0, bt1, As, Bs, [&](int bt, const float (&acc)[4][8]) {
         const int nb = bt * BN + tx * 4;
         if ((bt + 1) * BN <= N) {                         // a whole tile: no atom to leave out
 #pragma unroll
@@ -144,7 +156,7 @@ __device__ __forceinline__ void sweep_tiles(const float* __restrict__ D, int N, 
                 }
             }
         }
-    }
+    });
 }
 
 // Re-scoring of a row whose two largest fp32 |correlations| are too close to call, by the

@@ -152,6 +152,23 @@ def test_attention_from_codes_matches_oracle(csr, B, H, T, N, d, s, coef_dtype):
     want = orc.value_mix(D, W, idx, coef.astype(np.float64))
     mbound = (W[:, :, :, None] * np.abs(coef)[:, None, :, :]).sum((2, 3))[:, :, None]       # sum w |coef| ||atom||
     assert mix.shape == want.shape and np.all(np.abs(mix - want) <= 4e-6 * mbound + 1e-30)
+    if T:
+        # fixed-point tables and ordered sums: the same bits on every run
+        again = csr.csr_value_mix(Dd, torch.from_numpy(W).to(DEV), it, ct).cpu().numpy()
+        assert np.array_equal(mix, again)
+        # weights that are not a softmax row: one large, the rest tiny, some negative
+        Wp = (W * 1e-4).astype(np.float32)
+        Wp[:, :, T // 2] = 3.0
+        Wp[:, :, ::7] *= -1.0
+        mix = csr.csr_value_mix(Dd, torch.from_numpy(Wp).to(DEV), it, ct).cpu().numpy()
+        want = orc.value_mix(D, Wp, idx, coef.astype(np.float64))
+        mbound = (np.abs(Wp)[:, :, :, None] * np.abs(coef)[:, None, :, :]).sum((2, 3))[:, :, None]
+        assert np.all(np.abs(mix - want) <= 4e-6 * mbound + 1e-30)
+        # a NaN weight still reaches the output of its own head, and only that one
+        Wn = W.copy()
+        Wn[0, 0, T // 3] = np.nan
+        mix = csr.csr_value_mix(Dd, torch.from_numpy(Wn).to(DEV), it, ct).cpu().numpy()
+        assert np.all(np.isnan(mix[0, 0])) and np.all(np.isfinite(mix[0, 1:])) and np.all(np.isfinite(mix[1:]))
 
 
 def test_scores_from_codes_equal_scores_from_the_restored_tensor(csr):
