@@ -106,7 +106,8 @@ def run_decode_case(seqs, kv_heads, N, s, reps):
 def run_attention_case(reps):
     """Attention straight from the codes on the GQA long-context shape: 64 code streams (8
     sequences x 8 KV heads) of 16384 tokens, s = 16, 4 query heads per KV head.  Rates are
-    algorithmic HBM bytes (codes read once, scores written / weights read once) over time;
+    algorithmic HBM bytes (codes read once, scores written / weights read once) over time, with
+    inputs rotated so that they come from HBM;
     the restored-tensor route (de-sparse kernel to bf16, then reading it back once) is timed
     beside it as the traffic it avoids."""
     dev = torch.device("cuda", torch.cuda.current_device())
@@ -117,13 +118,37 @@ def run_attention_case(reps):
     coef = torch.randn((B, T, s), device=dev, generator=g).to(torch.float16)
     Q = torch.randn((B, H, d), device=dev, generator=g)
     W = torch.softmax(torch.randn((B, H, T), device=dev, generator=g), dim=-1)
-    sc = torch.empty((B, H, T), dtype=torch.float32, device=dev)
     out = torch.empty((B, H, d), dtype=torch.float32, device=dev)
     xh = torch.empty((B * T, d), dtype=torch.bfloat16, device=dev)
-    t_sc = _time(lambda: csr.csr_key_scores(D, Q, idx, coef, 1.0, scores=sc), reps)
-    t_mx = _time(lambda: csr.csr_value_mix(D, W, idx, coef, out=out), reps)
-    t_rc = _time(lambda: csr.csr_reconstruct_ex(D, idx.view(B * T, s), coef.view(B * T, s), X_hat=xh), reps)
-    t_da = _time(lambda: csr.csr_decode_attention(D, D, Q, idx, coef, idx, coef, 1.0 / d ** 0.5, weights=sc, out=out), reps)
+    # three copies of the codes, weights and score arrays taken in turn: 250 MB, twice the L2, so
+    # every call streams its codes from HBM as a decoding step over a long cache does
+    copies = [(idx.clone(), coef.clone(), W.clone(), torch.empty((B, H, T), dtype=torch.float32, device=dev)) for _ in range(3)]
+    turn = [0]
+
+    def nxt():
+        turn[0] = (turn[0] + 1) % len(copies)
+        return copies[turn[0]]
+
+    def f_scores():
+        i, c, _, sc = nxt()
+        csr.csr_key_scores(D, Q, i, c, 1.0, scores=sc)
+
+    def f_mix():
+        i, c, w, _ = nxt()
+        csr.csr_value_mix(D, w, i, c, out=out)
+
+    def f_restore():
+        i, c, _, _ = nxt()
+        csr.csr_reconstruct_ex(D, i.view(B * T, s), c.view(B * T, s), X_hat=xh)
+
+    def f_attention():
+        i, c, _, sc = nxt()
+        csr.csr_decode_attention(D, D, Q, i, c, i, c, 1.0 / d ** 0.5, weights=sc, out=out)
+
+    t_sc = _time(f_scores, reps)
+    t_mx = _time(f_mix, reps)
+    t_rc = _time(f_restore, reps)
+    t_da = _time(f_attention, reps)
     code_b, sw_b = B * T * s * 4.0, B * H * T * 4.0
     return {"case": "attention_from_codes", "B": B, "H": H, "T": T, "N": N, "d": d, "s": s,
             "key_scores_ms": round(t_sc, 4), "key_scores_hbm_gbs": (code_b + sw_b) / (t_sc * 1e-3) / 1e9,
