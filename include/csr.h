@@ -15,7 +15,9 @@
  *   - Calls are asynchronous with respect to the host: work is enqueued on the given
  *     CUDA stream (the 8-argument forms use the legacy default stream, 0) and the
  *     function returns without synchronising, except csr_encode_host and
- *     csr_device_status, which synchronise.
+ *     csr_device_status, which synchronise.  A device-pointer call whose scratch does
+ *     not have to grow (a repeat of an earlier call's shapes, or csr_encode_static) only
+ *     launches kernels and may be captured into a CUDA graph and replayed.
  *   - Layout.  D is [N][d] row-major fp32: one atom per row, the d channels contiguous
  *     (the paper's d x N matrix of "Sparse representation", stored column by column).
  *     Atoms are assumed unit l2-norm; this is not checked and the formulas are applied

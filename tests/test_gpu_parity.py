@@ -273,6 +273,35 @@ def test_fast_few_rows_split_dictionary_path(csr, M, N, d, s, kind, monkeypatch)
         assert rep.ok, rep.detail
 
 
+@pytest.mark.parametrize("M", [16, 1024, 70000])
+def test_encode_captured_in_a_cuda_graph(csr, M):
+    """A decoding loop replays its step as a CUDA graph: after one ordinary call (which sizes
+    the library's buffers) the encode, clustered or not, can be captured and replayed."""
+    rng = np.random.default_rng(M)
+    N, d, s = 4096, 128, 8
+    Dd = torch.from_numpy(wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))).to(DEV)
+    X1 = torch.from_numpy(rng.standard_normal((M, d)).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    X2 = torch.from_numpy(rng.standard_normal((M, d)).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    want1 = csr.csr_encode_ex(Dd, X1, s)
+    want2 = csr.csr_encode_ex(Dd, X2, s)
+    h = csr.csr_dict_create(Dd)
+    X = X1.clone()
+    idx = torch.zeros((M, s), dtype=torch.int16, device=DEV).view(torch.uint16)
+    coef = torch.zeros((M, s), dtype=torch.float16, device=DEV)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        csr.csr_encode_ex(Dd, X, s, out_idx=idx, out_coef=coef, dict=h)
+    for want, src in ((want1, X1), (want2, X2)):
+        X.copy_(src)
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(_np_idx(idx), _np_idx(want[0])) and torch.equal(coef, want[1])
+    assert csr.csr_device_status() == csr.CSR_OK
+    del g
+    csr.csr_dict_destroy(h)
+
+
 def test_fast_fp32_input_and_odd_s(csr):
     rng = np.random.default_rng(13)
     D = wl.normalise_rows(rng.standard_normal((1024, 128)).astype(np.float32))
