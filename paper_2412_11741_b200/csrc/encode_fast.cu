@@ -952,6 +952,8 @@ EncodeTiledFn get_encode_tiled() {
     return fn;
 }
 
+constexpr int kClusterLaunchRefused = 1;                  // internal: not a CSR_ERR_* code
+
 template <int D_, int G>
 void cluster_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int cluster_ctas, int grid, size_t smem,
                     cudaStream_t stream) {
@@ -1022,7 +1024,11 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
         e = cudaLaunchKernelEx(&cfg, encode_fast_kernel<D_, G, true>, tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
                                a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask, status, n_splits,
                                static_cast<uint2*>(nullptr));
-        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "encode_fast cluster launch: %s", cudaGetErrorString(e));
+        if (e != cudaSuccess) {
+            // refused at launch (nothing ran): the caller takes another path
+            cudaGetLastError();
+            return kClusterLaunchRefused;
+        }
         return CSR_OK;
     }
     encode_fast_kernel<D_, G, false><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
@@ -1088,8 +1094,25 @@ int cluster_split(int64_t M, int N, float budget_us, int* grid) {
 }
 
 template <int D_>
+int launch_clustered_g(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, float budget_us,
+                       bool* done);
+
+// *done says whether the clustered launch took the job; a launch the driver refuses leaves
+// it to the other paths.
+template <int D_>
 int launch_clustered(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, float budget_us,
                      bool* done) {
+    const int rc = launch_clustered_g<D_>(a, tmap, Db, status, budget_us, done);
+    if (rc == kClusterLaunchRefused) {
+        *done = false;
+        return CSR_OK;
+    }
+    return rc;
+}
+
+template <int D_>
+int launch_clustered_g(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, float budget_us,
+                       bool* done) {
     int grid = 0, ns = 0;
     *done = false;
     switch (group_size(D_, a.N)) {
