@@ -231,6 +231,7 @@ struct FastSmem {
     uint64_t acc_empty[2];
     uint64_t res_ready[2];
     uint64_t drained;
+    uint64_t pair_bar;                                 // CL == 2: second warp group's result is in xout
     uint64_t xbar[2];                                  // cluster exchange: gathered / merged, one phase per iteration each
     unsigned long long xin[2 * TILE_M];                // cluster exchange: (key, ~tile) of the rows this CTA merges, per source CTA
     unsigned long long xout[2 * TILE_M];               // cluster exchange: merged (key, ~tile) of every row
@@ -565,7 +566,7 @@ split_pick_kernel(const uint16_t* __restrict__ Db, int N, uint4* __restrict__ Rb
 // ---------------------------------------------------------------------------------------
 // the encoder
 // ---------------------------------------------------------------------------------------
-template <int D_, int G, bool CL>
+template <int D_, int G, int CL>
 __global__ void __launch_bounds__(NT, 1)
 encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* __restrict__ Db,
                    const void* __restrict__ X, int x_dtype, int64_t ldx, int64_t M, int N, int s,
@@ -585,6 +586,11 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
     //    After each sweep every row's best (key, tile) is max-reduced into every CTA's shared
     //    memory, every CTA then makes the same pick and the same residual update on its own
     //    copy of the rows, and CTA 0 of the cluster writes the codes.
+    //    CL == 2: at most TILE_M rows in all (one decoding step of a small batch).  Only the
+    //    first row tile exists; the two accumulators take the CTA's dictionary tiles in turn
+    //    and the second group of epilogue warps drains the second accumulator for the same
+    //    rows; the unused second row tile holds the exchange buffers, large enough for every
+    //    CTA to hear from every CTA directly (one hop).
     //  - otherwise ONE iteration per launch (s == 1 is passed): each row's best (key, tile) goes
     //    to `partial` and the pick kernel takes over.
     const int t_begin = n_splits > 1 ? (int)(blockIdx.x % n_splits) : 0;
@@ -608,12 +614,17 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             mbar_init(&sm.res_ready[t], TILE_M);
         }
         mbar_init(&sm.drained, 1);
-        if constexpr (CL) {
+        if constexpr (CL == 1) {
             // one phase per iteration: this thread arms it with the bytes the peers will send
             mbar_init(&sm.xbar[0], 1);
             mbar_init(&sm.xbar[1], 1);
             mbar_expect_tx(&sm.xbar[0], 2 * TILE_M * 8);
             mbar_expect_tx(&sm.xbar[1], 2 * TILE_M * 8);
+        }
+        if constexpr (CL == 2) {
+            mbar_init(&sm.xbar[0], 1);
+            mbar_expect_tx(&sm.xbar[0], static_cast<uint32_t>(n_splits) * TILE_M * 8);
+            mbar_init(&sm.pair_bar, TILE_M);
         }
         sm.abort = 0;
         fence_barrier_init();
@@ -663,7 +674,54 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         }
     } else if (warp == MMA_WARP) {
         // ------------------------------ MMA issuer ------------------------------
-        if (lane == 0) {
+        if (lane == 0 && CL == 2) {
+            // one row tile; the CTA's dictionary tiles go to the two accumulators in turn
+            uint32_t p = 0, accn[2] = {0u, 0u};
+            bool ok = true;
+            for (int g = 0; g < s && ok; ++g) {
+                if (!wait_bounded(&sm.res_ready[0], g & 1, wc)) {
+                    ok = false;
+                    break;
+                }
+                int j = 0;
+                for (int t = t_begin; t < T && ok; t += t_step, p += KH, ++j) {
+                    const int acc = j & 1;
+                    if (!wait_bounded(&sm.acc_empty[acc], (accn[acc] & 1) ^ 1, wc)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t d_tmem = tmem_base + acc * TILE_N;
+#pragma unroll
+                    for (int h = 0; h < KH; ++h) {
+                        const uint32_t ps = p + h;
+                        const int stage = ps % STAGES;
+                        if (!wait_bounded(&sm.full_b[stage], (ps / STAGES) & 1, wc)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint64_t a0 = make_smem_desc(smem_u32(&sm.A[0][h * (TILE_M * 128)]));
+                        const uint64_t b0 = make_smem_desc(smem_u32(&sm.B[stage][0]));
+#pragma unroll
+                        for (int k = 0; k < KSTEPS; ++k) {
+                            const uint64_t off = static_cast<uint64_t>((k * 32) >> 4);
+                            umma_bf16(d_tmem, a0 + off, b0 + off, kInstrDesc, (h | k) ? 1u : 0u);
+                        }
+                        umma_commit(&sm.empty_b[stage]);
+                    }
+                    if (ok) {
+                        umma_commit(&sm.acc_full[acc]);
+                        ++accn[acc];
+                    }
+                }
+            }
+            if (!ok) {
+                umma_commit(&sm.drained);
+                const unsigned long long t0 = globaltimer_ns();
+                while (!mbar_try_wait(&sm.drained, 0))
+                    if (globaltimer_ns() - t0 > 20000000ull) break;
+            }
+        } else if (lane == 0) {
             uint32_t p = 0, accn = 0, steps = 0;
             bool ok = true;
             for (int64_t pair = pair_first; pair < n_pairs && ok; pair += pair_step) {
@@ -714,14 +772,15 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         }
     } else {
         // ------------------------------ epilogue ------------------------------
-        const int tile = warp >> 2;
+        const int acc = warp >> 2;                        // the accumulator this warp drains
+        const int tile = CL == 2 ? 0 : acc;               // the row tile its rows belong to
         const int q = warp & 3;
         const int r = q * 32 + lane;                      // row inside the tile == TMEM lane
         const int slot = tile * TILE_M + r;               // row inside the CTA's pair
         uint8_t* Atile = &sm.A[tile][0];
         uint16_t (*code_idx)[CODE_BLOCK] = &sm.code_idx[tile * TILE_M];
         float (*code_coef)[CODE_BLOCK] = &sm.code_coef[tile * TILE_M];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + tile * TILE_N;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * TILE_N;
         uint32_t accn = 0;
         [[maybe_unused]] uint32_t xn = 0;
         bool ok = true;
@@ -732,7 +791,9 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             uint32_t row_mask = 0xffffffffu;
             if constexpr (CL) row_mask = __ballot_sync(0xffffffffu, valid);
             // ---- R_0 = x, rounded to bf16, into the operand tile ----
-            if (x_dtype == CSR_DTYPE_BF16) {
+            if (CL == 2 && acc == 1) {
+                // the second warp group has no rows of its own
+            } else if (x_dtype == CSR_DTYPE_BF16) {
                 const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(X) + m * ldx);
 #pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
@@ -773,14 +834,16 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     *reinterpret_cast<uint4*>(Atile + swz_off(r, c)) = v;
                 }
             }
-            fence_proxy_async_smem();
-            mbar_arrive(&sm.res_ready[tile]);
+            if (CL != 2 || acc == 0) {
+                fence_proxy_async_smem();
+                mbar_arrive(&sm.res_ready[tile]);
+            }
 
             for (int g = 0; g < s && ok; ++g) {
                 // ---- sweep: running arg-max of |correlation| over all atom tiles ----
                 uint32_t best_key = 0, best_t = 0;
-                for (int t = t_begin; t < T; t += t_step, ++accn) {
-                    bool got = wait_bounded(&sm.acc_full[tile], accn & 1, wc);
+                for (int t = t_begin + (CL == 2 ? acc * t_step : 0); t < T; t += (CL == 2 ? 2 : 1) * t_step, ++accn) {
+                    bool got = wait_bounded(&sm.acc_full[acc], accn & 1, wc);
                     got = __all_sync(0xffffffffu, got);
                     if (!got) {
                         ok = false;
@@ -812,7 +875,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     // every column of this accumulator is in registers: hand it back
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.acc_empty[tile]);
+                    if (lane == 0) mbar_arrive(&sm.acc_empty[acc]);
                     chunk_key_max<G, 128>(v0, key_mask, k0, k1);
                     chunk_key_max<G, 160>(v1, key_mask, k0, k1);
                     chunk_key_max<G, 192>(v2, key_mask, k0, k1);
@@ -828,7 +891,54 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     if (valid) partial[m * n_splits + t_begin] = make_uint2(best_key, best_t);
                     continue;
                 }
-                if constexpr (CL) {
+                if constexpr (CL == 2) {
+                    // ---- the row's best over this CTA's tiles (both accumulators), then over the
+                    // whole dictionary: every CTA sends its (key, ~tile) of the row to every CTA.
+                    // The entries are double-buffered by iteration: a peer writes iteration g + 2's
+                    // only after it has heard this CTA's iteration g + 1, which the thread that
+                    // reads the entries sends after it has read iteration g's. ----
+                    unsigned long long mine = (static_cast<unsigned long long>(best_key) << 32) | (0xFFFFFFFFu - best_t);
+                    // (a CTA with a single dictionary tile has no use for the second group, which
+                    // would otherwise run ahead of the first: nothing paces it but its sweep)
+                    const bool two_groups = t_begin + t_step < T;
+                    if (acc == 1) {
+                        if (!two_groups) break;
+                        sm.xout[r] = mine;
+                        mbar_arrive(&sm.pair_bar);
+                        ++xn;
+                        continue;                           // nothing more for this group until the next sweep
+                    }
+                    bool got = !two_groups || wait_bounded(&sm.pair_bar, xn & 1, wc);
+                    if (got) {
+                        if (two_groups) {
+                            const unsigned long long other = *reinterpret_cast<volatile unsigned long long*>(&sm.xout[r]);
+                            mine = other > mine ? other : mine;
+                        }
+                        constexpr int XMAX = FastSmem<D_>::kATileBytes / (2 * TILE_M * 8);   // CTAs the buffers hold
+                        unsigned long long* xg = reinterpret_cast<unsigned long long*>(&sm.A[1][0]) + (xn & 1) * XMAX * TILE_M;
+                        const uint32_t dst = smem_u32(&xg[t_begin * TILE_M + r]), bar = smem_u32(&sm.xbar[0]);
+                        for (int c = 0; c < n_splits; ++c) st_async_u64(map_to_cta(dst, c), mine, map_to_cta(bar, c));
+                        got = wait_bounded_cluster(&sm.xbar[0], xn & 1, wc);
+                        if (got) {
+                            if (r == 0) mbar_expect_tx(&sm.xbar[0], static_cast<uint32_t>(n_splits) * TILE_M * 8);
+                            unsigned long long top = 0ull;
+                            for (int c = 0; c < n_splits; ++c) {
+                                const unsigned long long v = *reinterpret_cast<volatile unsigned long long*>(&xg[c * TILE_M + r]);
+                                top = v > top ? v : top;
+                            }
+                            mine = top;
+                        }
+                    }
+                    got = __all_sync(0xffffffffu, got);
+                    if (!got) {
+                        ok = false;
+                        break;
+                    }
+                    ++xn;
+                    best_key = static_cast<uint32_t>(mine >> 32);
+                    best_t = 0xFFFFFFFFu - static_cast<uint32_t>(mine);
+                }
+                if constexpr (CL == 1) {
                     // ---- every CTA of the cluster learns the row's best over the whole dictionary:
                     // the highest key and, among equal keys, the lowest tile.  Row i of the pair is
                     // merged by CTA i % n_splits: gather there, merge, send the result to everyone.
@@ -978,16 +1088,18 @@ int max_clusters(int cluster_ctas) {
     if (cached[cluster_ctas] == 0) {
         const size_t smem = sizeof(FastSmem<D_>) + 1024;
         int n = 0;
-        bool good = cudaFuncSetAttribute(encode_fast_kernel<D_, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        bool good = cudaFuncSetAttribute(encode_fast_kernel<D_, G, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem) == cudaSuccess;
         if (good && cluster_ctas > 8)
-            good = cudaFuncSetAttribute(encode_fast_kernel<D_, G, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
-                   cudaSuccess;
+            good = cudaFuncSetAttribute(encode_fast_kernel<D_, G, 1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
+                       cudaSuccess &&
+                   cudaFuncSetAttribute(encode_fast_kernel<D_, G, 2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
+                       cudaSuccess;
         if (good) {
             cudaLaunchConfig_t cfg = {};
             cudaLaunchAttribute attr[1];
             cluster_config<D_, G>(cfg, attr, cluster_ctas, cluster_ctas, smem, 0);
-            good = cudaOccupancyMaxActiveClusters(&n, encode_fast_kernel<D_, G, true>, &cfg) == cudaSuccess;
+            good = cudaOccupancyMaxActiveClusters(&n, encode_fast_kernel<D_, G, 1>, &cfg) == cudaSuccess;
         }
         if (!good) {
             cudaGetLastError();                        // a refusal is an answer, not a failure of the call
@@ -1002,10 +1114,13 @@ template <int D_, int G>
 int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uint32_t* status, int n_splits,
            uint2* partial, int cluster_grid = 0) {
     const size_t smem = sizeof(FastSmem<D_>) + 1024;
+    // at most one tile of rows in all: the clustered kernel that spends both accumulators on it
+    const bool one_tile = cluster_grid > 0 && a.M <= TILE_M && n_splits <= FastSmem<D_>::kATileBytes / (2 * TILE_M * 8);
     cudaError_t e =
         cluster_grid > 0
-            ? cudaFuncSetAttribute(encode_fast_kernel<D_, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-            : cudaFuncSetAttribute(encode_fast_kernel<D_, G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            ? cudaFuncSetAttribute(one_tile ? encode_fast_kernel<D_, G, 2> : encode_fast_kernel<D_, G, 1>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+            : cudaFuncSetAttribute(encode_fast_kernel<D_, G, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     const int64_t n_pairs = (a.M + 2 * TILE_M - 1) / (2 * TILE_M);
     const int grid = n_splits > 1 ? (int)(n_pairs * n_splits)
@@ -1021,7 +1136,7 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute attr[1];
         cluster_config<D_, G>(cfg, attr, n_splits, cluster_grid, smem, a.stream);
-        e = cudaLaunchKernelEx(&cfg, encode_fast_kernel<D_, G, true>, tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
+        e = cudaLaunchKernelEx(&cfg, one_tile ? encode_fast_kernel<D_, G, 2> : encode_fast_kernel<D_, G, 1>, tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
                                a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask, status, n_splits,
                                static_cast<uint2*>(nullptr));
         if (e != cudaSuccess) {
@@ -1031,7 +1146,7 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
         }
         return CSR_OK;
     }
-    encode_fast_kernel<D_, G, false><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
+    encode_fast_kernel<D_, G, 0><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
                                                            a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask,
                                                            status, n_splits, partial);
     e = cudaGetLastError();
@@ -1078,6 +1193,8 @@ int cluster_split(int64_t M, int N, float budget_us, int* grid) {
     int best_ns = 0;
     for (int ns = 16; ns >= 2; ns >>= 1) {
         if (ns > T) continue;
+        // one tile of rows: the exchange buffers (the unused row tile) bound the cluster size
+        if (M <= TILE_M && ns > FastSmem<D_>::kATileBytes / (2 * TILE_M * 8)) continue;
         const int nc = max_clusters<D_, G>(ns);
         if (nc < 1) continue;
         const int64_t rounds = (n_pairs + nc - 1) / nc;

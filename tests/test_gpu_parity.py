@@ -235,7 +235,9 @@ def test_fast_any_dictionary_size(csr, N, G, monkeypatch):
 
 @pytest.mark.parametrize("M,N,d,s,kind", [(1, 8192, 128, 16, "bf16"), (128, 8192, 128, 16, "bf16"), (300, 1000, 128, 5, "f32"),
                                           (2000, 4096, 64, 8, "f16"), (9000, 2048, 128, 4, "bf16"), (16, 65536, 64, 3, "bf16"),
-                                          (24500, 65536, 128, 2, "bf16")])     # more row pairs than clusters fit at once
+                                          (24500, 65536, 128, 2, "bf16"),      # more row pairs than clusters fit at once
+                                          (16, 4096, 128, 8, "bf16"), (100, 6144, 128, 5, "f32"), (64, 2048, 64, 4, "f16"),
+                                          (128, 16384, 128, 6, "bf16"), (129, 8192, 128, 4, "bf16")])   # one row tile: 1, 1-2, 1, 4 tiles per CTA; just over
 def test_fast_few_rows_split_dictionary_path(csr, M, N, d, s, kind, monkeypatch):
     """Few rows: the dictionary is split across the CTAs of a cluster (one launch) or, without
     clusters, across CTAs with one sweep and one pick launch per iteration.  Both must return
