@@ -232,6 +232,7 @@ struct FastSmem {
     uint64_t res_ready[2];
     uint64_t drained;
     uint64_t pair_bar;                                 // CL == 2: second warp group's result is in xout
+    uint64_t pick_bar;                                 // CL == 2: the rows' picks are in xin (for the second group)
     uint64_t xbar[2];                                  // cluster exchange: gathered / merged, one phase per iteration each
     unsigned long long xin[2 * TILE_M];                // cluster exchange: (key, ~tile) of the rows this CTA merges, per source CTA
     unsigned long long xout[2 * TILE_M];               // cluster exchange: merged (key, ~tile) of every row
@@ -611,7 +612,8 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
         for (int t = 0; t < 2; ++t) {
             mbar_init(&sm.acc_full[t], 1);
             mbar_init(&sm.acc_empty[t], 4);
-            mbar_init(&sm.res_ready[t], TILE_M);
+            // (with one tile of rows both warp groups update rows of it)
+            mbar_init(&sm.res_ready[t], CL == 2 ? 2 * TILE_M : TILE_M);
         }
         mbar_init(&sm.drained, 1);
         if constexpr (CL == 1) {
@@ -625,6 +627,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
             mbar_init(&sm.xbar[0], 1);
             mbar_expect_tx(&sm.xbar[0], static_cast<uint32_t>(n_splits) * TILE_M * 8);
             mbar_init(&sm.pair_bar, TILE_M);
+            mbar_init(&sm.pick_bar, TILE_M);
         }
         sm.abort = 0;
         fence_barrier_init();
@@ -834,14 +837,13 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     *reinterpret_cast<uint4*>(Atile + swz_off(r, c)) = v;
                 }
             }
-            if (CL != 2 || acc == 0) {
-                fence_proxy_async_smem();
-                mbar_arrive(&sm.res_ready[tile]);
-            }
+            fence_proxy_async_smem();
+            mbar_arrive(&sm.res_ready[tile]);
 
             for (int g = 0; g < s && ok; ++g) {
                 // ---- sweep: running arg-max of |correlation| over all atom tiles ----
                 uint32_t best_key = 0, best_t = 0;
+                [[maybe_unused]] int n0_other = 0;
                 for (int t = t_begin + (CL == 2 ? acc * t_step : 0); t < T; t += (CL == 2 ? 2 : 1) * t_step, ++accn) {
                     bool got = wait_bounded(&sm.acc_full[acc], accn & 1, wc);
                     got = __all_sync(0xffffffffu, got);
@@ -901,15 +903,19 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     // (a CTA with a single dictionary tile has no use for the second group, which
                     // would otherwise run ahead of the first: nothing paces it but its sweep)
                     const bool two_groups = t_begin + t_step < T;
+                    int* pick_n0 = reinterpret_cast<int*>(&sm.xin[0]);
+                    bool got = true;
                     if (acc == 1) {
-                        if (!two_groups) break;
-                        sm.xout[r] = mine;
-                        mbar_arrive(&sm.pair_bar);
-                        ++xn;
-                        continue;                           // nothing more for this group until the next sweep
+                        if (two_groups) {
+                            sm.xout[r] = mine;
+                            mbar_arrive(&sm.pair_bar);
+                        }
+                        // the second half of every warp's rows is picked and updated by this group
+                        got = wait_bounded(&sm.pick_bar, xn & 1, wc);
+                    } else if (two_groups) {
+                        got = wait_bounded(&sm.pair_bar, xn & 1, wc);
                     }
-                    bool got = !two_groups || wait_bounded(&sm.pair_bar, xn & 1, wc);
-                    if (got) {
+                    if (got && acc == 0) {
                         if (two_groups) {
                             const unsigned long long other = *reinterpret_cast<volatile unsigned long long*>(&sm.xout[r]);
                             mine = other > mine ? other : mine;
@@ -937,6 +943,16 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     ++xn;
                     best_key = static_cast<uint32_t>(mine >> 32);
                     best_t = 0xFFFFFFFFu - static_cast<uint32_t>(mine);
+                    if (acc == 0) {
+                        pick_n0[r] = min(static_cast<int>(best_t) * TILE_N +
+                                             (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G,
+                                         ((N + 7) / 8) * 8 - G);
+                        mbar_arrive(&sm.pick_bar);
+                        row_mask &= 0x0000FFFFu;
+                    } else {
+                        n0_other = *reinterpret_cast<volatile int*>(&pick_n0[r]);
+                        row_mask &= 0xFFFF0000u;
+                    }
                 }
                 if constexpr (CL == 1) {
                     // ---- every CTA of the cluster learns the row's best over the whole dictionary:
@@ -986,9 +1002,10 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 const int gi = g & (CODE_BLOCK - 1);
                 // (NaN correlations can make a zero-filled column past the dictionary win: keep the
                 // gather inside the padded bf16 copy whatever the keys say)
-                const int n0 = min(static_cast<int>(best_t) * TILE_N +
-                                       (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G,
-                                   ((N + 7) / 8) * 8 - G);
+                int n0 = min(static_cast<int>(best_t) * TILE_N +
+                                 (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G,
+                             ((N + 7) / 8) * 8 - G);
+                if (CL == 2 && acc == 1) n0 = n0_other;
                 if constexpr (CL)
                     pick_and_update<D_, G, true>(Atile, q, lane, Db, n0, g + 1 < s, code_idx, code_coef, gi, row_mask);
                 else
@@ -999,7 +1016,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 }
                 __syncwarp();
                 // ---- flush the collected codes eight at a time ----
-                if ((gi == CODE_BLOCK - 1 || g == s - 1) && valid && writes_codes) {
+                if ((gi == CODE_BLOCK - 1 || g == s - 1) && valid && writes_codes && (CL != 2 || (lane < 16) == (acc == 0))) {
                     const int g0 = g - gi;
                     const int64_t o = m * ldc + g0;
                     if (gi == CODE_BLOCK - 1 && vec_codes) {
