@@ -213,7 +213,12 @@ int csr_dict_destroy(csr_dict_t* dict);
  *
  * Several problems in one call (one dictionary per layer, per K / V, per chunk): the
  * problems are validated first, all of them, and nothing is enqueued if one is invalid;
- * then they are enqueued in order on their streams.  Returns the first failure.
+ * then they are enqueued in order on their streams.  Neighbouring fast-mode problems on
+ * the same stream that each bring their own dictionary copy (`dict` or `workspace`) depend
+ * on nothing shared and are enqueued side by side: the stream forks into library-owned
+ * side streams and joins again before the call returns, so work enqueued afterwards sees
+ * all of them (the K rows and the V rows of one decoding step take the time of one).
+ * Returns the first failure.
  */
 int csr_encode_grouped(const csr_encode_params_t* problems, int count);
 int csr_reconstruct_grouped(const csr_reconstruct_params_t* problems, int count);

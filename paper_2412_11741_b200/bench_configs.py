@@ -100,6 +100,16 @@ def run_decode_case(seqs, kv_heads, N, s, reps):
     os.environ["CSR_FAST_NO_SPLIT"] = "1"
     out["fast_one_launch_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, Xb, s, out_idx=idx, out_coef=coef), reps)
     del os.environ["CSR_FAST_NO_SPLIT"]
+    # the step as a cache sees it: the K rows and the V rows (half of M each) against their own
+    # dictionaries, one grouped call with dictionary handles
+    D2 = torch.nn.functional.normalize(D.flip(0) + 0.5 * D, dim=1).contiguous()     # a second dictionary
+    h1, h2 = csr.csr_dict_create(D), csr.csr_dict_create(D2)
+    half = M // 2
+    parts = [(D, Xb[:half], s, idx[:half], coef[:half], h1), (D2, Xb[half:], s, idx[half:], coef[half:], h2)]
+    out["fast_k_and_v_grouped_us"] = 1e3 * _time(lambda: csr.csr_encode_grouped(parts), reps)
+    out["fast_k_then_v_us"] = 1e3 * _time(lambda: [csr.csr_encode_ex(p[0], p[1], s, out_idx=p[3], out_coef=p[4], dict=p[5]) for p in parts], reps)
+    csr.csr_dict_destroy(h1)
+    csr.csr_dict_destroy(h2)
     return out
 
 

@@ -313,14 +313,19 @@ def _reconstruct_params(D, idx, coef, out_dtype, X_hat):
 
 
 def csr_encode_grouped(problems, *, mode: int = CSR_MODE_BF16_FAST) -> None:
-    """csr_encode_grouped: `problems` is a sequence of (D, X, s, out_idx, out_coef) with CUDA
-    tensors; X, out_idx and out_coef may be column slices of wider arrays (row strides are
-    passed on).  All problems are validated before any is enqueued."""
+    """csr_encode_grouped: `problems` is a sequence of (D, X, s, out_idx, out_coef) or
+    (D, X, s, out_idx, out_coef, dict) with CUDA tensors (dict: a csr_dict_create handle of D);
+    X, out_idx and out_coef may be column slices of wider arrays (row strides are passed on).
+    All problems are validated before any is enqueued; neighbouring fast-mode problems that
+    each bring a handle are enqueued side by side."""
     arr = (csr_encode_params_t * len(problems))()
-    for i, (D, X, s, out_idx, out_coef) in enumerate(problems):
+    for i, prob in enumerate(problems):
+        D, X, s, out_idx, out_coef = prob[:5]
         assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.stride(1) == 1 and D.dtype == torch.float32
         assert out_idx.dtype == torch.uint16 and out_idx.stride(1) == 1 and out_coef.stride(1) == 1
         arr[i] = _encode_params(D, X, s, out_idx, out_coef, mode, _stream_ptr(X), None)
+        if len(prob) > 5 and prob[5] is not None:
+            arr[i].dict = prob[5]
     if len(problems):
         with torch.cuda.device(problems[0][0].device):
             _check(lib().csr_encode_grouped(arr, len(problems)))

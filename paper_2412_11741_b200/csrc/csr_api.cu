@@ -49,6 +49,7 @@ constexpr size_t kStatusBytes = 256;
 constexpr uint32_t kDictMagic = 0x43535244u;   // "CSRD"
 
 // Library-owned, grow-only device buffers of one device.
+constexpr int kSideStreams = 3;
 struct DeviceBuffers {
     void* work = nullptr;      // [status word | encoder scratch]
     size_t work_bytes = 0;
@@ -59,9 +60,14 @@ struct DeviceBuffers {
     size_t stage_x_bytes = 0, stage_code_bytes = 0;
     cudaStream_t copy_streams[2] = {nullptr, nullptr};
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
+    // grouped calls: problems that may run side by side
+    cudaStream_t side[kSideStreams] = {};
+    cudaEvent_t side_done[kSideStreams] = {};
+    cudaEvent_t fork = nullptr;
 };
 DeviceBuffers g_dev[kMaxDevices];
 std::mutex g_mu;
+std::mutex g_group_mu;     // one grouped fork/join at a time: its events are shared
 
 int current_device(int* dev) {
     cudaError_t e = cudaGetDevice(dev);
@@ -237,8 +243,27 @@ int64_t workspace_bytes(int mode, int d, int N) {
     return (int64_t)(kStatusBytes + 1024 + encode_fast_workspace_bytes(d, N));
 }
 
-// Runs one encode on device pointers.
-int encode_device(const csr_encode_params_t* p) {
+// Streams and events of a grouped call, made on first use.
+int ensure_side_streams(DeviceBuffers** out) {
+    int dev;
+    if (int rc = current_device(&dev)) return rc;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceBuffers& b = g_dev[dev];
+    if (!b.fork) {
+        cudaError_t e = cudaEventCreateWithFlags(&b.fork, cudaEventDisableTiming);
+        for (int i = 0; i < kSideStreams && e == cudaSuccess; ++i) {
+            e = cudaStreamCreateWithFlags(&b.side[i], cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b.side_done[i], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "side streams: %s", cudaGetErrorString(e));
+    }
+    *out = &b;
+    return CSR_OK;
+}
+
+// Runs one encode on device pointers.  `shared_scratch` = false keeps the call off the parts of
+// the library-owned buffer that two encodes in flight would both write.
+int encode_device(const csr_encode_params_t* p, bool shared_scratch = true) {
     if (p->M == 0) return CSR_OK;
     EncodeArgs a;
     a.D = static_cast<const float*>(p->D);
@@ -268,7 +293,8 @@ int encode_device(const csr_encode_params_t* p) {
     // few rows: the cluster path needs no scratch; its fallback (a launch pair per iteration)
     // does, and gets it from the library-owned buffer only (a caller workspace is sized for
     // the bf16 copy)
-    const bool split = !p->workspace && encode_fast_split_applies(p->M, p->N) && !getenv("CSR_FAST_NO_SPLIT");
+    const bool split =
+        shared_scratch && !p->workspace && encode_fast_split_applies(p->M, p->N) && !getenv("CSR_FAST_NO_SPLIT");
     const size_t dict_b = (encode_fast_workspace_bytes(p->d, p->N) + 1023) / 1024 * 1024;
     const size_t split_b = split ? encode_fast_split_scratch_bytes(p->M, p->d, p->N) : 0;
     if (p->dict) {
@@ -416,8 +442,51 @@ int csr_encode_grouped(const csr_encode_params_t* problems, int count) {
     if (count < 0 || (count > 0 && !problems)) return fail(CSR_ERR_INVALID_ARG, "problems is NULL or count < 0");
     for (int i = 0; i < count; ++i)
         if (int rc = check_encode(&problems[i], false)) return rc;
-    for (int i = 0; i < count; ++i)
-        if (int rc = encode_device(&problems[i])) return rc;
+    // Problems that follow one another on the same stream, in the fast mode, each with its own
+    // dictionary copy (a handle or a caller workspace) share nothing the library owns but the
+    // status word: they are enqueued side by side (the stream forks into side streams and
+    // joins again), which is what the K and V rows of one decoding step want: each fills a
+    // fraction of the GPU.  Everything else runs in order.
+    auto independent = [](const csr_encode_params_t& q) {
+        return q.mode == CSR_MODE_BF16_FAST && (q.dict || q.workspace) && q.M > 0;
+    };
+    int i = 0;
+    while (i < count) {
+        int j = i + 1;
+        if (independent(problems[i]))
+            while (j < count && independent(problems[j]) && problems[j].stream == problems[i].stream) ++j;
+        if (j - i < 2) {
+            if (int rc = encode_device(&problems[i])) return rc;
+            i = j;
+            continue;
+        }
+        DeviceBuffers* b = nullptr;
+        if (int rc = ensure_side_streams(&b)) return rc;
+        std::lock_guard<std::mutex> group_lock(g_group_mu);
+        cudaStream_t main = static_cast<cudaStream_t>(problems[i].stream);
+        cudaError_t e = cudaEventRecord(b->fork, main);
+        bool used[kSideStreams] = {};
+        int rc = CSR_OK;
+        for (int k = i + 1; k < j && rc == CSR_OK && e == cudaSuccess; ++k) {
+            const int sidx = (k - i - 1) % kSideStreams;
+            if (!used[sidx]) e = cudaStreamWaitEvent(b->side[sidx], b->fork, 0);
+            used[sidx] = true;
+            csr_encode_params_t q = problems[k];
+            q.stream = b->side[sidx];
+            if (e == cudaSuccess) rc = encode_device(&q, false);
+        }
+        if (rc == CSR_OK && e == cudaSuccess) rc = encode_device(&problems[i], false);
+        // join whatever was forked, also after a failure: the caller's stream must not run ahead
+        for (int sidx = 0; sidx < kSideStreams; ++sidx) {
+            if (!used[sidx]) continue;
+            cudaError_t e2 = cudaEventRecord(b->side_done[sidx], b->side[sidx]);
+            if (e2 == cudaSuccess) e2 = cudaStreamWaitEvent(main, b->side_done[sidx], 0);
+            if (e == cudaSuccess) e = e2;
+        }
+        if (rc != CSR_OK) return rc;
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "grouped encode fork/join: %s", cudaGetErrorString(e));
+        i = j;
+    }
     return CSR_OK;
 }
 
@@ -698,6 +767,16 @@ int csr_release_workspace(void) {
         b.stage_x[i] = b.stage_idx[i] = b.stage_coef[i] = nullptr;
     }
     b.stage_x_bytes = b.stage_code_bytes = 0;
+    if (b.fork) {
+        cudaEventDestroy(b.fork);
+        b.fork = nullptr;
+        for (int i = 0; i < kSideStreams; ++i) {
+            cudaStreamDestroy(b.side[i]);
+            cudaEventDestroy(b.side_done[i]);
+            b.side[i] = nullptr;
+            b.side_done[i] = nullptr;
+        }
+    }
     return CSR_OK;
 }
 

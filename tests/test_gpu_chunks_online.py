@@ -83,6 +83,32 @@ def test_packed_codes_of_two_chunks_use_vector_stores_when_they_can(csr):
         assert torch.equal(c2.cpu(), coef[:, s * c:s * (c + 1)].cpu())
 
 
+@pytest.mark.parametrize("M", [64, 3000])
+def test_grouped_problems_with_handles_run_side_by_side(csr, M):
+    """The K rows and the V rows of a decoding step: two dictionaries, two handles, one grouped
+    call.  Such problems are enqueued side by side; the codes are those of separate calls, and
+    work enqueued afterwards on the caller's stream sees all of them (the join)."""
+    rng = np.random.default_rng(M)
+    N, d, s = 2048, 128, 8
+    Ds = [torch.from_numpy(wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))).to(DEV) for _ in range(3)]
+    Xs = [torch.from_numpy(rng.standard_normal((M, d)).astype(np.float32)).to(DEV).to(torch.bfloat16) for _ in range(3)]
+    want = [csr.csr_encode_ex(D, X, s) for D, X in zip(Ds, Xs)]
+    hs = [csr.csr_dict_create(D) for D in Ds]
+    idx = [torch.zeros((M, s), dtype=torch.int16, device=DEV).view(torch.uint16) for _ in range(3)]
+    coef = [torch.zeros((M, s), dtype=torch.float16, device=DEV) for _ in range(3)]
+    # the third problem brings no handle: it runs after the first two, in order
+    csr.csr_encode_grouped([(Ds[0], Xs[0], s, idx[0], coef[0], hs[0]), (Ds[1], Xs[1], s, idx[1], coef[1], hs[1]),
+                            (Ds[2], Xs[2], s, idx[2], coef[2])])
+    total = sum(c.float().sum() for c in coef)                        # on the caller's stream, after the join
+    torch.cuda.synchronize()
+    assert csr.csr_device_status() == csr.CSR_OK
+    for k in range(3):
+        assert np.array_equal(_np_idx(idx[k]), _np_idx(want[k][0])) and torch.equal(coef[k], want[k][1])
+    assert float(total) == float(sum(w[1].float().sum() for w in want))
+    for h in hs:
+        csr.csr_dict_destroy(h)
+
+
 @pytest.mark.parametrize("d,dtype", [(128, "bf16"), (64, "f32")])
 def test_online_atoms_match_oracle_and_are_used_by_the_encoder(csr, d, dtype):
     """Sampled rows of the cache become unit-norm atoms behind the offline part; the encoder
