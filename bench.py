@@ -35,9 +35,9 @@ UNIT = "vectors/s"
 WORKLOAD = "gqa_long_context: 8 seq x 16384 tok x 8 kv_heads x {K,V}, d=128, M=2097152, N=8192, s=16, bf16"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of encode_fast_kernel<128, 1, false> at M = 524288, N = 8192,
+# dram__bytes_read.sum + dram__bytes_write.sum of encode_fast_kernel<128, 1, 0> at M = 524288, N = 8192,
 # s = 16 (profiles/encode_fast_small_case_ncu_full.md), per row; traffic grows in proportion to M.
-DRAM_BYTES_PER_ROW_NCU = (136.882688e6 + 19.478784e6) / 524288
+DRAM_BYTES_PER_ROW_NCU = (137.349376e6 + 20.825344e6) / 524288
 
 
 def _peaks():
@@ -275,7 +275,7 @@ def run_cuda(args):
         achieved = flops / (enc * 1e-3) / 1e12
         hbm_bytes = M * d * 2 + N * d * 4 + M * s * 4
         roof = {
-            "bound": "tensor", "kernel": "encode_fast_kernel<128, 1, false>", "achieved": achieved, "peak": peaks["bf16_tflops"],
+            "bound": "tensor", "kernel": "encode_fast_kernel<128, 1, 0>", "achieved": achieved, "peak": peaks["bf16_tflops"],
             "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
             "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
             "flops_per_launch": flops, "kernel_ms": enc, "traffic": DRAM_BYTES_PER_ROW_NCU * M,
