@@ -41,6 +41,22 @@
 // issuer.  All hand-offs are mbarriers; every wait is bounded by a wall-clock limit,
 // after which the CTA raises a flag in the status word, lets its copies land, frees
 // its TMEM and exits.
+//
+// Few rows (the vectors one decoding step adds) would leave all but a few SMs idle, each of
+// them sweeping the whole dictionary s times.  Three instantiations of the kernel cover
+// that case (template argument CL):
+//   CL = 0  the kernel above; with n_splits > 1 it sweeps only a slice of the dictionary for
+//           ONE iteration and leaves the rows' maxima to split_pick_kernel (a launch pair
+//           per iteration: the fallback where clusters cannot be launched);
+//   CL = 1  n_splits CTAs form a thread-block cluster, hold the same pair of row tiles and
+//           each sweep a slice; after every sweep the rows' maxima are exchanged through
+//           distributed shared memory (st.async credited to the peers' mbarriers: gather at
+//           the CTA that merges a row, merged value back to everyone) and every CTA makes
+//           the same pick and update, so all s iterations run in one launch;
+//   CL = 2  the same with at most 128 rows in all: both accumulators and both epilogue warp
+//           groups serve the one row tile, and the other row tile's shared memory holds
+//           exchange buffers large enough for a one-hop all-to-all.
+// The codes are the same bits in every case.
 #include <cuda.h>
 
 #include <cstdlib>
@@ -235,7 +251,9 @@ struct FastSmem {
     uint64_t pick_bar;                                 // CL == 2: the rows' picks are in xin (for the second group)
     uint64_t xbar[2];                                  // cluster exchange: gathered / merged, one phase per iteration each
     unsigned long long xin[2 * TILE_M];                // cluster exchange: (key, ~tile) of the rows this CTA merges, per source CTA
+                                                       // (CL == 2: the rows' winning atoms, for the second warp group)
     unsigned long long xout[2 * TILE_M];               // cluster exchange: merged (key, ~tile) of every row
+                                                       // (CL == 2: the second warp group's maxima)
     uint32_t tmem_base;
     volatile uint32_t abort;
 };
