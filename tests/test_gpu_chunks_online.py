@@ -105,6 +105,19 @@ def test_grouped_problems_with_handles_run_side_by_side(csr, M):
     for k in range(3):
         assert np.array_equal(_np_idx(idx[k]), _np_idx(want[k][0])) and torch.equal(coef[k], want[k][1])
     assert float(total) == float(sum(w[1].float().sum() for w in want))
+    # the same call captured into a CUDA graph (the fork and the join become graph edges)
+    for k in range(3):
+        idx[k].zero_()
+        coef[k].zero_()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        csr.csr_encode_grouped([(Ds[0], Xs[0], s, idx[0], coef[0], hs[0]), (Ds[1], Xs[1], s, idx[1], coef[1], hs[1])])
+    g.replay()
+    torch.cuda.synchronize()
+    for k in range(2):
+        assert np.array_equal(_np_idx(idx[k]), _np_idx(want[k][0])) and torch.equal(coef[k], want[k][1])
+    del g
     for h in hs:
         csr.csr_dict_destroy(h)
 
