@@ -353,7 +353,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 // than twice the rate of fp32 ones (measured 17.5 against 7.7 per ns per SM), and integer
 // addition does not depend on the order, so the table is the same on every run.  A first
 // pass over the unit's weights and coefficients gives, per head, S = sum |w_t| and
-// U = max |coef|; no table entry can exceed S * U in magnitude, and the scale is the power
+// U = max over tokens of sum_g |coef[t][g]| (a token's entries may all name one atom); no
+// table entry can exceed S * U in magnitude, and the scale is the power
 // of two that maps S * U to at most 2^29, which leaves the rounding of the individual terms
 // (half a unit each) far inside the 32-bit range.  Each term w * coef is rounded once to
 // fp32, as a floating-point accumulation would, and once to the grid, whose step is
@@ -386,8 +387,10 @@ value_scatter_kernel(int N, const float* __restrict__ W, int B, int H, const uin
 #pragma unroll
                 for (int h = 0; h < HGP; ++h)
                     if (h < hg) sw[h] += fabsf(W[((int64_t)b * H + h0 + h) * T + t]);
+                float l1 = 0.f;                            // all of a token's entries may name the same atom
                 for_each_code(idx, coef, coef_dtype, ((int64_t)b * T + t) * s, s, N, vec,
-                              [&](int, float cf) { umax = fmaxf(umax, fabsf(cf)); if (cf != cf) umax = INFINITY; });
+                              [&](int, float cf) { l1 += fabsf(cf); });
+                umax = l1 == l1 ? fmaxf(umax, l1) : INFINITY;
             }
             umax = block_max(umax, red);
             float scale[HGP], inv_scale[HGP];

@@ -210,6 +210,25 @@ def test_attention_from_codes_matches_oracle(csr, B, H, T, N, d, s, coef_dtype):
         assert np.all(np.isnan(mix[0, 0])) and np.all(np.isfinite(mix[0, 1:])) and np.all(np.isfinite(mix[1:]))
 
 
+def test_value_mix_table_cannot_overflow(csr):
+    """The value mix accumulates in 32-bit fixed point scaled from a bound on the table entries.
+    The bound must hold in the worst case: every entry of every token names the same atom, with
+    equal coefficients and equal weights, so one table entry receives everything."""
+    B, H, T, N, d, s = 2, 3, 40000, 512, 64, 64
+    rng = np.random.default_rng(5)
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    idx = np.full((B, T, s), 7, dtype=np.int32)
+    idx[1] = 300
+    coef = np.full((B, T, s), 2.5, dtype=np.float32)
+    coef[1] *= -1.0
+    W = np.ones((B, H, T), dtype=np.float32)
+    it = torch.from_numpy(idx.astype(np.uint16).view(np.int16)).to(DEV).view(torch.uint16)
+    mix = csr.csr_value_mix(torch.from_numpy(D).to(DEV), torch.from_numpy(W).to(DEV), it,
+                            torch.from_numpy(coef).to(DEV).to(torch.float16)).cpu().numpy()
+    want = np.stack([np.tile(2.5 * s * T * D[7].astype(np.float64), (H, 1)), np.tile(-2.5 * s * T * D[300].astype(np.float64), (H, 1))])
+    assert np.all(np.abs(mix - want) <= 1e-6 * 2.5 * s * T)
+
+
 def test_scores_from_codes_equal_scores_from_the_restored_tensor(csr):
     """End to end on key-like data: encode, then q . x~ from the codes equals q . x~ from the
     de-sparse kernel's output (fp32), to fp32 rounding."""
