@@ -394,7 +394,8 @@ value_scatter_kernel(int N, const float* __restrict__ W, int B, int H, const uin
             }
             umax = block_max(umax, red);
             float scale[HGP], inv_scale[HGP];
-            bool fixed_point = umax < INFINITY;
+            // (the half-unit roundings of the terms must stay far inside the range too)
+            bool fixed_point = umax < INFINITY && (c1 - c0) * CHUNK_T * static_cast<int64_t>(s) <= (1ll << 30);
 #pragma unroll
             for (int h = 0; h < HGP; ++h) {
                 const float S = block_sum(sw[h], red);
