@@ -72,12 +72,14 @@ constexpr int GB = 64;
 template <int D_>
 struct DivSmem {
     float DiT[D_][GB + 4];     // [channel][atom i]
-    float DjT[D_][GB + 4];     // [channel][atom j]
+    float DjT[D_][GB + 4];     // [channel][atom j]; once the block of G is in registers its first
+                               // GB rows hold (G - I) transposed, [atom j][atom i]
     float Dj[GB][D_ + 4];      // [atom j][channel]
-    float GsT[GB][GB + 4];     // (G - I) transposed: [atom j][atom i]
 };
+// gridDim.y halves of the atoms j share a block of atoms i; each adds its part of the gradient
+// (two addends on zeroed memory: the sum does not depend on which comes first).
 template <int D_>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div, double* __restrict__ losses) {
     extern __shared__ __align__(16) unsigned char div_raw[];
     DivSmem<D_>& sm = *reinterpret_cast<DivSmem<D_>*>(div_raw);
@@ -107,7 +109,7 @@ div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div
     };
     gload(i0);
     sstore(sm.DiT, false);
-    gload(0);
+    gload((int)((int64_t)((N + GB - 1) / GB) * blockIdx.y / gridDim.y) * GB);
     // G block: thread owns rows pr .. pr+3, columns pc .. pc+3; gradient block: rows pr .. pr+3,
     // channels tx*4 .. +3 (and 64 + tx*4 .. +3 when d = 128)
     const int tx = tid & 15, pr = (tid >> 4) * 4, pc = tx * 4;
@@ -117,11 +119,14 @@ div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div
 #pragma unroll
         for (int c = 0; c < CPT; ++c) acc[a][c] = 0.f;
     double lsum = 0.0;
-    for (int j0 = 0; j0 < N; j0 += GB) {
+    float (*GsT)[GB + 4] = sm.DjT;
+    const int jblocks = (N + GB - 1) / GB;
+    const int jb0 = jblocks * blockIdx.y / gridDim.y, jb1 = jblocks * (blockIdx.y + 1) / gridDim.y;
+    for (int j0 = jb0 * GB; j0 < jb1 * GB; j0 += GB) {
         __syncthreads();                                   // the previous tile has been used
         sstore(sm.DjT, true);
         __syncthreads();
-        if (j0 + GB < N) gload(j0 + GB);
+        if (j0 + GB < jb1 * GB) gload(j0 + GB);
         float g[4][4];
 #pragma unroll
         for (int a = 0; a < 4; ++a)
@@ -138,6 +143,7 @@ div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div
 #pragma unroll
                 for (int b = 0; b < 4; ++b) g[a][b] = fmaf(x[a], y[b], g[a][b]);
         }
+        __syncthreads();                                   // every thread is done with DjT
 #pragma unroll
         for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -145,14 +151,14 @@ div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div
                 const int i = i0 + pr + a, j = j0 + pc + b;
                 float v = g[a][b] - (i == j ? 1.f : 0.f);
                 if (i >= N || j >= N) v = 0.f;
-                sm.GsT[pc + b][pr + a] = v;
+                GsT[pc + b][pr + a] = v;
                 lsum += (double)v * (double)v;
             }
         __syncthreads();
         // acc[row][c] += sum_j (G - I)[row][j] * Dj[j][c]
 #pragma unroll 4
         for (int j = 0; j < GB; ++j) {
-            const float4 wv = *reinterpret_cast<const float4*>(&sm.GsT[j][pr]);
+            const float4 wv = *reinterpret_cast<const float4*>(&GsT[j][pr]);
             const float w[4] = {wv.x, wv.y, wv.z, wv.w};
             float dch[CPT];
 #pragma unroll
@@ -175,10 +181,7 @@ div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div
         if (i0 + pr + a >= N) continue;
         float* dst = grad_div + (int64_t)(i0 + pr + a) * D_;
 #pragma unroll
-        for (int q = 0; q < CPT / 4; ++q)
-            *reinterpret_cast<float4*>(dst + q * 64 + tx * 4) =
-                make_float4(scale * acc[a][4 * q + 0], scale * acc[a][4 * q + 1], scale * acc[a][4 * q + 2],
-                            scale * acc[a][4 * q + 3]);
+        for (int c = 0; c < CPT; ++c) atomicAdd(dst + (c >> 2) * 64 + tx * 4 + (c & 3), scale * acc[a][c]);
     }
     for (int o = 16; o; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
     if ((tid & 31) == 0) atomicAdd(&losses[1], lsum / ((double)N * (double)N));
@@ -221,7 +224,9 @@ int run(const TrainArgs& a) {
     const size_t smem = sizeof(DivSmem<D_>);
     e = cudaFuncSetAttribute(div_grad_kernel<D_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    div_grad_kernel<D_><<<(a.N + GB - 1) / GB, 256, smem, a.stream>>>(a.D, a.N, a.grad_div, a.losses);
+    e = cudaMemsetAsync(a.grad_div, 0, gbytes, a.stream);
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    div_grad_kernel<D_><<<dim3((a.N + GB - 1) / GB, 2), 256, smem, a.stream>>>(a.D, a.N, a.grad_div, a.losses);
     update_kernel<D_><<<(a.N + 7) / 8, 256, 0, a.stream>>>(a.D, a.N, a.grad_mse, a.grad_div, a.lr, a.beta);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "dict_train launch: %s", cudaGetErrorString(e));
