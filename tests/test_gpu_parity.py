@@ -275,6 +275,23 @@ def test_fast_few_rows_split_dictionary_path(csr, M, N, d, s, kind, monkeypatch)
         assert rep.ok, rep.detail
 
 
+@pytest.mark.parametrize("G", [1, 2, 4, 8])
+@pytest.mark.parametrize("M,d", [(100, 128), (1000, 128), (40, 64)])
+def test_fast_few_rows_every_group_size(csr, G, M, d, monkeypatch):
+    """The clustered kernels exist for every arg-max group size: with the group size fixed, few
+    rows must get the codes of the one-CTA-per-row-pair kernel bit for bit."""
+    rng = np.random.default_rng(G * 1000 + M)
+    N, s = 8192, 6
+    Dd = torch.from_numpy(wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))).to(DEV)
+    Xd = torch.from_numpy(rng.standard_normal((M, d)).astype(np.float32)).to(DEV).to(torch.bfloat16)
+    monkeypatch.setenv("CSR_FAST_GROUP", str(G))
+    i1, c1 = csr.csr_encode_ex(Dd, Xd, s)
+    monkeypatch.setenv("CSR_FAST_NO_SPLIT", "1")
+    i2, c2 = csr.csr_encode_ex(Dd, Xd, s)
+    assert csr.csr_device_status() == csr.CSR_OK
+    assert np.array_equal(_np_idx(i1), _np_idx(i2)) and torch.equal(c1, c2)
+
+
 @pytest.mark.parametrize("M", [16, 1024, 70000])
 def test_encode_captured_in_a_cuda_graph(csr, M):
     """A decoding loop replays its step as a CUDA graph: after one ordinary call (which sizes
