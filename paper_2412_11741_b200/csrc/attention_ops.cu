@@ -116,8 +116,10 @@ ad_kernel(const float* __restrict__ D, int N, const float* __restrict__ A, int R
         for (int pc = 0; pc < pieces; ++pc) {
 #pragma unroll
             for (int u = 0; u < AV; ++u) {
-                const int f = tid + u * NT;               // float4 index: row = f / 16, atoms 4 * (f % 16) ..
-                const int r = r0 + f / (OA / 4), n = n0 + 4 * (f % (OA / 4));
+                // float4 index: consecutive lanes take consecutive rows (the transposed stores
+                // below are then free of bank conflicts), atoms 4 * (f / 64) ..
+                const int f = tid + u * NT;
+                const int r = r0 + f % OR, n = n0 + 4 * (f / OR);
                 if (r >= R || n >= ne) continue;
                 const float* src = A + (((int64_t)(r / H) * pieces + pc) * H + r % H) * N + n;
                 float4 v;
@@ -147,7 +149,7 @@ ad_kernel(const float* __restrict__ D, int N, const float* __restrict__ A, int R
 #pragma unroll
         for (int u = 0; u < AV; ++u) {
             const int f = tid + u * NT;
-            const int r = f / (OA / 4), a4 = 4 * (f % (OA / 4));
+            const int r = f % OR, a4 = 4 * (f / OR);
             sm.As[a4 + 0][r] = av[u].x;
             sm.As[a4 + 1][r] = av[u].y;
             sm.As[a4 + 2][r] = av[u].z;

@@ -91,7 +91,7 @@ div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div
     auto gload = [&](int r0) {
 #pragma unroll
         for (int u = 0; u < V; ++u) {
-            const int f = tid + u * 256, r = f / (D_ / 4), c4 = f % (D_ / 4);
+            const int f = tid + u * 256, r = f % GB, c4 = f / GB;     // lanes along the atoms: see sstore
             st[u] = (r0 + r < N) ? *reinterpret_cast<const float4*>(D + (int64_t)(r0 + r) * D_ + 4 * c4)
                                  : make_float4(0.f, 0.f, 0.f, 0.f);
         }
@@ -99,7 +99,9 @@ div_grad_kernel(const float* __restrict__ D, int N, float* __restrict__ grad_div
     auto sstore = [&](float (*T)[GB + 4], bool row_major) {
 #pragma unroll
         for (int u = 0; u < V; ++u) {
-            const int f = tid + u * 256, r = f / (D_ / 4), c4 = f % (D_ / 4);
+            // consecutive lanes hold consecutive atoms of the same four channels, so the four
+            // transposed stores and the row-major one are free of bank conflicts
+            const int f = tid + u * 256, r = f % GB, c4 = f / GB;
             T[4 * c4 + 0][r] = st[u].x;
             T[4 * c4 + 1][r] = st[u].y;
             T[4 * c4 + 2][r] = st[u].z;
