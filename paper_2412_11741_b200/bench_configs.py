@@ -155,15 +155,32 @@ def run_attention_case(reps):
         i, c, _, sc = nxt()
         csr.csr_decode_attention(D, D, Q, i, c, i, c, 1.0 / d ** 0.5, weights=sc, out=out)
 
+    # one layer's whole decoding step: the B new K rows and B new V rows are encoded (two
+    # dictionaries, handles, one grouped call), then the attention over the coded cache
+    D2 = torch.nn.functional.normalize(D.flip(0) + 0.5 * D, dim=1).contiguous()
+    hk, hv = csr.csr_dict_create(D), csr.csr_dict_create(D2)
+    k_new = torch.randn((B, d), device=dev, generator=g).to(torch.bfloat16)
+    v_new = torch.randn((B, d), device=dev, generator=g).to(torch.bfloat16)
+    ni = [torch.empty((B, s), dtype=torch.uint16, device=dev) for _ in range(2)]
+    nc = [torch.empty((B, s), dtype=torch.float16, device=dev) for _ in range(2)]
+
+    def f_step():
+        i, c, _, sc = nxt()
+        csr.csr_encode_grouped([(D, k_new, s, ni[0], nc[0], hk), (D2, v_new, s, ni[1], nc[1], hv)])
+        csr.csr_decode_attention(D, D2, Q, i, c, i, c, 1.0 / d ** 0.5, weights=sc, out=out)
+
     t_sc = _time(f_scores, reps)
     t_mx = _time(f_mix, reps)
     t_rc = _time(f_restore, reps)
     t_da = _time(f_attention, reps)
+    t_st = _time(f_step, reps)
+    csr.csr_dict_destroy(hk)
+    csr.csr_dict_destroy(hv)
     code_b, sw_b = B * T * s * 4.0, B * H * T * 4.0
     return {"case": "attention_from_codes", "B": B, "H": H, "T": T, "N": N, "d": d, "s": s,
             "key_scores_ms": round(t_sc, 4), "key_scores_hbm_gbs": (code_b + sw_b) / (t_sc * 1e-3) / 1e9,
             "value_mix_ms": round(t_mx, 4), "value_mix_hbm_gbs": (code_b + sw_b) / (t_mx * 1e-3) / 1e9,
-            "decode_attention_ms": round(t_da, 4), "restore_to_bf16_ms": round(t_rc, 4), "restored_bytes": B * T * d * 2.0, "code_bytes": code_b}
+            "decode_attention_ms": round(t_da, 4), "encode_new_rows_plus_attention_ms": round(t_st, 4), "restore_to_bf16_ms": round(t_rc, 4), "restored_bytes": B * T * d * 2.0, "code_bytes": code_b}
 
 
 def run_train_case(reps):
