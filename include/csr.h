@@ -249,8 +249,13 @@ int csr_dict_append(void* D, int N_cur, int N_cap, int d, const void* X, int x_d
  *     terms added in stored order g = 0 .. s-1 in fp32.  Q is [B][H][d], q_dtype F32, BF16 or F16;
  *     scores is [B][H][T] fp32 (before softmax).
  * csr_value_mix:   out[b][h][:] = sum_t W[b][h][t] * X~_V[b][t][:],
- *     W is [B][H][T] fp32 (attention weights), out is [B][H][d] fp32.  Accumulated with
- *     atomic fp32 adds: results are reproducible to rounding, not bit for bit.
+ *     W is [B][H][T] fp32 (attention weights; any finite values, not only softmax rows),
+ *     out is [B][H][d] fp32.  The per-atom sums a[n] = sum over (t, g) with idx = n of
+ *     W[t] * coef[t][g] are accumulated in 32-bit fixed point scaled to the largest value a
+ *     sum can reach (each term is rounded once to fp32 and once to a grid no coarser than
+ *     2^-29 of that bound), then out = a D in fp32 in a fixed order: the result is the same
+ *     bits on every run.  A NaN or Inf weight or coefficient is carried through fp32 sums
+ *     instead and reaches the outputs of its stream.
  *
  * idx and coef are [B][T][s] (coef_dtype F16 or F32); an idx >= N is clamped to N-1.
  * Limits: d in {64, 128}, 1 <= N <= 49152 (one head's N partial products must fit in
