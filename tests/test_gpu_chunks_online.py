@@ -161,6 +161,8 @@ def test_online_atoms_match_oracle_and_are_used_by_the_encoder(csr, d, dtype):
 @pytest.mark.parametrize("B,H,T,N,d,s,coef_dtype", [
     (3, 4, 5000, 2048, 128, 8, torch.float16), (2, 1, 1500, 8192, 128, 16, torch.float32),
     (2, 8, 700, 1024, 64, 4, torch.float16), (1, 9, 300, 16384, 128, 3, torch.float32), (2, 2, 0, 256, 64, 2, torch.float16),
+    (1, 4, 20000, 1024, 128, 8, torch.float16),       # one stream cut into many token ranges
+    (200, 2, 1100, 512, 64, 4, torch.float16),        # more streams than SMs
 ])
 def test_attention_from_codes_matches_oracle(csr, B, H, T, N, d, s, coef_dtype):
     """Scores and weighted value sums computed straight from the codes against the oracle,
