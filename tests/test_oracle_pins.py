@@ -381,6 +381,44 @@ def test_attention_from_codes_closed_forms():
     assert np.allclose(sc[0, 0] + res.residual @ q[0, 0], X.astype(np.float64) @ q[0, 0], atol=1e-12)
 
 
+def test_decode_attention_is_dense_softmax_attention_of_the_restored_cache():
+    """decode_attention against the textbook: restore K and V as dense matrices with a plain
+    matrix product of a scattered code matrix (not the oracle's reconstruct), then
+    softmax(scale * q K^T) V with scipy's softmax.  The weights are rows of a distribution;
+    with one key far ahead of the rest the output is that token's restored value row."""
+    from scipy.special import softmax
+    rng = np.random.default_rng(21)
+    B, H, T, s, d, N = 2, 3, 50, 4, 16, 40
+    Dk = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    Dv = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    ki, vi = rng.integers(0, N, (B, T, s)).astype(np.int32), rng.integers(0, N, (B, T, s)).astype(np.int32)
+    kc, vc = rng.standard_normal((B, T, s)), rng.standard_normal((B, T, s))
+    Q = rng.standard_normal((B, H, d))
+    out, w = orc.decode_attention(Dk, Dv, Q, ki, kc, vi, vc, scale=0.25)
+
+    def dense(D, idx, coef):                              # [B][T][d] from a [T][N] code matrix times D
+        X = np.zeros((B, T, d))
+        for b in range(B):
+            R = np.zeros((T, N))
+            np.add.at(R, (np.repeat(np.arange(T), s), idx[b].ravel()), coef[b].ravel())
+            X[b] = R @ D.astype(np.float64)
+        return X
+
+    K, V = dense(Dk, ki, kc), dense(Dv, vi, vc)
+    want_w = softmax(0.25 * np.einsum("bhd,btd->bht", Q, K), axis=2)
+    assert np.allclose(w, want_w, atol=1e-12) and np.allclose(w.sum(2), 1.0, atol=1e-12)
+    assert np.allclose(out, np.einsum("bht,btd->bhd", want_w, V), atol=1e-12)
+    # one key per stream with a huge score: the output is that token's restored value row
+    kc2 = kc.copy()
+    ki2 = ki.copy()
+    ki2[:, 7, :] = 3
+    kc2[:, 7, :] = 0.0
+    kc2[:, 7, 0] = 1.0                                     # K[7] = atom 3
+    Q2 = np.broadcast_to(1e4 * Dk[3].astype(np.float64), (B, H, d)).copy()
+    out2, w2 = orc.decode_attention(Dk, Dv, Q2, ki2, kc2 * np.where(np.arange(T)[None, :, None] == 7, 1.0, 1e-3), vi, vc, scale=1.0)
+    assert np.allclose(w2[:, :, 7], 1.0, atol=1e-9) and np.allclose(out2, V[:, None, 7, :], atol=1e-6)
+
+
 # ---------------------------------------------------------------------------------------
 # one training step of the offline dictionary
 # ---------------------------------------------------------------------------------------
