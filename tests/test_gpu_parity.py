@@ -237,7 +237,8 @@ def test_fast_any_dictionary_size(csr, N, G, monkeypatch):
                                           (2000, 4096, 64, 8, "f16"), (9000, 2048, 128, 4, "bf16"), (16, 65536, 64, 3, "bf16"),
                                           (24500, 65536, 128, 2, "bf16"),      # more row pairs than clusters fit at once
                                           (16, 4096, 128, 8, "bf16"), (100, 6144, 128, 5, "f32"), (64, 2048, 64, 4, "f16"),
-                                          (128, 16384, 128, 6, "bf16"), (129, 8192, 128, 4, "bf16")])   # one row tile: 1, 1-2, 1, 4 tiles per CTA; just over
+                                          (128, 16384, 128, 6, "bf16"), (129, 8192, 128, 4, "bf16"),    # one row tile: 1, 1-2, 1, 4 tiles per CTA; just over
+                                          (5, 300, 128, 3, "bf16"), (130, 600, 64, 2, "f32"), (7, 257, 64, 9, "f16")])   # two or three dictionary tiles
 def test_fast_few_rows_split_dictionary_path(csr, M, N, d, s, kind, monkeypatch):
     """Few rows: the dictionary is split across the CTAs of a cluster (one launch) or, without
     clusters, across CTAs with one sweep and one pick launch per iteration.  Both must return
