@@ -448,7 +448,7 @@ value_scatter_kernel(int N, const float* __restrict__ W, int B, int H, const uin
 }
 
 // Softmax over the T scores of one (stream, head) row, in place; one CTA per row, fp32, the
-// maximum subtracted first.  Rows are a few tens of KB and were just written: they come
+// maximum subtracted first; the row is read three times (maximum, sum, result) and written once.  Rows are a few tens of KB and were just written: they come
 // from L2.
 __global__ void __launch_bounds__(NT)
 softmax_rows_kernel(float* __restrict__ S, int64_t T) {
@@ -469,11 +469,7 @@ softmax_rows_kernel(float* __restrict__ S, int64_t T) {
     __syncthreads();
     mx = bcast;
     float sum = 0.f;
-    for (int64_t t = threadIdx.x; t < T; t += NT) {
-        const float e = __expf(row[t] - mx);
-        row[t] = e;
-        sum += e;
-    }
+    for (int64_t t = threadIdx.x; t < T; t += NT) sum += __expf(row[t] - mx);
     for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     __syncthreads();
     if (lane == 0) red[warp] = sum;
@@ -485,7 +481,7 @@ softmax_rows_kernel(float* __restrict__ S, int64_t T) {
     }
     __syncthreads();
     const float inv = bcast;
-    for (int64_t t = threadIdx.x; t < T; t += NT) row[t] *= inv;
+    for (int64_t t = threadIdx.x; t < T; t += NT) row[t] = __expf(row[t] - mx) * inv;
 }
 
 // Query heads whose N-vectors fit in shared memory side by side: 8, 4, 2 or 1 (0 = none fits).
