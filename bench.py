@@ -37,7 +37,7 @@ WORKLOAD = "gqa_long_context: 8 seq x 16384 tok x 8 kv_heads x {K,V}, d=128, M=2
 
 # dram__bytes_read.sum + dram__bytes_write.sum of encode_fast_kernel<128, 1, 0> at M = 524288, N = 8192,
 # s = 16 (profiles/encode_fast_small_case_ncu_full.md), per row; traffic grows in proportion to M.
-DRAM_BYTES_PER_ROW_NCU = (137.349376e6 + 20.825344e6) / 524288
+DRAM_BYTES_PER_ROW_NCU = (137.220352e6 + 19.116288e6) / 524288
 
 
 def _peaks():
