@@ -1,6 +1,9 @@
 """Throughput and reconstruction error of the codec on every synthetic configuration.
 
-  python -m paper_2412_11741_b200.bench_configs [--configs c1,c2,c3,c4,c5,decode,attention,train,pack] [--reps 30]
+  python bench_configs.py [--configs c1,c2,c3,c4,c5,decode,attention,train,pack] [--reps 30] [--rows M] [--exact-rows E]
+
+(`c5d64`, `c5n2048` ... `c5n16384`, `c4s4` ... `c4s32` name single cases; --rows shortens a case to
+its first M rows, for profiler captures of one kernel.)
 
 One JSON line per case: vectors/s and TFLOP/s of the fast encoder (median of the last two
 thirds of `reps` back-to-back launches, i.e. after the clocks have settled under the power
@@ -16,8 +19,13 @@ import json
 
 import torch
 
-from . import binding as csr
-from . import build, workloads as wl
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+
+from paper_2412_11741_b200 import binding as csr  # noqa: E402
+from paper_2412_11741_b200 import build, workloads as wl  # noqa: E402
 
 
 def _median_tail(xs):
@@ -38,8 +46,10 @@ def _time(fn, reps):
     return _median_tail([a.elapsed_time(b) for a, b in ev])
 
 
-def run_case(w, reps, exact_rows=16384):
+def run_case(w, reps, exact_rows=16384, rows=0):
     dev = torch.device("cuda", torch.cuda.current_device())
+    if rows and rows < w.M:
+        w.X = w.X[:rows]
     M, N, d, s = w.M, w.N, w.d, w.s
     D = torch.from_numpy(w.D).to(dev)
     X = torch.from_numpy(w.X).to(dev)
@@ -60,10 +70,12 @@ def run_case(w, reps, exact_rows=16384):
         xs = X[r0:r0 + step].float()
         err_sum += float(((xh[r0:r0 + step].float() - xs).norm(dim=1) / xs.norm(dim=1).clamp_min(1e-30)).sum())
     me = min(M, exact_rows)
-    Xe = X[:me].contiguous()
-    ie = torch.empty((me, s), dtype=torch.uint16, device=dev)
-    ce = torch.empty((me, s), dtype=torch.float32, device=dev)
-    ex_ms = _time(lambda: csr.csr_encode_ex(D, Xe, s, mode=csr.CSR_MODE_FP32_EXACT, out_idx=ie, out_coef=ce), 5)
+    ex_ms = float("nan")
+    if me > 0:
+        Xe = X[:me].contiguous()
+        ie = torch.empty((me, s), dtype=torch.uint16, device=dev)
+        ce = torch.empty((me, s), dtype=torch.float32, device=dev)
+        ex_ms = _time(lambda: csr.csr_encode_ex(D, Xe, s, mode=csr.CSR_MODE_FP32_EXACT, out_idx=ie, out_coef=ce), 5)
     flops = 2.0 * M * N * d * s
     return {
         "case": w.name, "M": M, "N": N, "d": d, "s": s, "x_dtype": w.x_dtype,
@@ -72,7 +84,7 @@ def run_case(w, reps, exact_rows=16384):
         "reconstruct_ms": round(rec_ms, 4),
         "reconstruct_hbm_gbs": M * (4 * s + 2 * d) / (rec_ms * 1e-3) / 1e9,
         "reconstruct_l2_gather_gbs": M * s * d * 4 / (rec_ms * 1e-3) / 1e9,
-        "exact_mode_vectors_per_s": me / (ex_ms * 1e-3), "exact_mode_rows": me,
+        "exact_mode_vectors_per_s": me / (ex_ms * 1e-3) if me else None, "exact_mode_rows": me,
     }
 
 
@@ -226,6 +238,12 @@ def cases(names):
             for N in (2048, 4096, 8192, 16384):
                 yield wl.dict_sweep(N)
             yield wl.dict_sweep(4096, d=64)
+        elif n == "c5d64":
+            yield wl.dict_sweep(4096, d=64)
+        elif n.startswith("c5n"):
+            yield wl.dict_sweep(int(n[3:]))
+        elif n.startswith("c4s"):
+            yield wl.sparsity_sweep(int(n[3:]))
         else:
             raise SystemExit(f"unknown configuration {n}")
 
@@ -234,13 +252,15 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="c1,c2,c3,c4,c5,decode,attention,train,pack")
     ap.add_argument("--reps", type=int, default=30)
+    ap.add_argument("--rows", type=int, default=0, help="use only the first ROWS rows of each encode case")
+    ap.add_argument("--exact-rows", type=int, default=16384, help="rows given to the fp32-exact encoder (0 = skip it)")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device (there is no CPU fallback)")
     build.build()
     names = args.configs.split(",")
     for w in cases([n for n in names if n not in ("decode", "attention", "train", "pack")]):
-        print(json.dumps(run_case(w, args.reps)), flush=True)
+        print(json.dumps(run_case(w, args.reps, args.exact_rows, args.rows)), flush=True)
     if "decode" in names:
         for seqs, kv_heads in ((1, 8), (8, 8), (64, 8)):
             print(json.dumps(run_decode_case(seqs, kv_heads, 8192, 16, args.reps)), flush=True)
