@@ -91,7 +91,6 @@ def run_case(w, reps, exact_rows=16384, rows=0):
 def run_decode_case(seqs, kv_heads, N, s, reps):
     """Latency of encoding the vectors ONE decoding step adds (seqs x kv_heads x {K, V} rows of
     d = 128) in each mode."""
-    import os
     dev = torch.device("cuda", torch.cuda.current_device())
     w = wl.gqa_long(tokens=1, N=N, s=s, seqs=seqs, kv_heads=kv_heads)
     D = torch.from_numpy(w.D).to(dev)
@@ -102,16 +101,15 @@ def run_decode_case(seqs, kv_heads, N, s, reps):
     coef = torch.empty((M, s), dtype=torch.float16, device=dev)
     out = {"case": f"decode_step_{seqs}x{kv_heads}x2", "M": M, "N": N, "d": w.d, "s": s}
     out["exact_split_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, X, s, mode=csr.CSR_MODE_FP32_EXACT, out_idx=idx, out_coef=coef), reps)
-    os.environ["CSR_EXACT_NO_SPLIT"] = "1"
+    csr.csr_set_option("exact_split", 1)
     out["exact_row_tile_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, X, s, mode=csr.CSR_MODE_FP32_EXACT, out_idx=idx, out_coef=coef), 3)
-    del os.environ["CSR_EXACT_NO_SPLIT"]
+    csr.csr_set_option("exact_split", 0)
     out["fast_cluster_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, Xb, s, out_idx=idx, out_coef=coef), reps)
-    os.environ["CSR_FAST_NO_CLUSTER"] = "1"
+    csr.csr_set_option("fast_split", 2)
     out["fast_split_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, Xb, s, out_idx=idx, out_coef=coef), reps)
-    del os.environ["CSR_FAST_NO_CLUSTER"]
-    os.environ["CSR_FAST_NO_SPLIT"] = "1"
+    csr.csr_set_option("fast_split", 1)
     out["fast_one_launch_us"] = 1e3 * _time(lambda: csr.csr_encode_ex(D, Xb, s, out_idx=idx, out_coef=coef), reps)
-    del os.environ["CSR_FAST_NO_SPLIT"]
+    csr.csr_set_option("fast_split", 0)
     # the step as a cache sees it: the K rows and the V rows (half of M each) against their own
     # dictionaries, one grouped call with dictionary handles
     D2 = torch.nn.functional.normalize(D.flip(0) + 0.5 * D, dim=1).contiguous()     # a second dictionary

@@ -14,14 +14,31 @@
  *     has finished on its stream.
  *   - Calls are asynchronous with respect to the host: work is enqueued on the given
  *     CUDA stream (the 8-argument forms use the legacy default stream, 0) and the
- *     function returns without synchronising, except csr_encode_host and
- *     csr_device_status, which synchronise.  A device-pointer call whose scratch does
- *     not have to grow (a repeat of an earlier call's shapes, or csr_encode_static) only
- *     launches kernels and may be captured into a CUDA graph and replayed.
+ *     function returns without synchronising, except the host entry points,
+ *     csr_dict_check_norms and csr_device_status, which synchronise.  A device-pointer
+ *     call whose scratch does not have to grow (a repeat of an earlier call's shapes, a
+ *     call with its own workspace or dictionary handle, or csr_encode_static) only
+ *     launches kernels and may be captured into a CUDA graph and replayed.  A call that
+ *     would have to grow the library's scratch while its stream is being captured is
+ *     refused with CSR_ERR_WORKSPACE (growing allocates); an outgrown scratch block is
+ *     kept until csr_release_workspace, so graphs captured earlier stay valid.
+ *   - Library-owned scratch.  Unless a call brings its own memory, it works in ONE
+ *     library-owned buffer per device: the fast mode's bf16 copy of D (csr_encode,
+ *     csr_encode_ex without `workspace` or `dict`), the few-rows paths' per-row maxima,
+ *     the per-atom tables of csr_key_scores / csr_value_mix / csr_decode_attention, the
+ *     codes and gradients of csr_dict_train_step, and one status word.  Calls that use it
+ *     must therefore be ORDERED on the device (same stream, or events between streams):
+ *     two of them running side by side on different streams overwrite each other's
+ *     scratch and return wrong results without any error.  Concurrent callers give each
+ *     encode its own `workspace` or `dict` and, for the wait status, its own
+ *     `dev_status`; such a call touches nothing the library owns.
  *   - Layout.  D is [N][d] row-major fp32: one atom per row, the d channels contiguous
  *     (the paper's d x N matrix of "Sparse representation", stored column by column).
- *     Atoms are assumed unit l2-norm; this is not checked and the formulas are applied
- *     as written if they are not.  X and X_hat are [M][d] row-major.  Codes are
+ *     Atoms are assumed unit l2-norm; the encoders do not check this and apply the
+ *     formulas as written if they are not (csr_dict_check_norms checks a dictionary once).
+ *     The exact mode's promise of fp64-identical picks assumes atom norms of at most
+ *     1 + 1e-3: its rounding band scales with the residual's norm only.
+ *     X and X_hat are [M][d] row-major.  Codes are
  *     idx [M][s] and coef [M][s] row-major, entry g of a row being iteration g of the
  *     pursuit.
  *   - Limits: d in {64, 128}; 1 <= N <= 65536 (indices are stored as uint16); 1 <= s <= 64;
@@ -40,7 +57,7 @@
 extern "C" {
 #endif
 
-#define CSR_VERSION 100
+#define CSR_VERSION 110
 
 #define CSR_OK 0
 #define CSR_ERR_INVALID_ARG (-1)
@@ -67,8 +84,7 @@ extern "C" {
  *                        tiles of 64 than half the SMs) the dictionary is split across
  *                        the SMs instead of the rows, two launches per iteration, with
  *                        identical codes; this path uses the library-owned scratch
- *                        (not taken when a caller workspace is given, or when the
- *                        environment variable CSR_EXACT_NO_SPLIT is set).
+ *                        (not taken when a caller workspace is given).
  *   CSR_MODE_BF16_FAST   correlations on the tcgen05 tensor cores with bf16 operands
  *                        (residual and atoms rounded to bf16) and fp32 accumulation.
  *                        Near-tied picks may differ from an fp64 evaluation; the mean
@@ -78,12 +94,9 @@ extern "C" {
  *                        as many pairs of 128-row tiles as SMs) the dictionary is split
  *                        across the CTAs of thread-block clusters that share the rows,
  *                        still one launch, with identical codes; where clusters cannot be
- *                        launched (or CSR_FAST_NO_CLUSTER is set) and the library-owned
- *                        scratch is in use, across CTAs with one sweep and one pick launch
- *                        per iteration (both off when the environment variable
- *                        CSR_FAST_NO_SPLIT is set).  The variable
- *                        CSR_FAST_GROUP (1, 2, 4 or 8) overrides the arg-max group size
- *                        the kernel would choose; every setting meets the same gates.
+ *                        launched and the library-owned scratch is in use, across CTAs
+ *                        with one sweep and one pick launch per iteration.
+ *                        (csr_set_option can force each of these paths.)
  */
 #define CSR_MODE_FP32_EXACT 0
 #define CSR_MODE_BF16_FAST 1
@@ -108,6 +121,10 @@ typedef struct csr_encode_params {
     int64_t ld_code;        /* elements between consecutive rows of out_idx and of out_coef;
                                0 = s (dense) */
     const void* dict;       /* csr_dict_t* from csr_dict_create, or NULL (see there) */
+    uint32_t* dev_status;   /* fast mode: optional device word (4-byte aligned) that the call zeroes
+                               on its stream and a kernel sets non-zero if one of its bounded
+                               waits expired; NULL = the library's word, read by
+                               csr_device_status.  Ignored by the host entry points. */
 } csr_encode_params_t;
 
 typedef struct csr_reconstruct_params {
@@ -283,8 +300,8 @@ int csr_value_mix(const void* D, int N, int d, const float* W, int B, int H, con
  * BEFORE the update; the paper's adaptive weight for the next batch is
  * beta = min(0.1 * L_MSE / L_div, 1.0), which the caller forms from them.  The optimiser is
  * a plain gradient step (the paper names none).  D is updated in place and must not be
- * used by other work on the device meanwhile.  Uses the library-owned scratch; asynchronous
- * on `stream`.  Gradient sums use atomic fp32 adds: reproducible to rounding.
+ * used by other work on the device meanwhile.  Uses the library-owned scratch (order it
+ * with the other users of that scratch); asynchronous on `stream`.  Gradient sums use atomic fp32 adds: reproducible to rounding.
  */
 typedef struct csr_train_params {
     uint32_t struct_size;   /* sizeof(csr_train_params_t) */
@@ -306,7 +323,10 @@ int csr_dict_train_step(const csr_train_params_t* p);
  * out_coef are host pointers, ideally page-locked).  X is copied to the device in
  * chunks that overlap with the encoding of the previous chunk, the codes are copied
  * back, and the function returns after everything has finished.  D stays a device
- * pointer.  Uses library-owned device staging buffers (grow-only, per device).
+ * pointer.  Uses library-owned device staging buffers (grow-only, per device) and two
+ * library-owned streams, which first wait for everything enqueued so far on params.stream
+ * (so a dictionary still being written there is complete before it is read); the fast
+ * mode's bf16 copy of D is made once per call.  dev_status is ignored.
  */
 int csr_encode_host(const csr_encode_params_t* p);
 
@@ -353,9 +373,41 @@ int csr_encode_static(const void* D, const void* X, int64_t M, int d, int N, int
                       void* out_coef, void* stream, uint32_t* dev_status);
 
 /*
+ * One-off check of the unit-norm assumption ("Sparse representation": the atoms of D are
+ * unit vectors; "NeuralDict": ReNorm restores that after every update).  Computes
+ * max_n | ||D[n]||_2 - 1 | in fp32 on `stream`, waits for it, stores it in *max_dev (host
+ * pointer, may be NULL) and returns CSR_ERR_INVALID_ARG if it exceeds `tol` (tol < 0: report
+ * only).  Not on the hot path: the encoders never call it.  Atoms normalised in fp32 are off
+ * by up to about 1e-7.  Uses a word of the library-owned scratch: order it like the
+ * other users of that scratch.
+ */
+int csr_dict_check_norms(const void* D, int N, int d, float tol, void* stream, float* max_dev);
+
+/*
+ * Process-wide tuning and diagnostic switches; none is needed in normal use (tests use them
+ * to drive every code path, measurements to compare them).  All paths return the same codes.
+ *   "fast_group"     0 (default: the library chooses) or 1, 2, 4, 8: atoms per arg-max group
+ *                    of the fast encoder's sweep;
+ *   "fast_split"     0 (default: few rows split the dictionary across thread-block
+ *                    clusters, else across CTAs with a launch pair per iteration),
+ *                    1 = always one CTA per pair of row tiles over the whole dictionary,
+ *                    2 = no clusters;
+ *   "exact_split"    0 (default: the exact mode splits the dictionary for few rows), 1 = never;
+ *   "wait_limit_ns"  bound of every device-side wait of the fast encoder in nanoseconds
+ *                    (default 2e9).  0 lets no wait outlast a single look at its barrier, so
+ *                    the first hand-off that is not already complete expires: the call
+ *                    returns, its outputs are unspecified and the status word reports
+ *                    CSR_ERR_TIMEOUT (how the expiry path is exercised).
+ * Takes effect for calls made afterwards; not synchronised with calls in flight on other
+ * host threads.  Returns CSR_ERR_INVALID_ARG for an unknown name or value.
+ */
+int csr_set_option(const char* name, int64_t value);
+
+/*
  * Synchronises the stream and reports whether a kernel of this library has given up on a
  * bounded wait since the last call of this function on the current device: CSR_OK or
- * CSR_ERR_TIMEOUT (or CSR_ERR_CUDA if the stream itself is in error).
+ * CSR_ERR_TIMEOUT (or CSR_ERR_CUDA if the stream itself is in error).  Reads the library's
+ * status word(s); a call that was given its own dev_status reports there instead.
  */
 int csr_device_status(void* stream);
 

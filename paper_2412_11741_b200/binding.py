@@ -34,7 +34,7 @@ CSR_MODE_BF16_FAST = 1
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
     "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_decode_attention", "csr_dict_append", "csr_dict_create", "csr_dict_destroy", "csr_dict_train_step", "csr_key_scores", "csr_pack_coefficients", "csr_value_mix",
-    "csr_encode_static", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
+    "csr_encode_static", "csr_dict_check_norms", "csr_set_option", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
 )
 
 
@@ -49,6 +49,7 @@ class csr_encode_params_t(ctypes.Structure):
         ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("ldx", ctypes.c_int64), ("ld_code", ctypes.c_int64),
         ("dict", ctypes.c_void_p),
+        ("dev_status", ctypes.c_void_p),
     ]
 
 
@@ -92,7 +93,7 @@ def lib() -> ctypes.CDLL:
             raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2412_11741_b200.build` "
                               "(there is no fallback path)")
         L = ctypes.CDLL(LIB_PATH)
-        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
+        vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float
         L.csr_encode.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp]
         L.csr_encode.restype = i32
         L.csr_encode_ex.argtypes = [ctypes.POINTER(csr_encode_params_t)]
@@ -115,7 +116,6 @@ def lib() -> ctypes.CDLL:
         L.csr_reconstruct_grouped.restype = i32
         L.csr_dict_append.argtypes = [vp, i32, i32, i32, vp, i32, i64, i64, vp, i32, vp]
         L.csr_dict_append.restype = i32
-        f32 = ctypes.c_float
         L.csr_key_scores.argtypes = [vp, i32, i32, vp, i32, i32, i32, vp, vp, i32, i64, i32, f32, vp, vp]
         L.csr_key_scores.restype = i32
         L.csr_value_mix.argtypes = [vp, i32, i32, vp, i32, i32, vp, vp, i32, i64, i32, vp, vp]
@@ -131,6 +131,10 @@ def lib() -> ctypes.CDLL:
         L.csr_dict_destroy.restype = i32
         L.csr_dict_train_step.argtypes = [ctypes.POINTER(csr_train_params_t)]
         L.csr_dict_train_step.restype = i32
+        L.csr_dict_check_norms.argtypes = [vp, i32, i32, f32, vp, ctypes.POINTER(f32)]
+        L.csr_dict_check_norms.restype = i32
+        L.csr_set_option.argtypes = [ctypes.c_char_p, i64]
+        L.csr_set_option.restype = i32
         L.csr_device_status.argtypes = [vp]
         L.csr_device_status.restype = i32
         L.csr_release_workspace.argtypes = []
@@ -224,9 +228,10 @@ def _encode_params(D, X, s, out_idx, out_coef, mode, stream, workspace) -> csr_e
 def csr_encode_ex(D: torch.Tensor, X: torch.Tensor, s: int, *, mode: int = CSR_MODE_BF16_FAST,
                   coef_dtype: torch.dtype = torch.float16, out_idx: Optional[torch.Tensor] = None,
                   out_coef: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-                  dict: Optional[int] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+                  dict: Optional[int] = None, dev_status: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """csr_encode_ex on CUDA tensors: D [N][d] fp32, X [M][d] fp32 or bf16.
-    Returns (idx [M][s] uint16, coef [M][s] coef_dtype); runs on torch's current stream."""
+    Returns (idx [M][s] uint16, coef [M][s] coef_dtype); runs on torch's current stream.
+    dev_status: optional int32/uint32 CUDA tensor of one element that receives the wait status."""
     assert D.is_cuda and X.is_cuda and D.is_contiguous() and X.dim() == 2 and X.stride(1) == 1
     assert D.dtype == torch.float32 and D.dim() == 2 and X.shape[1] == D.shape[1]
     M = X.shape[0]
@@ -237,6 +242,9 @@ def csr_encode_ex(D: torch.Tensor, X: torch.Tensor, s: int, *, mode: int = CSR_M
     p = _encode_params(D, X, s, out_idx, out_coef, mode, _stream_ptr(X), workspace)
     if dict is not None:
         p.dict = dict
+    if dev_status is not None:
+        assert dev_status.is_cuda and dev_status.element_size() == 4 and dev_status.numel() >= 1
+        p.dev_status = dev_status.data_ptr()
     with torch.cuda.device(X.device):
         _check(lib().csr_encode_ex(ctypes.byref(p)))
     return out_idx, out_coef
@@ -491,6 +499,21 @@ def csr_reconstruct(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor,
     with torch.cuda.device(D.device):
         _check(lib().csr_reconstruct(D.data_ptr(), idx.data_ptr(), coef.data_ptr(), M, d, N, s, X_hat.data_ptr()))
     return X_hat
+
+
+def csr_dict_check_norms(D: torch.Tensor, tol: float = -1.0) -> float:
+    """csr_dict_check_norms: returns max_n | ||D[n]|| - 1 | (synchronises torch's current stream);
+    raises CsrError if it exceeds tol (tol < 0: report only)."""
+    assert D.is_cuda and D.is_contiguous() and D.dtype == torch.float32 and D.dim() == 2
+    out = ctypes.c_float(0.0)
+    with torch.cuda.device(D.device):
+        _check(lib().csr_dict_check_norms(D.data_ptr(), D.shape[0], D.shape[1], float(tol), _stream_ptr(D), ctypes.byref(out)))
+    return float(out.value)
+
+
+def csr_set_option(name: str, value: int) -> None:
+    """csr_set_option: process-wide tuning / diagnostic switches (see include/csr.h)."""
+    _check(lib().csr_set_option(name.encode(), int(value)))
 
 
 def csr_device_status(device=None) -> int:

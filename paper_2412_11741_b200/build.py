@@ -1,15 +1,21 @@
-"""Builds libcsr.so (the C-ABI library) in-tree with nvcc for sm_100a."""
+"""Builds libcsr.so (the C-ABI library) in-tree with nvcc for sm_100a.
+
+Every .cu file under csrc/ is compiled to an object of its own (in parallel, only when it
+or a header is newer than its object) and the objects are linked into libcsr.so.
+"""
 from __future__ import annotations
 
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
+OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libcsr.so")
-SOURCES = ["attention_ops.cu", "csr_api.cu", "dict_ops.cu", "encode_exact.cu", "encode_exact_split.cu", "encode_fast.cu", "encode_static.cu", "reconstruct.cu", "train_ops.cu"]
+FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC"]
 
 
 def _nvcc() -> str:
@@ -19,29 +25,53 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def _sources():
+    return sorted(f for f in os.listdir(CSRC) if f.endswith(".cu"))
+
+
+def _headers():
+    return [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh")] + [os.path.join(ROOT, "include", "csr.h")]
+
+
+def _stale(target: str, deps) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "csr.h")]
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(d) > t for d in deps)
+
+
+def needs_build() -> bool:
+    return _stale(LIB, [os.path.join(CSRC, f) for f in _sources()] + _headers())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-           "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lcudart"]
-    if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
+    os.makedirs(OBJ, exist_ok=True)
+    nvcc, hdrs = _nvcc(), _headers()
+
+    def compile_one(src: str):
+        obj = os.path.join(OBJ, src[:-3] + ".o")
+        if not force and not _stale(obj, [os.path.join(CSRC, src)] + hdrs):
+            return obj, 0, ""
+        cmd = [nvcc] + FLAGS + (["-Xptxas=-v"] if verbose else []) + ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c",
+                                                                        os.path.join(CSRC, src), "-o", obj]
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        return obj, res.returncode, res.stdout + res.stderr
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        results = list(pool.map(compile_one, _sources()))
+    for _, rc, log in results:
+        if verbose or rc != 0:
+            sys.stderr.write(log)
+    if any(rc != 0 for _, rc, _ in results):
         raise RuntimeError("nvcc failed building libcsr.so")
+    res = subprocess.run([nvcc, "-shared", "-o", LIB] + [o for o, _, _ in results] + ["-lcudart"], capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("linking libcsr.so failed")
     return LIB
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force="-f" in sys.argv or "-v" in sys.argv, verbose="-v" in sys.argv))

@@ -16,6 +16,16 @@ int fail(int code, const char* fmt, ...);
 // Device status word written by kernels whose bounded waits expire.
 constexpr uint32_t kStatusTimeout = 1u;
 
+// Process-wide switches set through csr_set_option (plain loads on the call path).
+struct Options {
+    int fast_group;                     // 0 = chosen by the library; 1, 2, 4, 8 = atoms per arg-max group
+    int fast_split;                     // 0 = chosen by the library; 1 = one CTA per pair of row tiles over the whole
+                                        // dictionary; 2 = few rows split the dictionary without clusters
+    int exact_split;                    // 0 = chosen by the library; 1 = the row-tile encoder also with few rows
+    unsigned long long wait_limit_ns;   // bound of every device-side wait
+};
+Options options();
+
 struct EncodeArgs {
     const float* D;
     const void* X;
@@ -73,6 +83,9 @@ int launch_reconstruct(const ReconstructArgs& a);
 // D_new[i][:] = X[rows[i]][:] / ||X[rows[i]][:]||_2 for i < n_rows (zero rows stay zero).
 int launch_dict_append(float* D_new, int d, const void* X, int x_dtype, int64_t M, int64_t ldx, const int64_t* rows,
                        int n_rows, cudaStream_t stream);
+
+// *max_bits (zeroed by the caller) receives the bit pattern of max_n | ||D[n]||_2 - 1 |.
+int launch_dict_norm_deviation(const float* D, int N, int d, uint32_t* max_bits, cudaStream_t stream);
 
 // Attention straight from the codes.  key_scores: Q = queries [B][H][d] (q_dtype), out = scores
 // [B][H][T].  value_mix: Q = attention weights [B][H][T] fp32, out = [B][H][d] fp32.

@@ -1,11 +1,12 @@
 // C boundary of libcsr: argument checks, workspace management, stream plumbing.
 // Every computation is done by the kernels in the other translation units.
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -28,6 +29,20 @@ int fail(int code, const char* fmt, ...) {
     vsnprintf(g_err, sizeof(g_err), fmt, ap);
     va_end(ap);
     return code;
+}
+
+namespace {
+std::atomic<int> g_opt_fast_group{0}, g_opt_fast_split{0}, g_opt_exact_split{0};
+std::atomic<unsigned long long> g_opt_wait_limit_ns{2000000000ull};      // 2 s per wait
+}  // namespace
+
+Options options() {
+    Options o;
+    o.fast_group = g_opt_fast_group.load(std::memory_order_relaxed);
+    o.fast_split = g_opt_fast_split.load(std::memory_order_relaxed);
+    o.exact_split = g_opt_exact_split.load(std::memory_order_relaxed);
+    o.wait_limit_ns = g_opt_wait_limit_ns.load(std::memory_order_relaxed);
+    return o;
 }
 
 int sm_count() {
@@ -53,6 +68,8 @@ constexpr int kSideStreams = 3;
 struct DeviceBuffers {
     void* work = nullptr;      // [status word | encoder scratch]
     size_t work_bytes = 0;
+    std::vector<void*> retired;   // outgrown work buffers: kept until csr_release_workspace, because
+                                  // kernels already enqueued (or captured into a graph) still use them
     void* stage_x[2] = {nullptr, nullptr};   // host-entry staging: X chunks
     void* stage_idx[2] = {nullptr, nullptr};
     void* stage_coef[2] = {nullptr, nullptr};
@@ -77,23 +94,36 @@ int current_device(int* dev) {
 }
 
 // Returns the library's work buffer (status word first), grown to hold `scratch` bytes.
-int ensure_work(size_t scratch, void** base) {
+// A buffer that has to grow is replaced, never freed: work already enqueued and captured
+// graphs keep the block they were given (csr_release_workspace frees them all).  Growing
+// allocates, so it is refused while `stream` is being captured.
+int ensure_work(size_t scratch, void** base, cudaStream_t stream) {
     int dev;
     if (int rc = current_device(&dev)) return rc;
     std::lock_guard<std::mutex> lk(g_mu);
     DeviceBuffers& b = g_dev[dev];
     const size_t need = kStatusBytes + 1024 + scratch;
     if (b.work_bytes < need) {
-        if (b.work) {
-            cudaDeviceSynchronize();
-            cudaFree(b.work);
-            b.work = nullptr;
-            b.work_bytes = 0;
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) {
+            cudaGetLastError();
+            cap = cudaStreamCaptureStatusNone;
         }
-        cudaError_t e = cudaMalloc(&b.work, need);
+        if (cap != cudaStreamCaptureStatusNone)
+            return fail(CSR_ERR_WORKSPACE,
+                        "the library scratch would have to grow to %zu bytes during stream capture: make the same "
+                        "call once before capturing, or pass a workspace / dictionary handle",
+                        need);
+        void* fresh = nullptr;
+        cudaError_t e = cudaMalloc(&fresh, need);
         if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMalloc(%zu): %s", need, cudaGetErrorString(e));
-        e = cudaMemset(b.work, 0, kStatusBytes);
-        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemset: %s", cudaGetErrorString(e));
+        e = cudaMemset(fresh, 0, kStatusBytes);
+        if (e != cudaSuccess) {
+            cudaFree(fresh);
+            return fail(CSR_ERR_CUDA, "cudaMemset: %s", cudaGetErrorString(e));
+        }
+        if (b.work) b.retired.push_back(b.work);
+        b.work = fresh;
         b.work_bytes = need;
     }
     *base = b.work;
@@ -144,6 +174,7 @@ int check_encode(const csr_encode_params_t* p, bool host_io) {
         }
     }
     if (p->workspace && !aligned16(p->workspace)) return fail(CSR_ERR_ALIGNMENT, "workspace must be 16-byte aligned");
+    if (reinterpret_cast<uintptr_t>(p->dev_status) % 4) return fail(CSR_ERR_ALIGNMENT, "dev_status must be 4-byte aligned");
     return CSR_OK;
 }
 
@@ -262,8 +293,9 @@ int ensure_side_streams(DeviceBuffers** out) {
 }
 
 // Runs one encode on device pointers.  `shared_scratch` = false keeps the call off the parts of
-// the library-owned buffer that two encodes in flight would both write.
-int encode_device(const csr_encode_params_t* p, bool shared_scratch = true) {
+// the library-owned buffer that two encodes in flight would both write.  `prepared` (fast mode
+// only) is a bf16 copy of D made by the caller of this function: no conversion is enqueued.
+int encode_device(const csr_encode_params_t* p, bool shared_scratch = true, const void* prepared = nullptr) {
     if (p->M == 0) return CSR_OK;
     EncodeArgs a;
     a.D = static_cast<const float*>(p->D);
@@ -279,35 +311,50 @@ int encode_device(const csr_encode_params_t* p, bool shared_scratch = true) {
     a.ldx = p->ldx ? p->ldx : p->d;
     a.ld_code = p->ld_code ? p->ld_code : p->s;
     a.stream = static_cast<cudaStream_t>(p->stream);
+    const Options opt = options();
     if (p->mode == CSR_MODE_FP32_EXACT) {
         // few rows: split the dictionary across the SMs (library-owned scratch; a caller
         // workspace is sized for the fast mode only, so with one the row-tile encoder runs)
-        if (!p->workspace && encode_exact_split_applies(p->M, p->N) && !getenv("CSR_EXACT_NO_SPLIT")) {
+        if (!p->workspace && encode_exact_split_applies(p->M, p->N) && opt.exact_split == 0) {
             void* base = nullptr;
-            if (int rc = ensure_work(encode_exact_split_scratch_bytes(p->M, p->d, p->N), &base)) return rc;
+            if (int rc = ensure_work(encode_exact_split_scratch_bytes(p->M, p->d, p->N), &base, a.stream)) return rc;
             return launch_encode_exact_split(a, align_up(static_cast<char*>(base) + kStatusBytes, 1024));
         }
         return launch_encode_exact(a);
     }
 
+    // The word a kernel raises when one of its waits expires: the caller's, else the library's.
+    uint32_t* status = p->dev_status;
+    if (status) {
+        cudaError_t e = cudaMemsetAsync(status, 0, sizeof(uint32_t), a.stream);
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    }
     // few rows: the cluster path needs no scratch; its fallback (a launch pair per iteration)
     // does, and gets it from the library-owned buffer only (a caller workspace is sized for
     // the bf16 copy)
-    const bool split =
-        shared_scratch && !p->workspace && encode_fast_split_applies(p->M, p->N) && !getenv("CSR_FAST_NO_SPLIT");
+    const bool split = shared_scratch && !p->workspace && !prepared && encode_fast_split_applies(p->M, p->N) &&
+                       opt.fast_split != 1;
     const size_t dict_b = (encode_fast_workspace_bytes(p->d, p->N) + 1023) / 1024 * 1024;
     const size_t split_b = split ? encode_fast_split_scratch_bytes(p->M, p->d, p->N) : 0;
-    if (p->dict) {
-        const csr_dict* dc = static_cast<const csr_dict*>(p->dict);
-        int dev = -1;
-        if (int rc = current_device(&dev)) return rc;
-        if (dc->magic != kDictMagic) return fail(CSR_ERR_INVALID_ARG, "dict is not a live csr_dict_t handle");
-        if (dc->device != dev || dc->D != p->D || dc->N != p->N || dc->d != p->d)
-            return fail(CSR_ERR_INVALID_ARG, "dict was created for another device, D, N or d");
-        void* wbase = nullptr;
-        if (int rc = ensure_work(split_b, &wbase)) return rc;     // status word (+ split scratch)
-        void* sp = split ? align_up(static_cast<char*>(wbase) + kStatusBytes, 1024) : nullptr;
-        return launch_encode_fast_prepared(a, dc->bf16, static_cast<uint32_t*>(wbase), sp);
+    if (p->dict || prepared) {
+        const void* copy = prepared;
+        if (p->dict) {
+            const csr_dict* dc = static_cast<const csr_dict*>(p->dict);
+            int dev = -1;
+            if (int rc = current_device(&dev)) return rc;
+            if (dc->magic != kDictMagic) return fail(CSR_ERR_INVALID_ARG, "dict is not a live csr_dict_t handle");
+            if (dc->device != dev || dc->D != p->D || dc->N != p->N || dc->d != p->d)
+                return fail(CSR_ERR_INVALID_ARG, "dict was created for another device, D, N or d");
+            copy = dc->bf16;
+        }
+        void* sp = nullptr;
+        if (!status || split) {                               // library status word (+ split scratch)
+            void* wbase = nullptr;
+            if (int rc = ensure_work(split_b, &wbase, a.stream)) return rc;
+            if (!status) status = static_cast<uint32_t*>(wbase);
+            if (split) sp = align_up(static_cast<char*>(wbase) + kStatusBytes, 1024);
+        }
+        return launch_encode_fast_prepared(a, copy, status, sp);
     }
     void* base = nullptr;
     if (p->workspace) {
@@ -316,15 +363,26 @@ int encode_device(const csr_encode_params_t* p, bool shared_scratch = true) {
             return fail(CSR_ERR_WORKSPACE, "workspace of %zu bytes given, %lld needed", p->workspace_bytes,
                         (long long)need);
         base = p->workspace;
-        cudaError_t e = cudaMemsetAsync(base, 0, kStatusBytes, a.stream);
-        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+        if (!status) {
+            cudaError_t e = cudaMemsetAsync(base, 0, kStatusBytes, a.stream);
+            if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+        }
     } else {
-        if (int rc = ensure_work(dict_b + split_b, &base)) return rc;
+        if (int rc = ensure_work(dict_b + split_b, &base, a.stream)) return rc;
     }
-    uint32_t* status = static_cast<uint32_t*>(base);
+    if (!status) status = static_cast<uint32_t*>(base);
     char* scratch = static_cast<char*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024));
     if (int rc = prepare_fast_dictionary(a.D, a.N, a.d, scratch, a.stream)) return rc;
     return launch_encode_fast_prepared(a, scratch, status, split ? scratch + dict_b : nullptr);
+}
+
+// The host entry points run on two library streams; this makes both wait for whatever the
+// caller has enqueued on `user` so far (the dictionary may still be in the making there).
+int order_after(DeviceBuffers& b, cudaStream_t user) {
+    cudaError_t e = cudaEventRecord(b.ev_in[0], user);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(b.copy_streams[i], b.ev_in[0], 0);
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "ordering after the caller's stream: %s", cudaGetErrorString(e));
+    return CSR_OK;
 }
 
 }  // namespace
@@ -541,7 +599,7 @@ int csr_key_scores(const void* D, int N, int d, const void* Q, int q_dtype, int 
                static_cast<cudaStream_t>(stream)};
     if (B == 0 || T == 0) return CSR_OK;
     void* base = nullptr;
-    if (int rc = ensure_work(attn_scratch_bytes(B, H, N, T), &base)) return rc;
+    if (int rc = ensure_work(attn_scratch_bytes(B, H, N, T), &base, a.stream)) return rc;
     return launch_key_scores(a, static_cast<float*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)));
 }
 
@@ -553,7 +611,7 @@ int csr_value_mix(const void* D, int N, int d, const float* W, int B, int H, con
                static_cast<cudaStream_t>(stream)};
     if (B == 0) return CSR_OK;
     void* base = nullptr;
-    if (int rc = ensure_work(attn_scratch_bytes(B, H, N, T), &base)) return rc;
+    if (int rc = ensure_work(attn_scratch_bytes(B, H, N, T), &base, a.stream)) return rc;
     return launch_value_mix(a, static_cast<float*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)));
 }
 
@@ -593,7 +651,7 @@ int csr_dict_train_step(const csr_train_params_t* p) {
     const size_t coef_b = ((size_t)p->M * p->s * 4 + 255) / 256 * 256;
     const size_t g_b = ((size_t)p->N * p->d * 4 + 255) / 256 * 256;
     void* base = nullptr;
-    if (int rc = ensure_work(enc + idx_b + coef_b + 2 * g_b, &base)) return rc;
+    if (int rc = ensure_work(enc + idx_b + coef_b + 2 * g_b, &base, static_cast<cudaStream_t>(p->stream))) return rc;
     char* q = static_cast<char*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)) + enc;
     TrainArgs a;
     a.D = static_cast<float*>(p->D);
@@ -643,9 +701,25 @@ int csr_encode_host(const csr_encode_params_t* p) {
     const int64_t chunk = host_chunk_rows(p->M);
     DeviceBuffers& b = g_dev[dev];
     if (int rc = ensure_staging(b, (size_t)chunk * xb, (size_t)chunk * (cb > ib ? cb : ib))) return rc;
+    if (int rc = order_after(b, static_cast<cudaStream_t>(p->stream))) return rc;
+    const int64_t n_chunks = (p->M + chunk - 1) / chunk;
+    // Several chunks in the fast mode: the bf16 copy of D is made once, on the first stream, and
+    // the second stream waits for it (one conversion per chunk into the one buffer, from two
+    // streams, would have each stream rewrite what the other's kernel is reading).
+    const void* prepared = nullptr;
+    if (p->mode == CSR_MODE_BF16_FAST && !p->dict && n_chunks > 1) {
+        void* base = nullptr;
+        if (int rc = ensure_work((encode_fast_workspace_bytes(p->d, p->N) + 1023) / 1024 * 1024, &base, b.copy_streams[0]))
+            return rc;
+        void* copy = align_up(static_cast<char*>(base) + kStatusBytes, 1024);
+        if (int rc = prepare_fast_dictionary(static_cast<const float*>(p->D), p->N, p->d, copy, b.copy_streams[0])) return rc;
+        cudaError_t e = cudaEventRecord(b.ev_in[1], b.copy_streams[0]);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(b.copy_streams[1], b.ev_in[1], 0);
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "dictionary copy hand-over: %s", cudaGetErrorString(e));
+        prepared = copy;
+    }
     // Chunk j uses slot j % 2 with its own stream for copy-in, encode and copy-out, so the
     // copies of one chunk overlap the kernels of the other.
-    const int64_t n_chunks = (p->M + chunk - 1) / chunk;
     int rc = CSR_OK;
     for (int64_t j = 0; j < n_chunks && rc == CSR_OK; ++j) {
         const int slot = (int)(j & 1);
@@ -666,7 +740,8 @@ int csr_encode_host(const csr_encode_params_t* p) {
         q.stream = st;
         q.workspace = nullptr;
         q.workspace_bytes = 0;
-        rc = encode_device(&q);
+        q.dev_status = nullptr;                           // the chunks run side by side: the library's word collects them
+        rc = encode_device(&q, n_chunks == 1, prepared);
         if (rc != CSR_OK) break;
         e = cudaMemcpyAsync(reinterpret_cast<char*>(p->out_idx) + (size_t)r0 * ib, b.stage_idx[slot],
                             (size_t)rows * ib, cudaMemcpyDeviceToHost, st);
@@ -693,6 +768,7 @@ int csr_reconstruct_host(const csr_reconstruct_params_t* p) {
     const int64_t chunk = host_chunk_rows(p->M);
     DeviceBuffers& b = g_dev[dev];
     if (int rc = ensure_staging(b, (size_t)chunk * xb, (size_t)chunk * (cb > ib ? cb : ib))) return rc;
+    if (int rc = order_after(b, static_cast<cudaStream_t>(p->stream))) return rc;
     // Chunk j uses slot j % 2 with its own stream: the copies of one chunk overlap the kernel
     // of the other.
     const int64_t n_chunks = (p->M + chunk - 1) / chunk;
@@ -735,19 +811,22 @@ int csr_device_status(void* stream) {
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "stream sync: %s", cudaGetErrorString(e));
     int dev;
     if (int rc = current_device(&dev)) return rc;
-    void* work;
+    // the current work buffer and the outgrown ones (captured graphs still raise their words)
+    std::vector<void*> blocks;
     {
         std::lock_guard<std::mutex> lk(g_mu);
-        work = g_dev[dev].work;
+        if (g_dev[dev].work) blocks.push_back(g_dev[dev].work);
+        blocks.insert(blocks.end(), g_dev[dev].retired.begin(), g_dev[dev].retired.end());
     }
-    if (!work) return CSR_OK;
-    uint32_t st = 0;
-    e = cudaMemcpy(&st, work, sizeof(st), cudaMemcpyDeviceToHost);
-    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "status read: %s", cudaGetErrorString(e));
-    if (st != 0) {
-        cudaMemset(work, 0, kStatusBytes);
-        return fail(CSR_ERR_TIMEOUT, "a device-side wait expired (status word 0x%x)", st);
+    uint32_t seen = 0;
+    for (void* work : blocks) {
+        uint32_t st = 0;
+        e = cudaMemcpy(&st, work, sizeof(st), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "status read: %s", cudaGetErrorString(e));
+        if (st != 0) cudaMemset(work, 0, kStatusBytes);
+        seen |= st;
     }
+    if (seen != 0) return fail(CSR_ERR_TIMEOUT, "a device-side wait expired (status word 0x%x)", seen);
     return CSR_OK;
 }
 
@@ -760,6 +839,8 @@ int csr_release_workspace(void) {
     cudaFree(b.work);
     b.work = nullptr;
     b.work_bytes = 0;
+    for (void* old : b.retired) cudaFree(old);
+    b.retired.clear();
     for (int i = 0; i < 2; ++i) {
         cudaFree(b.stage_x[i]);
         cudaFree(b.stage_idx[i]);
@@ -777,6 +858,49 @@ int csr_release_workspace(void) {
             b.side_done[i] = nullptr;
         }
     }
+    return CSR_OK;
+}
+
+int csr_set_option(const char* name, int64_t value) {
+    if (!name) return fail(CSR_ERR_INVALID_ARG, "name is NULL");
+    if (!strcmp(name, "fast_group")) {
+        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8)
+            return fail(CSR_ERR_INVALID_ARG, "fast_group must be 0 (library's choice), 1, 2, 4 or 8");
+        g_opt_fast_group.store((int)value);
+    } else if (!strcmp(name, "fast_split")) {
+        if (value < 0 || value > 2) return fail(CSR_ERR_INVALID_ARG, "fast_split must be 0, 1 or 2");
+        g_opt_fast_split.store((int)value);
+    } else if (!strcmp(name, "exact_split")) {
+        if (value < 0 || value > 1) return fail(CSR_ERR_INVALID_ARG, "exact_split must be 0 or 1");
+        g_opt_exact_split.store((int)value);
+    } else if (!strcmp(name, "wait_limit_ns")) {
+        if (value < 0 || value > 60000000000ll) return fail(CSR_ERR_INVALID_ARG, "wait_limit_ns must lie in [0, 6e10]");
+        g_opt_wait_limit_ns.store((unsigned long long)value);
+    } else {
+        return fail(CSR_ERR_INVALID_ARG, "unknown option '%s'", name);
+    }
+    return CSR_OK;
+}
+
+int csr_dict_check_norms(const void* D, int N, int d, float tol, void* stream, float* max_dev) {
+    if (int rc = check_dims(d, N, 1, 0)) return rc;
+    if (!D) return fail(CSR_ERR_INVALID_ARG, "D is NULL");
+    if (!aligned16(D)) return fail(CSR_ERR_ALIGNMENT, "D must be 16-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    void* base = nullptr;
+    if (int rc = ensure_work(0, &base, st)) return rc;
+    // a word of the status block that no kernel raises (the first word is the wait status)
+    uint32_t* word = static_cast<uint32_t*>(base) + 32;
+    cudaError_t e = cudaMemsetAsync(word, 0, sizeof(uint32_t), st);
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    if (int rc = launch_dict_norm_deviation(static_cast<const float*>(D), N, d, word, st)) return rc;
+    float dev_max = 0.f;
+    e = cudaMemcpyAsync(&dev_max, word, sizeof(float), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "norm check: %s", cudaGetErrorString(e));
+    if (max_dev) *max_dev = dev_max;
+    if (tol >= 0.f && !(dev_max <= tol))
+        return fail(CSR_ERR_INVALID_ARG, "an atom's l2-norm is off 1 by %g (tolerance %g)", (double)dev_max, (double)tol);
     return CSR_OK;
 }
 

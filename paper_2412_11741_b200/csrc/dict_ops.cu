@@ -33,6 +33,29 @@ __global__ void dict_append_kernel(float* __restrict__ D_new, const void* __rest
     for (int k = 0; k < PER; ++k) D_new[(int64_t)i * D_ + lane * PER + k] = v[k] * inv;
 }
 
+// Largest | ||atom||_2 - 1 | over the dictionary: one warp per atom, fp32 sum of squares as in
+// dict_append_kernel.  The deviations are non-negative floats, so their bit patterns order
+// like integers and one atomicMax keeps the largest; NaN norms count as +inf.
+template <int D_>
+__global__ void norm_deviation_kernel(const float* __restrict__ D, int N, uint32_t* __restrict__ max_bits) {
+    constexpr int PER = D_ / 32;
+    const int lane = threadIdx.x & 31;
+    const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (n >= N) return;
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+        const float v = D[(int64_t)n * D_ + lane * PER + k];
+        ss = fmaf(v, v, ss);
+    }
+    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (lane == 0) {
+        float dev = fabsf(sqrtf(ss) - 1.0f);
+        if (!(dev == dev)) dev = __uint_as_float(0x7f800000u);
+        atomicMax(max_bits, __float_as_uint(dev));
+    }
+}
+
 // Stored form of the coefficients ("Analysis for CSR": fp16 beside the 16-bit index): fp32 ->
 // fp16, round to nearest even, eight values per thread (two 16-byte loads, one 16-byte store).
 __global__ void pack_coef_kernel(const float4* __restrict__ src, uint4* __restrict__ dst, int64_t n8, const float* tail_src,
@@ -66,6 +89,18 @@ int launch_pack_coef(const float* coef32, int64_t n, void* coef16, cudaStream_t 
                                                      n8, coef32 + 8 * n8, reinterpret_cast<__half*>(coef16) + 8 * n8, tail);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "pack_coef launch: %s", cudaGetErrorString(e));
+    return CSR_OK;
+}
+
+int launch_dict_norm_deviation(const float* D, int N, int d, uint32_t* max_bits, cudaStream_t stream) {
+    const int wpb = 8;
+    const int blocks = (N + wpb - 1) / wpb;
+    if (d == 128)
+        norm_deviation_kernel<128><<<blocks, wpb * 32, 0, stream>>>(D, N, max_bits);
+    else
+        norm_deviation_kernel<64><<<blocks, wpb * 32, 0, stream>>>(D, N, max_bits);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "norm_deviation launch: %s", cudaGetErrorString(e));
     return CSR_OK;
 }
 

@@ -59,7 +59,7 @@
 // The codes are the same bits in every case.
 #include <cuda.h>
 
-#include <cstdlib>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -76,7 +76,6 @@ constexpr int PRODUCER_WARP = 8;
 constexpr int MMA_WARP = 9;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int CODE_BLOCK = 8;                         // codes collected before a flush
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s per wait
 
 // ---------------------------------------------------------------------------------------
 // PTX wrappers
@@ -100,6 +99,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         "{\n"
         ".reg .pred p;\n"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// One look at the barrier without suspending the thread.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
         "selp.u32 %0, 1, 0, p;\n"
         "}\n"
         : "=r"(ok)
@@ -261,19 +274,25 @@ struct FastSmem {
 struct WaitCtx {
     volatile uint32_t* abort;
     uint32_t* status;
+    unsigned long long limit_ns;
 };
 
-// Waits for the phase with the given parity; gives up after WAIT_LIMIT_NS or when another
-// thread of the CTA has given up.
+// Waits for the phase with the given parity; gives up after w.limit_ns (wall clock) or when
+// another thread of the CTA has given up.  A limit of zero allows one look at the barrier
+// that does not suspend the thread: whatever is not complete by then counts as expired.
 __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, const WaitCtx& w) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
-    for (uint32_t it = 1; it < (1u << 28); ++it) {
+    if (w.limit_ns != 0) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0) {
-            if (*w.abort) return false;
-            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) break;
+        const unsigned long long t0 = globaltimer_ns();
+        for (uint32_t it = 1; it < (1u << 28); ++it) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if ((it & 63u) == 0) {
+                if (*w.abort) return false;
+                if (globaltimer_ns() - t0 > w.limit_ns) break;
+            }
         }
+    } else if (mbar_test_wait(bar, parity)) {
+        return true;
     }
     *w.abort = 1;
     atomicOr(w.status, kStatusTimeout);
@@ -288,7 +307,7 @@ __device__ __forceinline__ bool wait_bounded_cluster(uint64_t* bar, uint32_t par
         if (mbar_try_wait_cluster(bar, parity)) return true;
         if ((it & 63u) == 0) {
             if (*w.abort) return false;
-            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) break;
+            if (globaltimer_ns() - t0 > w.limit_ns) break;
         }
     }
     *w.abort = 1;
@@ -590,7 +609,8 @@ __global__ void __launch_bounds__(NT, 1)
 encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* __restrict__ Db,
                    const void* __restrict__ X, int x_dtype, int64_t ldx, int64_t M, int N, int s,
                    uint16_t* __restrict__ out_idx, void* __restrict__ out_coef, int coef_dtype, int64_t ldc, int vec_codes,
-                   uint32_t key_mask, uint32_t* status, int n_splits, uint2* __restrict__ partial) {
+                   uint32_t key_mask, uint32_t* status, int n_splits, uint2* __restrict__ partial,
+                   unsigned long long wait_limit_ns) {
     using S = FastSmem<D_>;
     extern __shared__ uint8_t smem_raw[];
     S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -620,7 +640,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
     constexpr int KSTEPS = STAGE_CH / UMMA_K;               // MMAs per stage
     constexpr int CHUNKS = D_ / 8;                          // 16-byte chunks per row
     constexpr int NG = TILE_N / G;                          // arg-max groups per accumulator
-    const WaitCtx wc{&sm.abort, status};
+    const WaitCtx wc{&sm.abort, status, wait_limit_ns};
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) {
@@ -1086,14 +1106,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn get_encode_tiled() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    static const EncodeTiledFn fn = [] {               // initialised once, also with concurrent callers
         void* p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+            return reinterpret_cast<EncodeTiledFn>(p);
+        return static_cast<EncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
 
@@ -1118,8 +1138,12 @@ void cluster_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int clus
 // or clusters of that size cannot be launched here).  Asked once per size.
 template <int D_, int G>
 int max_clusters(int cluster_ctas) {
-    static int cached[17] = {0};                       // 0 = not asked yet, -1 = none
-    if (cluster_ctas < 2 || cluster_ctas > 16) return 0;
+    static int cached_dev[64][17] = {};                // per device: 0 = not asked yet, -1 = none
+    static std::mutex mu;
+    int dev = 0;
+    if (cluster_ctas < 2 || cluster_ctas > 16 || cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    std::lock_guard<std::mutex> lk(mu);
+    int* cached = cached_dev[dev];                     // (function attributes are per device as well)
     if (cached[cluster_ctas] == 0) {
         const size_t smem = sizeof(FastSmem<D_>) + 1024;
         int n = 0;
@@ -1166,6 +1190,7 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
     // 16-byte code stores need eight codes per flush and 16-byte aligned rows in both arrays
     const uintptr_t ci = reinterpret_cast<uintptr_t>(a.out_idx), cc = reinterpret_cast<uintptr_t>(a.out_coef);
     const int vec_codes = (a.s % 8 == 0) && (a.ld_code % 8 == 0) && (ci % 16 == 0) && (cc % 16 == 0);
+    const unsigned long long wait_limit = options().wait_limit_ns;
     if (cluster_grid > 0) {
         // n_splits CTAs per cluster, cluster_grid CTAs in all
         cudaLaunchConfig_t cfg = {};
@@ -1173,7 +1198,7 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
         cluster_config<D_, G>(cfg, attr, n_splits, cluster_grid, smem, a.stream);
         e = cudaLaunchKernelEx(&cfg, one_tile ? encode_fast_kernel<D_, G, 2> : encode_fast_kernel<D_, G, 1>, tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
                                a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask, status, n_splits,
-                               static_cast<uint2*>(nullptr));
+                               static_cast<uint2*>(nullptr), wait_limit);
         if (e != cudaSuccess) {
             // refused at launch (nothing ran): the caller takes another path
             cudaGetLastError();
@@ -1183,7 +1208,7 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
     }
     encode_fast_kernel<D_, G, 0><<<grid, NT, smem, a.stream>>>(tmap, Db, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
                                                            a.out_coef, a.coef_dtype, a.ld_code, vec_codes, key_mask,
-                                                           status, n_splits, partial);
+                                                           status, n_splits, partial, wait_limit);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "encode_fast launch: %s", cudaGetErrorString(e));
     return CSR_OK;
@@ -1191,14 +1216,12 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
 
 // Atoms per arg-max group.  Larger groups save arg-max arithmetic during the sweep (which
 // grows with N) and cost a wider gather at the end of every sweep (which does not); the
-// defaults are where the measured crossovers lie.  CSR_FAST_GROUP (1, 2, 4 or 8) overrides
-// them; it is a tuning knob only: every setting returns a valid maximum of the same bf16
-// correlations.
+// defaults are where the measured crossovers lie.  The option "fast_group" (1, 2, 4 or 8)
+// overrides them; it is a tuning knob only: every setting picks, per row, an atom whose bf16
+// correlation is the largest to within the width of the group tag.
 int group_size(int d, int N) {
-    if (const char* e = getenv("CSR_FAST_GROUP")) {
-        const int v = atoi(e);
-        if (v == 1 || v == 2 || v == 4 || v == 8) return v;
-    }
+    const int v = options().fast_group;
+    if (v == 1 || v == 2 || v == 4 || v == 8) return v;
     if (d == 64) return 4;
     return N >= 16384 ? 4 : 1;
 }
@@ -1399,7 +1422,7 @@ int launch_encode_fast_prepared(const EncodeArgs& a, const void* dict_bf16, uint
     // few rows: one launch of CTA clusters that share the dictionary (needs no scratch) ...
     // (unless the launch-per-iteration split below, which can spread a pair of row tiles over more
     // than 16 CTAs, is expected to be faster: very large dictionaries)
-    if (!getenv("CSR_FAST_NO_SPLIT") && !getenv("CSR_FAST_NO_CLUSTER")) {
+    if (options().fast_split == 0) {
         float budget = 3.0e38f;
         if (split_scratch && split_count(a.M, a.N, &budget) <= 1) budget = 3.0e38f;
         bool done = false;

@@ -34,8 +34,8 @@ def test_exports_match_header(lib):
 
 def test_version_and_struct_sizes(lib):
     from paper_2412_11741_b200 import binding
-    assert binding.csr_version() == 100
-    assert ctypes.sizeof(binding.csr_encode_params_t) == 120
+    assert binding.csr_version() == 110
+    assert ctypes.sizeof(binding.csr_encode_params_t) == 128
     assert ctypes.sizeof(binding.csr_reconstruct_params_t) == 96
 
 
@@ -55,7 +55,7 @@ def _params(binding, **kw):
     (dict(d=96), -2), (dict(N=0), -1), (dict(N=70000), -1), (dict(s=0), -1), (dict(s=65), -1), (dict(M=-1), -1),
     (dict(D=0), -1), (dict(X=0), -1), (dict(out_idx=0), -1), (dict(D=0x1008), -3),
     (dict(X=0x2004), -3), (dict(mode=7), -1), (dict(x_dtype=3), -1), (dict(coef_dtype=1), -1),
-    (dict(struct_size=8), -1), (dict(workspace=0x5008), -3),
+    (dict(struct_size=8), -1), (dict(workspace=0x5008), -3), (dict(dev_status=0x6002), -3),
 ])
 def test_encode_argument_errors(lib, kw, code):
     from paper_2412_11741_b200 import binding
@@ -119,3 +119,20 @@ def test_workspace_query(lib):
     assert 8192 * 128 * 2 <= n <= 8192 * 128 * 2 + 4096
     with pytest.raises(binding.CsrError):
         binding.csr_encode_workspace_bytes(binding.CSR_MODE_BF16_FAST, 100, 8192)
+
+
+def test_options_and_norm_check_argument_errors(lib):
+    from paper_2412_11741_b200 import binding
+    assert lib.csr_set_option(b"fast_group", 4) == binding.CSR_OK
+    assert lib.csr_set_option(b"fast_group", 0) == binding.CSR_OK
+    assert lib.csr_set_option(b"fast_group", 3) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_set_option(b"fast_split", 3) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_set_option(b"exact_split", -1) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_set_option(b"wait_limit_ns", -5) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_set_option(b"wait_limit_ns", 2_000_000_000) == binding.CSR_OK
+    assert lib.csr_set_option(b"no_such_option", 1) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_set_option(None, 1) == binding.CSR_ERR_INVALID_ARG
+    out = ctypes.c_float()
+    assert lib.csr_dict_check_norms(0, 1024, 128, 1e-3, None, ctypes.byref(out)) == binding.CSR_ERR_INVALID_ARG
+    assert lib.csr_dict_check_norms(0x1000, 1024, 96, 1e-3, None, ctypes.byref(out)) == binding.CSR_ERR_UNSUPPORTED
+    assert lib.csr_dict_check_norms(0x1004, 1024, 128, 1e-3, None, ctypes.byref(out)) == binding.CSR_ERR_ALIGNMENT

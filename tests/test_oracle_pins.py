@@ -269,19 +269,29 @@ def test_format_golden():
 
 # --- planted mistakes must be caught (the pins are not vacuous) -----------------------------
 
-def test_pins_detect_unsigned_coefficient():
+def test_unsigned_reading_of_eq2_is_not_what_the_oracle_computes():
+    """Eq. 2 prints the coefficient as a supremum of absolute values.  Taken literally (subtract
+    |c| d) the residual GAINS energy whenever the best correlation is negative; the oracle keeps
+    the sign.  On an input whose first pick has a negative correlation the oracle's output
+    satisfies the energy identity and the literal reading, written out here, does not; the two
+    residuals differ from the first step on."""
     rng = np.random.default_rng(0)
     D = _rand_dict(rng, 64, 16)
-    x = rng.standard_normal(16)
-    R = x.copy()
+    x = rng.standard_normal(16).astype(np.float32)
+    res = orc.mp_encode(D, x[None, :], 4)
+    assert res.coef[0, 0] < 0                              # the case that tells the readings apart
+    R = x.astype(np.float64).copy()
     e = 0.0
     for _ in range(4):
         c = D.astype(np.float64) @ R
         i = int(np.argmax(np.abs(c)))
-        R = R - abs(c[i]) * D[i]          # the literal reading of Eq. 2
+        R = R - abs(c[i]) * D[i]                           # the literal reading of Eq. 2
         e += c[i] ** 2
-    # with an unsigned coefficient the energy identity breaks for this input
-    assert abs((x ** 2).sum() - (R ** 2).sum() - e) > 1e-3
+    x64 = x.astype(np.float64)
+    assert abs((x64 ** 2).sum() - (R ** 2).sum() - e) > 1e-3                       # literal reading: identity broken
+    e_or = float((res.coef[0] ** 2 * (2.0 - (D[res.idx[0]].astype(np.float64) ** 2).sum(1))).sum())
+    assert abs((x64 ** 2).sum() - (res.residual[0] ** 2).sum() - e_or) < 1e-12     # the oracle: identity holds
+    assert np.linalg.norm(res.residual[0]) < np.linalg.norm(R) - 1e-3
 
 
 # ---------------------------------------------------------------------------------------
@@ -472,3 +482,76 @@ def test_training_steps_renormalise_and_lower_the_loss():
         first = l_mse if first is None else first
         assert np.allclose(np.linalg.norm(D.astype(np.float64), axis=1), 1.0, atol=1e-6)
     assert l_mse < 0.8 * first
+
+
+def test_train_step_with_zero_mse_gradient_is_the_diversity_step_in_closed_form():
+    """Rows of X that ARE atoms (orthogonal to every other atom) are encoded exactly with s = 1, so
+    grad L_MSE = 0 and the step is ReNorm(D - lr * beta * grad L_div).  With all atoms
+    orthonormal except d_0 and d_1 at a known angle (d_0 . d_1 = c), D D^T - I has the single
+    pair of entries c, so grad L_div is (4 / N^2) * c * d_1 on atom 0, (4 / N^2) * c * d_0 on atom 1
+    and zero elsewhere: written out by hand below.  A doubled lr, beta applied to the wrong
+    gradient or a wrong 4 / N^2 changes atoms 0 and 1."""
+    N, d = 6, 8
+    D = np.zeros((N, d), np.float32)
+    D[0, 0] = 1.0
+    D[1, 0], D[1, 1] = 0.6, 0.8
+    for n in range(2, N):
+        D[n, n] = 1.0
+    X = np.stack([D[2], 2.5 * D[4], -1.5 * D[3]]).astype(np.float32)
+    lr, beta = 0.05, 0.3
+    Dn, l_mse, l_div, res = orc.dict_train_step(D, X, 1, lr, beta)
+    assert res.idx[:, 0].tolist() == [2, 4, 3] and l_mse == 0.0
+    D64 = D.astype(np.float64)
+    c = float(D64[0] @ D64[1])
+    n1 = float(D64[1] @ D64[1])                           # 0.6^2 + 0.8^2 in fp32 values: 1 up to 1e-8
+    want = D64.copy()
+    # (D D^T - I) D, rows 0 and 1: row 0 = c d_1, row 1 = c d_0 + (|d_1|^2 - 1) d_1
+    want[0] = D64[0] - lr * beta * (4.0 / N ** 2) * (c * D64[1])
+    want[1] = D64[1] - lr * beta * (4.0 / N ** 2) * (c * D64[0] + (n1 - 1.0) * D64[1])
+    want /= np.linalg.norm(want, axis=1, keepdims=True)
+    assert np.abs(Dn.astype(np.float64) - want).max() < 1e-7
+    assert l_div == pytest.approx((2 * c * c + (n1 - 1.0) ** 2) / N ** 2, rel=1e-9)
+    assert np.abs(Dn[0] - D[0]).max() > 1e-4              # the step is not a no-op
+
+
+def test_train_step_with_orthonormal_atoms_is_the_mse_step_in_closed_form():
+    """Orthonormal atoms: grad L_div = 0 whatever beta is, and the step is ReNorm(D - lr * grad
+    L_MSE).  One row x = (3, 1, 0, 0) over the identity dictionary with s = 1: the pursuit takes
+    atom 0 with c = 3, the error is e = (0, 1, 0, 0), the only gradient row is
+    -2 c e = (0, -6, 0, 0) on atom 0, so atom 0 becomes (1, 6 lr, 0, 0) / norm and the others stay."""
+    D = np.eye(4, dtype=np.float32)
+    X = np.array([[3.0, 1.0, 0.0, 0.0]], np.float32)
+    lr, beta = 0.01, 7.0                                  # a large beta: it must not touch this step
+    Dn, l_mse, l_div, res = orc.dict_train_step(D, X, 1, lr, beta)
+    assert res.idx[0, 0] == 0 and res.coef[0, 0] == 3.0
+    assert l_mse == pytest.approx(1.0, abs=1e-15) and l_div == 0.0
+    want = np.eye(4)
+    want[0] = np.array([1.0, 6.0 * lr, 0.0, 0.0]) / np.sqrt(1.0 + 36.0 * lr * lr)
+    assert np.abs(Dn.astype(np.float64) - want).max() < 1e-7
+    # two rows sharing an atom add up: x_2 = (-2, 0, 1, 0) also takes atom 0 (c = -2, e = (0, 0, 1, 0))
+    X2 = np.array([[3.0, 1.0, 0.0, 0.0], [-2.0, 0.0, 1.0, 0.0]], np.float32)
+    Dn2, l_mse2, _, _ = orc.dict_train_step(D, X2, 1, lr, beta)
+    w0 = np.array([1.0, 6.0 * lr, -4.0 * lr, 0.0])        # -lr * (-2*3*e_1 + -2*(-2)*e_2)
+    want[0] = w0 / np.linalg.norm(w0)
+    assert np.abs(Dn2.astype(np.float64) - want).max() < 1e-7 and l_mse2 == pytest.approx(2.0, abs=1e-15)
+
+
+def test_train_step_displacement_is_linear_in_lr_to_first_order():
+    """Doubling lr doubles the displacement of every atom up to O(lr^2): the codes do not depend
+    on lr, and ReNorm of a unit atom moved by a small step removes the step's radial part and
+    changes the rest only to second order."""
+    rng = np.random.default_rng(31)
+    N, d, M, s = 24, 8, 200, 3
+    D = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32))
+    X = rng.standard_normal((M, d)).astype(np.float32)
+    lr, beta = 1e-4, 0.5
+    D1 = orc.dict_train_step(D, X, s, lr, beta)[0].astype(np.float64)
+    D2 = orc.dict_train_step(D, X, s, 2 * lr, beta)[0].astype(np.float64)
+    d1, d2 = D1 - D, D2 - D
+    assert np.abs(d1).max() > 1e-4                        # far above the fp32 rounding of the outputs (6e-8)
+    assert np.abs(d2 - 2 * d1).max() < 0.02 * np.abs(d1).max() + 3e-7
+    # and beta scales the diversity part alone: the difference of two betas is lr * dbeta * grad L_div (tangential part)
+    Da = orc.dict_train_step(D, X, s, lr, 0.0)[0].astype(np.float64)
+    g = (4.0 / N ** 2) * ((D.astype(np.float64) @ D.astype(np.float64).T - np.eye(N)) @ D.astype(np.float64))
+    tang = g - (g * D).sum(1, keepdims=True) * D          # ReNorm removes the radial part to first order
+    assert np.abs((Da - D1) - lr * beta * tang).max() < 0.02 * np.abs(lr * beta * tang).max() + 3e-7

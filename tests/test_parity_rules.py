@@ -68,3 +68,58 @@ def test_fast_rules_accept_bf16_emulation_and_reject_mistakes():
     assert not parity.compare_fast(w.D, X, w.s, shifted, coef, res).ok
     stale = np.repeat(idx[:, :1], w.s, axis=1)
     assert not parity.compare_fast(w.D, X, w.s, stale, np.repeat(coef[:, :1], w.s, axis=1), res).ok
+
+
+def _emulated_report(w, rows, seed):
+    X = w.X[wl.stratified_rows(w.M, rows, seed)]
+    if w.x_dtype != "bf16":
+        X = wl.round_to_bf16(X)                          # what the fast mode encodes
+    res = orc.mp_encode(w.D, X, w.s)
+    idx, coef = _bf16_mp(w.D, X, w.s)
+    return parity.compare_fast(w.D, X, w.s, idx, coef, res)
+
+
+def test_fast_gate_constants_come_from_the_bf16_emulation(capsys):
+    """Where the fast-mode gates' numbers come from: bf16-operand matching pursuit (operands
+    rounded to bf16, fp32 sums, residual rounded to bf16 after every update) on samples of every
+    configuration first leaves the oracle's trajectory at steps whose best two atoms are at most
+    about 1.2 accumulated roundings apart (the gate allows FAST_GAP_C = 2.5), and its error
+    ratios stay inside the caps with room to spare.  Prints the distribution per configuration."""
+    cases = [(wl.llama2_layer(tokens=64), 2048), (wl.gqa_long(tokens=64), 2048), (wl.sparsity_sweep(4, tokens=64), 2048),
+             (wl.sparsity_sweep(32, tokens=64), 1024), (wl.dict_sweep(2048, M=4096), 2048),
+             (wl.dict_sweep(16384, M=2048), 1024), (wl.dict_sweep(4096, d=64, M=4096), 2048), (wl.tiny(), 2048)]
+    lines = []
+    for seed, (w, rows) in enumerate(cases):
+        rep = _emulated_report(w, rows, seed)
+        lines.append(f"{w.name:26s} s={w.s:2d} N={w.N:5d} d={w.d:3d} rows={rep.rows}: same {rep.same_rows / rep.rows:.3f} "
+                     f"margin max {rep.max_first_margin:.3f} rel gap max {rep.max_first_gap:.4f} "
+                     f"ratio p50 {rep.ratio_p50:.4f} p99 {rep.ratio_p99:.4f} max {rep.ratio_max:.4f} mean {rep.mean_ratio:.5f}")
+        assert rep.ok, (w.name, rep.detail)
+        assert rep.max_first_margin <= 0.6 * parity.FAST_GAP_C, (w.name, rep.max_first_margin)
+        assert rep.ratio_max <= 0.5 * (1 + parity.fast_ratio_cap(w.s)) + 0.05, (w.name, rep.ratio_max)
+    with capsys.disabled():
+        print("\n" + "\n".join(lines))
+
+
+def test_fast_gate_scales_with_the_residual_not_with_a_flat_gap():
+    """Dictionaries of a handful of atoms: after a few steps the residual is nearly orthogonal to
+    every atom, all correlations are tiny and RELATIVE gaps of 10 % and more separate atoms that
+    bf16 cannot tell apart, while the absolute rule of the gate still holds; and a pick that is
+    wrong by a clear margin at the first step is rejected whatever its relative gap."""
+    rng = np.random.default_rng(77)
+    for N in (5, 100):
+        D = wl.normalise_rows(rng.standard_normal((N, 128)).astype(np.float32))
+        X = wl.round_to_bf16(rng.standard_normal((600, 128)).astype(np.float32))
+        res = orc.mp_encode(D, X, 4)
+        idx, coef = _bf16_mp(D, X, 4)
+        rep = parity.compare_fast(D, X, 4, idx, coef, res)
+        assert rep.ok, (N, rep.detail)
+    # second-best atom at step 0 for every row: relative gaps of a few per cent, far outside the gate
+    w = wl.llama2_layer(tokens=8, N=1024)
+    X = w.X[:256]
+    res = orc.mp_encode(w.D, X, 1)
+    C = np.abs(X.astype(np.float64) @ w.D.astype(np.float64).T)
+    second = np.argsort(-C, axis=1)[:, 1].astype(np.int32)[:, None]
+    c2 = np.take_along_axis(X.astype(np.float64) @ w.D.astype(np.float64).T, second.astype(np.int64), 1)
+    rep = parity.compare_fast(w.D, X, 1, second, c2, res)
+    assert not rep.ok and "roundings apart" in rep.detail
