@@ -109,7 +109,7 @@ class ClockSampler:
         except Exception:
             pass
         if sm:
-            # under load = the upper half of the samples (idle samples before/after are dropped)
+            # the sampler runs only around the timed region: the median over all samples is the clock under load
             out["sm_mhz"] = statistics.median(sm)
             out["sm_max_mhz"] = max(mx)
             out["samples"] = len(sm)
@@ -311,6 +311,37 @@ def run_cuda(args):
     return 0
 
 
+def launch_ranks(n: int, argv, script: str = None, backend_env: dict = None) -> int:
+    """Starts n ranks of `script` (this file) on one node, one process per GPU, the way the
+    multi-GPU form of this benchmark is meant to be launched, and returns the exit code.  Rank 0's
+    single JSON line reaches this process's stdout unchanged.  NCCL's own log (which states the
+    communicator's rank count) goes to files that are then copied to stderr."""
+    import socket
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    env = dict(os.environ)
+    logdir = tempfile.mkdtemp(prefix="bench_nccl_")
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    env.setdefault("NCCL_DEBUG_FILE", os.path.join(logdir, "nccl_%h_%p.log"))
+    env.update(backend_env or {})
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), script or os.path.abspath(__file__)] + list(argv)
+    rc = subprocess.call(cmd, env=env)
+    try:
+        for name in sorted(os.listdir(logdir)):
+            for line in open(os.path.join(logdir, name), errors="replace"):
+                if "nranks" in line or "Init COMPLETE" in line:
+                    sys.stderr.write(line)
+            os.unlink(os.path.join(logdir, name))
+        os.rmdir(logdir)
+    except OSError:
+        pass
+    return rc
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -322,6 +353,9 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # called as `python bench.py --gpus N`: start the N ranks here
+        return launch_ranks(args.gpus, sys.argv[1:])
     return run_cuda(args)
 
 

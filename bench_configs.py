@@ -62,8 +62,9 @@ def run_case(w, reps, exact_rows=16384, rows=0):
         raise RuntimeError(csr.csr_last_error_string())
     handle = csr.csr_dict_create(D)
     enc_prepared_ms = _time(lambda: csr.csr_encode_ex(D, X, s, out_idx=idx, out_coef=coef, dict=handle), reps)
-    csr.csr_dict_destroy(handle)
     xh = torch.empty((M, d), dtype=torch.bfloat16, device=dev)
+    rec_prepared_ms = _time(lambda: csr.csr_reconstruct_ex(D, idx, coef, X_hat=xh, dict=handle), max(5, reps // 3))
+    csr.csr_dict_destroy(handle)
     rec_ms = _time(lambda: csr.csr_reconstruct_ex(D, idx, coef, X_hat=xh), max(5, reps // 3))
     err_sum, step = 0.0, 1 << 18
     for r0 in range(0, M, step):
@@ -84,6 +85,9 @@ def run_case(w, reps, exact_rows=16384, rows=0):
         "reconstruct_ms": round(rec_ms, 4),
         "reconstruct_hbm_gbs": M * (4 * s + 2 * d) / (rec_ms * 1e-3) / 1e9,
         "reconstruct_l2_gather_gbs": M * s * d * 4 / (rec_ms * 1e-3) / 1e9,
+        "reconstruct_ms_prepared_dict": round(rec_prepared_ms, 4),
+        "reconstruct_prepared_hbm_gbs": M * (4 * s + 2 * d) / (rec_prepared_ms * 1e-3) / 1e9,
+        "reconstruct_prepared_l2_gather_gbs": M * s * d * 2 / (rec_prepared_ms * 1e-3) / 1e9,
         "exact_mode_vectors_per_s": me / (ex_ms * 1e-3) if me else None, "exact_mode_rows": me,
     }
 

@@ -142,6 +142,8 @@ typedef struct csr_reconstruct_params {
     void* stream;
     int64_t ld_code;        /* elements between consecutive rows of idx and of coef; 0 = s */
     int64_t ld_xhat;        /* elements between consecutive rows of X_hat; 0 = d */
+    const void* dict;       /* csr_dict_t* from csr_dict_create, or NULL: gather the atoms from the
+                               handle's bf16 copy of D instead of the fp32 D (see csr_reconstruct) */
 } csr_reconstruct_params_t;
 
 /*
@@ -168,6 +170,14 @@ int64_t csr_encode_workspace_bytes(int mode, int d, int N);
  * De-sparse ("De-Sparse to restore", Eq. 12): X_hat[m,:] = sum_g coef[m][g] * D[idx[m][g]][:],
  * accumulated in fp32 in the order g = 0 .. s-1; repeated indices accumulate.  Every idx
  * must be < N (larger values are clamped to N-1 rather than read out of bounds).
+ *
+ * With params.dict (a handle of the same D, N, d) the atoms are read from the handle's bf16
+ * copy, which halves the bytes gathered per row (what bounds this kernel from about s = 4
+ * up).  The result is then Eq. 12 over the atoms rounded to bf16: it differs from the fp32-atom
+ * result by at most 2^-8 * sum_g |coef_g * D[idx_g][k]| per channel k (bf16 keeps 8 significant
+ * bits).  Codes made by the fast
+ * mode were computed against exactly these rounded atoms, so for them this is the consistent
+ * choice.
  *
  * 8-argument form: coef is fp16, X_hat is bf16, stream 0.
  */
@@ -356,10 +366,13 @@ int csr_reconstruct_host(const csr_reconstruct_params_t* p);
  * Limits and rules
  *   - N8 * d <= CSR_STATIC_MAX_DICT_ELEMS with N8 = N rounded up to a multiple of 8 (8192
  *     atoms of 128 channels, a 2 MiB bf16 copy);
- *     larger dictionaries are rejected with CSR_ERR_UNSUPPORTED.  Every GPU on which the
- *     library is loaded holds the array (2 MiB + 2 KiB) until the process exits.
+ *     larger dictionaries are rejected with CSR_ERR_UNSUPPORTED.
  *   - The first call on a device looks up the array's device address, once, with that
- *     device current; make that first call before any stream capture begins.
+ *     device current.  That lookup (and the first launch of each kernel) makes the CUDA
+ *     runtime load the part of the library image that holds the array, which is when the
+ *     2 MiB + 2 KiB are taken from that GPU's memory, to be held until the process exits.
+ *     Make one call per device and per shape class (many rows; few rows) at start-up and
+ *     before any stream capture begins; later calls take nothing from device memory.
  *   - All calls on a device share the one array, and it keeps what the last call wrote.
  *     Each call rewrites the dictionary copy in full and zeroes its status word before
  *     use, so stale contents never matter; but two calls whose work overlaps on the GPU

@@ -62,6 +62,7 @@ class csr_reconstruct_params_t(ctypes.Structure):
         ("d", ctypes.c_int32), ("N", ctypes.c_int32), ("s", ctypes.c_int32), ("reserved1", ctypes.c_int32),
         ("X_hat", ctypes.c_void_p), ("stream", ctypes.c_void_p),
         ("ld_code", ctypes.c_int64), ("ld_xhat", ctypes.c_int64),
+        ("dict", ctypes.c_void_p),
     ]
 
 
@@ -457,9 +458,12 @@ def csr_decode_attention(Dk: torch.Tensor, Dv: torch.Tensor, Q: torch.Tensor, k_
 
 def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *,
                        out_dtype: torch.dtype = torch.bfloat16,
-                       X_hat: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """csr_reconstruct_ex on CUDA tensors; returns X_hat [M][d]."""
+                       X_hat: Optional[torch.Tensor] = None, dict: Optional[int] = None) -> torch.Tensor:
+    """csr_reconstruct_ex on CUDA tensors; returns X_hat [M][d].  dict: a csr_dict_create handle of
+    D, to gather bf16 atoms."""
     p, X_hat = _reconstruct_params(D, idx, coef, out_dtype, X_hat)
+    if dict is not None:
+        p.dict = dict
     with torch.cuda.device(D.device):
         _check(lib().csr_reconstruct_ex(ctypes.byref(p)))
     return X_hat

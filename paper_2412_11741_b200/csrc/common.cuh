@@ -67,6 +67,7 @@ size_t encode_fast_split_scratch_bytes(int64_t M, int d, int N);
 
 struct ReconstructArgs {
     const float* D;
+    const void* dict_bf16;   // bf16 copy of D ([N rounded up to 8][d]) to gather from instead, or NULL
     const uint16_t* idx;
     const void* coef;
     int coef_dtype;

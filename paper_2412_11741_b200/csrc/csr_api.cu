@@ -237,6 +237,14 @@ int check_reconstruct(const csr_reconstruct_params_t* p, bool host_io) {
                     (long long)p->ld_code, (long long)p->ld_xhat);
     if (host_io && (p->ld_code || p->ld_xhat)) return fail(CSR_ERR_UNSUPPORTED, "the host entry points take dense arrays");
     if (!aligned16(p->D)) return fail(CSR_ERR_ALIGNMENT, "D must be 16-byte aligned");
+    if (p->dict) {
+        const csr_dict* dc = static_cast<const csr_dict*>(p->dict);
+        int dev = -1;
+        if (int rc = current_device(&dev)) return rc;
+        if (dc->magic != kDictMagic) return fail(CSR_ERR_INVALID_ARG, "dict is not a live csr_dict_t handle");
+        if (dc->device != dev || dc->D != p->D || dc->N != p->N || dc->d != p->d)
+            return fail(CSR_ERR_INVALID_ARG, "dict was created for another device, D, N or d");
+    }
     if (!host_io) {
         const size_t xe = dtype_size(p->out_dtype), ce = p->coef_dtype == CSR_DTYPE_F16 ? 2 : 4;
         if (!aligned16(p->X_hat) || (p->ld_xhat && (p->ld_xhat * xe) % 16 != 0))
@@ -254,6 +262,7 @@ int check_reconstruct(const csr_reconstruct_params_t* p, bool host_io) {
 ReconstructArgs reconstruct_args(const csr_reconstruct_params_t* p) {
     ReconstructArgs a;
     a.D = static_cast<const float*>(p->D);
+    a.dict_bf16 = p->dict ? static_cast<const csr_dict*>(p->dict)->bf16 : nullptr;
     a.idx = p->idx;
     a.coef = p->coef;
     a.coef_dtype = p->coef_dtype;

@@ -7,8 +7,12 @@
 // that owns all free device memory, or in a latency-critical section where an implicit
 // device synchronisation (which cudaMalloc and cudaFree may cause) is not acceptable.
 // For them the scratch lives in a file-scope __device__ array that is part of the
-// library image: every GPU that loads libcsr.so holds these bytes until the process exits,
-// and no call here allocates or frees anything.
+// library image, and no call here calls an allocating routine.  The image's device data is
+// placed by the CUDA runtime when the module that holds it is first used on a device (with
+// lazy module loading: at the first call of this entry point there, which looks the array
+// up; the first launch of each kernel loads its code the same way), so the first call on a
+// device belongs to start-up; from the second call on nothing is taken from device memory.
+// Every GPU that has made that first call holds the bytes until the process exits.
 #include <mutex>
 
 #include "common.cuh"

@@ -17,7 +17,8 @@ Rules (derived from the stated tolerances):
           gap_g * |c_g|  <=  FAST_GAP_C * 2^-9 * sqrt(sum_{j<=g} ||R_j||^2)
       (left: the absolute distance between the oracle's best and second-best
       |correlation|; right: every residual R_j the fast mode has carried was rounded to
-      bf16, relative error 2^-9 per element, and those errors add up like a random walk;
+      bf16 (at most 2^-8, about 2^-9.8 r.m.s. relative error per element), and those errors add up
+      like a random walk;
       the atoms' own rounding, 2^-9 ||R_g||, is covered by the j = g term).  At g = 0 this is
       2^-9 * FAST_GAP_C * ||x||, i.e. a relative gap of about 2^-6.5 for the usual
       |c_0| ~ 0.3 ||x||; it widens only as the residual shrinks.  FAST_GAP_C = 2.5 is twice

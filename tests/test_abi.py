@@ -36,7 +36,7 @@ def test_version_and_struct_sizes(lib):
     from paper_2412_11741_b200 import binding
     assert binding.csr_version() == 110
     assert ctypes.sizeof(binding.csr_encode_params_t) == 128
-    assert ctypes.sizeof(binding.csr_reconstruct_params_t) == 96
+    assert ctypes.sizeof(binding.csr_reconstruct_params_t) == 104
 
 
 def _params(binding, **kw):

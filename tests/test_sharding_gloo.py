@@ -63,3 +63,23 @@ def test_two_ranks_cover_all_rows_and_agree_on_rate(tmp_path):
     assert int(metas[0][0]) == 0 and int(metas[0][1]) == int(metas[1][0]) and int(metas[1][1]) == M
     assert np.array_equal(np.concatenate(parts), full)           # sharding changes no result
     assert metas[0][2] == metas[1][2] == M / 2.0                 # all units / slowest rank's time
+
+
+def test_bench_launcher_starts_one_rank_per_gpu(capfd):
+    """`python bench.py --gpus N` without torchrun's environment starts the N ranks itself:
+    the launcher, run here on a stub worker over gloo, brings up a process group of N ranks
+    and passes rank 0's single JSON line through."""
+    import importlib.util
+    import json
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_under_test", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    stub = os.path.join(root, "tests", "_stub_rank_worker.py")
+    rc = bench.launch_ranks(2, ["--gpus", "2", "--steps", "3"], script=stub)
+    out = capfd.readouterr().out
+    assert rc == 0
+    lines = [json.loads(l) for l in out.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["n_gpus"] == 2 and lines[0]["units"] == 2.0 and lines[0]["slowest"] == 2.0
+    assert lines[0]["argv"] == ["--gpus", "2", "--steps", "3"] and "x2" in lines[0]["parallelism"]
