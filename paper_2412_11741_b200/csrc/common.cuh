@@ -127,9 +127,17 @@ struct TrainArgs {
     float* grad_div;   // [N][d] scratch
     double* losses;    // [2]
     float lr, beta;
+    void* div_scratch;  // div_grad_scratch_bytes(N, d) bytes for the diversity gradient's operands
+    uint32_t* status;   // device word raised by a bounded wait that expires
     cudaStream_t stream;
 };
 int launch_dict_train(const TrainArgs& a);
+
+// Diversity loss and gradient on the tensor cores: losses[1] += ||D D^T - I||_F^2 / N^2 and
+// grad_div (zeroed by the caller) += (4 / N^2) (D D^T - I) D.
+size_t div_grad_scratch_bytes(int N, int d);
+int launch_div_grad(const float* D, int N, int d, float* grad_div, double* losses, void* scratch, uint32_t* status,
+                    cudaStream_t stream);
 
 // Element `off` of an array of dtype F32, BF16 or F16, widened exactly to fp32.
 __device__ __forceinline__ float load_elem(const void* p, int dtype, int64_t off) {

@@ -659,8 +659,9 @@ int csr_dict_train_step(const csr_train_params_t* p) {
     const size_t idx_b = ((size_t)p->M * p->s * 2 + 255) / 256 * 256;
     const size_t coef_b = ((size_t)p->M * p->s * 4 + 255) / 256 * 256;
     const size_t g_b = ((size_t)p->N * p->d * 4 + 255) / 256 * 256;
+    const size_t div_b = div_grad_scratch_bytes(p->N, p->d);
     void* base = nullptr;
-    if (int rc = ensure_work(enc + idx_b + coef_b + 2 * g_b, &base, static_cast<cudaStream_t>(p->stream))) return rc;
+    if (int rc = ensure_work(enc + idx_b + coef_b + 2 * g_b + div_b, &base, static_cast<cudaStream_t>(p->stream))) return rc;
     char* q = static_cast<char*>(align_up(static_cast<char*>(base) + kStatusBytes, 1024)) + enc;
     TrainArgs a;
     a.D = static_cast<float*>(p->D);
@@ -674,6 +675,8 @@ int csr_dict_train_step(const csr_train_params_t* p) {
     a.coef = reinterpret_cast<float*>(q + idx_b);
     a.grad_mse = reinterpret_cast<float*>(q + idx_b + coef_b);
     a.grad_div = reinterpret_cast<float*>(q + idx_b + coef_b + g_b);
+    a.div_scratch = q + idx_b + coef_b + 2 * g_b;
+    a.status = static_cast<uint32_t*>(base);
     a.losses = p->losses;
     a.lr = p->lr;
     a.beta = p->beta;
