@@ -143,7 +143,7 @@ typedef struct csr_reconstruct_params {
     int64_t ld_code;        /* elements between consecutive rows of idx and of coef; 0 = s */
     int64_t ld_xhat;        /* elements between consecutive rows of X_hat; 0 = d */
     const void* dict;       /* csr_dict_t* from csr_dict_create, or NULL: gather the atoms from the
-                               handle's bf16 copy of D instead of the fp32 D (see csr_reconstruct) */
+                               handle's fp16 copy of D instead of the fp32 D (see csr_reconstruct) */
 } csr_reconstruct_params_t;
 
 /*
@@ -171,13 +171,12 @@ int64_t csr_encode_workspace_bytes(int mode, int d, int N);
  * accumulated in fp32 in the order g = 0 .. s-1; repeated indices accumulate.  Every idx
  * must be < N (larger values are clamped to N-1 rather than read out of bounds).
  *
- * With params.dict (a handle of the same D, N, d) the atoms are read from the handle's bf16
- * copy, which halves the bytes gathered per row (what bounds this kernel from about s = 4
- * up).  The result is then Eq. 12 over the atoms rounded to bf16: it differs from the fp32-atom
- * result by at most 2^-8 * sum_g |coef_g * D[idx_g][k]| per channel k (bf16 keeps 8 significant
- * bits).  Codes made by the fast
- * mode were computed against exactly these rounded atoms, so for them this is the consistent
- * choice.
+ * With params.dict (a handle of the same D, N, d) the atoms are read from the handle's fp16
+ * copy of D, which halves the bytes gathered per row (what bounds this kernel from about
+ * s = 4 up) and, with fp16 coefficients, needs no conversion before the multiply.  The result
+ * is then Eq. 12 over the atoms rounded to fp16 (11 significant bits): it differs from the
+ * fp32-atom result by at most sum_g |coef_g| * (2^-11 * |D[idx_g][k]| + 2^-25) per channel k,
+ * well below the rounding of a bf16 or fp16 X_hat.
  *
  * 8-argument form: coef is fp16, X_hat is bf16, stream 0.
  */
@@ -210,7 +209,9 @@ int csr_decode_attention(const void* Dk, int Nk, const void* Dv, int Nv, int d, 
 int csr_pack_coefficients(const float* coef32, int64_t n, void* coef16, void* stream);
 
 /*
- * Prepared dictionary.  The fast mode works on a bf16 copy of D which the encode calls
+ * Prepared dictionary.  A handle holds two 16-bit copies of D: bf16 for the fast encoder and
+ * fp16 for the de-sparse kernel (params.dict of csr_reconstruct_ex).  The fast mode works on a
+ * bf16 copy of D which the encode calls
  * otherwise rebuild in scratch memory on every call (one extra launch of a few
  * microseconds: measured 83 -> 80 us on a 4160-row call, nothing on large ones).  A
  * dictionary is fixed for a layer's lifetime, so the copy can be made once and the encode

@@ -54,6 +54,8 @@ int launch_encode_exact_split(const EncodeArgs& a, void* scratch);
 // 1024-byte aligned); `status` is a device word that receives kStatusTimeout.
 int launch_encode_fast(const EncodeArgs& a, void* workspace, uint32_t* status);
 size_t encode_fast_workspace_bytes(int d, int N);
+// fp32 -> fp16 copy of D (round to nearest even), same [N][d] layout: the de-sparse kernel's gather source.
+int launch_dict_to_f16(const float* D, int N, int d, void* dst, cudaStream_t stream);
 // The two halves of launch_encode_fast: build the bf16 copy once, encode against it many times.
 int prepare_fast_dictionary(const float* D, int N, int d, void* workspace, cudaStream_t stream);
 // With few rows the dictionary is split across the CTAs of thread-block clusters (one launch,
@@ -67,7 +69,7 @@ size_t encode_fast_split_scratch_bytes(int64_t M, int d, int N);
 
 struct ReconstructArgs {
     const float* D;
-    const void* dict_bf16;   // bf16 copy of D ([N rounded up to 8][d]) to gather from instead, or NULL
+    const void* dict_f16;    // fp16 copy of D ([N][d]) to gather from instead, or NULL
     const uint16_t* idx;
     const void* coef;
     int coef_dtype;

@@ -16,7 +16,8 @@ struct csr_dict {
     const void* D;
     int N, d;
     void* raw;      // cudaMalloc'ed block
-    void* bf16;     // 1024-byte aligned copy inside it
+    void* bf16;     // 1024-byte aligned bf16 copy inside it (the fast encoder's operand)
+    void* f16;      // fp16 copy behind it (the de-sparse kernel's gather source)
 };
 
 namespace csr {
@@ -262,7 +263,7 @@ int check_reconstruct(const csr_reconstruct_params_t* p, bool host_io) {
 ReconstructArgs reconstruct_args(const csr_reconstruct_params_t* p) {
     ReconstructArgs a;
     a.D = static_cast<const float*>(p->D);
-    a.dict_bf16 = p->dict ? static_cast<const csr_dict*>(p->dict)->bf16 : nullptr;
+    a.dict_f16 = p->dict ? static_cast<const csr_dict*>(p->dict)->f16 : nullptr;
     a.idx = p->idx;
     a.coef = p->coef;
     a.coef_dtype = p->coef_dtype;
@@ -475,17 +476,21 @@ int csr_dict_create(const void* D, int N, int d, void* stream, csr_dict_t** out)
     if (int rc = current_device(&dev)) return rc;
     csr_dict* dc = new (std::nothrow) csr_dict();
     if (!dc) return fail(CSR_ERR_CUDA, "out of host memory");
-    cudaError_t e = cudaMalloc(&dc->raw, encode_fast_workspace_bytes(d, N) + 1024);
+    const size_t bf16_b = (encode_fast_workspace_bytes(d, N) + 1023) / 1024 * 1024;
+    cudaError_t e = cudaMalloc(&dc->raw, 1024 + bf16_b + (size_t)N * d * 2);
     if (e != cudaSuccess) {
         delete dc;
         return fail(CSR_ERR_CUDA, "cudaMalloc: %s", cudaGetErrorString(e));
     }
     dc->bf16 = align_up(dc->raw, 1024);
+    dc->f16 = static_cast<char*>(dc->bf16) + bf16_b;
     dc->device = dev;
     dc->D = D;
     dc->N = N;
     dc->d = d;
-    if (int rc = prepare_fast_dictionary(static_cast<const float*>(D), N, d, dc->bf16, static_cast<cudaStream_t>(stream))) {
+    int rc = prepare_fast_dictionary(static_cast<const float*>(D), N, d, dc->bf16, static_cast<cudaStream_t>(stream));
+    if (rc == CSR_OK) rc = launch_dict_to_f16(static_cast<const float*>(D), N, d, dc->f16, static_cast<cudaStream_t>(stream));
+    if (rc != CSR_OK) {
         cudaFree(dc->raw);
         delete dc;
         return rc;

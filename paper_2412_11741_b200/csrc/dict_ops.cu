@@ -56,6 +56,18 @@ __global__ void norm_deviation_kernel(const float* __restrict__ D, int N, uint32
     }
 }
 
+// fp32 -> fp16 copy of the dictionary (round to nearest even), four values per thread.
+__global__ void dict_to_f16_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, int64_t n_vec4) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec4; i += (int64_t)gridDim.x * blockDim.x) {
+        const float4 v = src[i];
+        __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t*>(&lo);
+        o.y = *reinterpret_cast<uint32_t*>(&hi);
+        dst[i] = o;
+    }
+}
+
 // Stored form of the coefficients ("Analysis for CSR": fp16 beside the 16-bit index): fp32 ->
 // fp16, round to nearest even, eight values per thread (two 16-byte loads, one 16-byte store).
 __global__ void pack_coef_kernel(const float4* __restrict__ src, uint4* __restrict__ dst, int64_t n8, const float* tail_src,
@@ -89,6 +101,16 @@ int launch_pack_coef(const float* coef32, int64_t n, void* coef16, cudaStream_t 
                                                      n8, coef32 + 8 * n8, reinterpret_cast<__half*>(coef16) + 8 * n8, tail);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "pack_coef launch: %s", cudaGetErrorString(e));
+    return CSR_OK;
+}
+
+int launch_dict_to_f16(const float* D, int N, int d, void* dst, cudaStream_t stream) {
+    const int64_t n_vec4 = (int64_t)N * d / 4;
+    int blocks = (int)((n_vec4 + 255) / 256);
+    if (blocks > 4 * sm_count()) blocks = 4 * sm_count();
+    dict_to_f16_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const float4*>(D), reinterpret_cast<uint2*>(dst), n_vec4);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "dict_to_f16 launch: %s", cudaGetErrorString(e));
     return CSR_OK;
 }
 

@@ -135,17 +135,21 @@ def test_reconstruct_one_million_rows_sampled(csr, d, N, s):
     csr.csr_reconstruct(Dd, idx16, coef16, X_hat=buf)
     assert bool(torch.isfinite(buf).all()) and torch.equal(buf, out16)
     del buf, out16
-    # atoms gathered from a prepared dictionary's bf16 copy: Eq. 12 over the rounded atoms, i.e.
-    # the oracle fed the bf16-rounded dictionary, to fp32 accuracy; and within the stated bound
-    # 2^-8 * sum_g |coef_g * atom_g[k]| of the fp32-atom result (bf16 keeps 8 significant bits)
+    # atoms gathered from a prepared dictionary's fp16 copy: Eq. 12 over the rounded atoms, i.e.
+    # the oracle fed the fp16-rounded dictionary, to fp32 accuracy; and within the stated bound
+    # sum_g |coef_g| (2^-11 |atom_g[k]| + 2^-25) of the fp32-atom result
     h = csr.csr_dict_create(Dd)
-    Db = wl.round_to_bf16(D)
-    refb = orc.reconstruct(Db, idx_s, coef_s.astype(np.float64))
-    outb = csr.csr_reconstruct_ex(Dd, idx16, coef, out_dtype=torch.float32, dict=h)
+    Dh = D.astype(np.float16).astype(np.float32)
+    refh = orc.reconstruct(Dh, idx_s, coef_s.astype(np.float64))
+    outb = csr.csr_reconstruct_ex(Dd, idx16, coef, out_dtype=torch.float32, dict=h)       # fp32 coefficients
     gotb = outb[st].cpu().numpy()
-    assert np.all(np.abs(gotb - refb) <= 2e-6 * scale)
-    bound = 2.0 ** -8 * (np.abs(coef_s.astype(np.float64))[:, :, None] * np.abs(D[idx_s].astype(np.float64))).sum(1)
+    assert np.all(np.abs(gotb - refh) <= 2e-6 * scale)
+    bound = (np.abs(coef_s.astype(np.float64))[:, :, None] * (2.0 ** -11 * np.abs(D[idx_s].astype(np.float64)) + 2.0 ** -25)).sum(1)
     assert np.all(np.abs(gotb - ref32) <= bound + 2e-6 * scale)
+    refh16 = orc.reconstruct(Dh, idx_s, coef16[st].float().cpu().numpy().astype(np.float64))
+    outh = csr.csr_reconstruct_ex(Dd, idx16, coef16, out_dtype=torch.float32, dict=h)      # fp16 coefficients: mixed-precision FMA
+    assert np.all(np.abs(outh[st].cpu().numpy() - refh16) <= 2e-6 * scale)
+    del outb, outh
     outb16 = csr.csr_reconstruct_ex(Dd, idx16, coef16, dict=h)
     assert torch.equal(outb16[st], csr.csr_reconstruct_ex(Dd, idx16, coef16, out_dtype=torch.float32, dict=h)[st].to(torch.bfloat16))
     with pytest.raises(csr.CsrError):
