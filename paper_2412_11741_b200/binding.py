@@ -283,13 +283,15 @@ def csr_encode_static(D: torch.Tensor, X: torch.Tensor, s: int, out_idx: torch.T
 
 
 def csr_encode_host(D: torch.Tensor, X_host: torch.Tensor, s: int, out_idx_host: torch.Tensor,
-                    out_coef_host: torch.Tensor, *, mode: int = CSR_MODE_BF16_FAST) -> None:
+                    out_coef_host: torch.Tensor, *, mode: int = CSR_MODE_BF16_FAST, dict: Optional[int] = None) -> None:
     """csr_encode_host: D on the device; X and the outputs are host tensors (pinned for speed).
     Returns after the codes have arrived in the host tensors."""
     assert D.is_cuda and not X_host.is_cuda and not out_idx_host.is_cuda and not out_coef_host.is_cuda
     assert X_host.is_contiguous() and out_idx_host.is_contiguous() and out_coef_host.is_contiguous()
     assert out_idx_host.dtype == torch.uint16 and tuple(out_idx_host.shape) == (X_host.shape[0], s)
     p = _encode_params(D, X_host, s, out_idx_host, out_coef_host, mode, None, None)
+    if dict is not None:
+        p.dict = dict
     with torch.cuda.device(D.device):
         _check(lib().csr_encode_host(ctypes.byref(p)))
 
@@ -470,7 +472,7 @@ def csr_reconstruct_ex(D: torch.Tensor, idx: torch.Tensor, coef: torch.Tensor, *
 
 
 def csr_reconstruct_host(D: torch.Tensor, idx_host: torch.Tensor, coef_host: torch.Tensor,
-                         X_hat_host: torch.Tensor) -> None:
+                         X_hat_host: torch.Tensor, *, dict: Optional[int] = None) -> None:
     """csr_reconstruct_host: D on the device; the codes and X_hat are host tensors (pinned for
     speed).  Returns after X_hat has arrived in the host tensor."""
     assert D.is_cuda and not idx_host.is_cuda and not coef_host.is_cuda and not X_hat_host.is_cuda
@@ -488,6 +490,8 @@ def csr_reconstruct_host(D: torch.Tensor, idx_host: torch.Tensor, coef_host: tor
     p.out_dtype = _TORCH_DTYPE[X_hat_host.dtype]
     p.M, p.d, p.N, p.s = M, d, N, s
     p.X_hat = X_hat_host.data_ptr()
+    if dict is not None:
+        p.dict = dict
     with torch.cuda.device(D.device):
         _check(lib().csr_reconstruct_host(ctypes.byref(p)))
 

@@ -1020,8 +1020,8 @@ int launch(const EncodeArgs& a, const CUtensorMap& tmap, const uint16_t* Db, uin
 int group_size(int d, int N) {
     const int v = options().fast_group;
     if (v == 1 || v == 2 || v == 4 || v == 8) return v;
-    if (d == 64) return 4;
-    return N >= 16384 ? 4 : 1;
+    if (d == 64) return N <= 2048 ? 2 : 4;
+    return 1;
 }
 
 template <int D_>

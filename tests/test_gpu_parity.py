@@ -593,6 +593,14 @@ def test_host_entry_point(csr):
     xh32 = torch.empty((w.M, w.d), dtype=torch.float32)          # pageable memory and fp32 output work too
     csr.csr_reconstruct_host(D, oi, oc, xh32)
     assert torch.equal(xh32, csr.csr_reconstruct_ex(D, idx, coef, out_dtype=torch.float32).cpu())
+    # with a prepared dictionary: the same codes, and the fp16-atom restore of the device entry point
+    h = csr.csr_dict_create(D)
+    oi2, oc2 = torch.zeros_like(oi), torch.zeros_like(oc)
+    csr.csr_encode_host(D, Xh, w.s, oi2, oc2, dict=h)
+    assert np.array_equal(_np_idx(oi2), _np_idx(idx)) and torch.equal(oc2, coef.cpu())
+    csr.csr_reconstruct_host(D, oi, oc, xh_host, dict=h)
+    assert torch.equal(xh_host.view(torch.int16), csr.csr_reconstruct_ex(D, idx, coef, dict=h).cpu().view(torch.int16))
+    csr.csr_dict_destroy(h)
 
 
 @pytest.mark.parametrize("seed", range(24))
