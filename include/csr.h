@@ -66,6 +66,7 @@ extern "C" {
 #define CSR_ERR_CUDA (-4)
 #define CSR_ERR_TIMEOUT (-5)
 #define CSR_ERR_WORKSPACE (-6)
+#define CSR_ERR_BOUNDS (-7)
 
 /* element types of X and X_hat (any of the three) and of coef (F32 or F16) */
 #define CSR_DTYPE_F32 0
@@ -420,7 +421,11 @@ int csr_set_option(const char* name, int64_t value);
 /*
  * Synchronises the stream and reports whether a kernel of this library has given up on a
  * bounded wait since the last call of this function on the current device: CSR_OK or
- * CSR_ERR_TIMEOUT (or CSR_ERR_CUDA if the stream itself is in error).  Reads the library's
+ * CSR_ERR_TIMEOUT (or CSR_ERR_CUDA if the stream itself is in error).  A library built with
+ * device-side checks (csr_debug_checks() == 1) also reports CSR_ERR_BOUNDS here: an index that a
+ * kernel was about to gather with was out of range (an idx >= N given to csr_reconstruct, a
+ * candidate atom past the dictionary in the fast encoder); the release build clamps such
+ * indices silently, the checked build clamps and records.  Reads the library's
  * status word(s); a call that was given its own dev_status reports there instead.
  */
 int csr_device_status(void* stream);
@@ -430,6 +435,8 @@ int csr_release_workspace(void);
 
 const char* csr_last_error_string(void);
 int csr_version(void);
+/* 1 if this library was built with the device-side index checks (build.py --debug), else 0. */
+int csr_debug_checks(void);
 
 #ifdef __cplusplus
 }

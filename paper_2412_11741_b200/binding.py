@@ -14,7 +14,9 @@ from typing import Optional, Tuple
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libcsr.so")
+# CSR_LIBRARY_PATH selects another build of the same library (e.g. libcsr_debug.so, built with
+# device-side index checks by `python -m paper_2412_11741_b200.build --debug`)
+LIB_PATH = os.environ.get("CSR_LIBRARY_PATH") or os.path.join(_PKG, "libcsr.so")
 
 CSR_OK = 0
 CSR_ERR_INVALID_ARG = -1
@@ -23,6 +25,7 @@ CSR_ERR_ALIGNMENT = -3
 CSR_ERR_CUDA = -4
 CSR_ERR_TIMEOUT = -5
 CSR_ERR_WORKSPACE = -6
+CSR_ERR_BOUNDS = -7
 
 CSR_DTYPE_F32 = 0
 CSR_DTYPE_BF16 = 1
@@ -34,7 +37,7 @@ CSR_MODE_BF16_FAST = 1
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
     "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_decode_attention", "csr_dict_append", "csr_dict_create", "csr_dict_destroy", "csr_dict_train_step", "csr_key_scores", "csr_pack_coefficients", "csr_value_mix",
-    "csr_encode_static", "csr_dict_check_norms", "csr_set_option", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version",
+    "csr_encode_static", "csr_dict_check_norms", "csr_set_option", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version", "csr_debug_checks",
 )
 
 
@@ -144,6 +147,8 @@ def lib() -> ctypes.CDLL:
         L.csr_last_error_string.restype = ctypes.c_char_p
         L.csr_version.argtypes = []
         L.csr_version.restype = i32
+        L.csr_debug_checks.argtypes = []
+        L.csr_debug_checks.restype = i32
         _lib = L
     return _lib
 
@@ -154,6 +159,10 @@ def csr_last_error_string() -> str:
 
 def csr_version() -> int:
     return int(lib().csr_version())
+
+
+def csr_debug_checks() -> bool:
+    return bool(lib().csr_debug_checks())
 
 
 def _check(rc: int) -> None:

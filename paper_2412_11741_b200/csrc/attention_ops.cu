@@ -16,10 +16,11 @@
 // value_mix: (1) every code stream is cut into `pieces` token ranges, one CTA each, which
 // scatters w * coef into a[head][N] in shared memory with atomic adds while it streams the
 // codes and then stores its a to the scratch array [B][pieces][H][N]; (2) out = a D with the
-// pieces summed in order on the way in, a small fp32 GEMM (split over atoms with atomic
-// adds when there are few heads).  The tables are accumulated in fixed point (see
-// value_scatter_kernel) and are the same on every run; the split over atoms of step (2),
-// when it is used, still adds in an order that varies.
+// pieces summed in order on the way in, a small fp32 GEMM (split into slices of the atoms
+// when there are few heads; the slices' partial results are then added in slice order by
+// add_slices_kernel).  The tables are accumulated in fixed point (see value_scatter_kernel),
+// and every floating-point sum is taken in a fixed order, so the result is the same bits on
+// every run.
 #include "exact_common.cuh"
 
 namespace csr {

@@ -15,6 +15,9 @@ int fail(int code, const char* fmt, ...);
 
 // Device status word written by kernels whose bounded waits expire.
 constexpr uint32_t kStatusTimeout = 1u;
+// Raised only by a library built with CSR_DEBUG_CHECKS (python -m paper_2412_11741_b200.build
+// --debug): an index about to be used for a gather was out of range and has been clamped.
+constexpr uint32_t kStatusBounds = 2u;
 
 // Process-wide switches set through csr_set_option (plain loads on the call path).
 struct Options {
@@ -79,6 +82,7 @@ struct ReconstructArgs {
     void* X_hat;
     int64_t ld_code;   // elements between consecutive rows of idx and of coef (>= s)
     int64_t ld_xhat;   // elements between consecutive rows of X_hat (>= d)
+    uint32_t* status;  // debug builds: the word that records a clamped index; else NULL
     cudaStream_t stream;
 };
 int launch_reconstruct(const ReconstructArgs& a);

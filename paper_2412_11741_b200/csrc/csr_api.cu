@@ -276,6 +276,11 @@ ReconstructArgs reconstruct_args(const csr_reconstruct_params_t* p) {
     a.ld_code = p->ld_code ? p->ld_code : p->s;
     a.ld_xhat = p->ld_xhat ? p->ld_xhat : p->d;
     a.stream = static_cast<cudaStream_t>(p->stream);
+    a.status = nullptr;
+#ifdef CSR_DEBUG_CHECKS
+    void* base = nullptr;                                     // the debug build reports clamped indices in the library's word
+    if (ensure_work(0, &base, a.stream) == CSR_OK) a.status = static_cast<uint32_t*>(base);
+#endif
     return a;
 }
 
@@ -403,6 +408,14 @@ using namespace csr;
 extern "C" {
 
 int csr_version(void) { return CSR_VERSION; }
+
+int csr_debug_checks(void) {
+#ifdef CSR_DEBUG_CHECKS
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 const char* csr_last_error_string(void) { return g_err; }
 
@@ -843,7 +856,10 @@ int csr_device_status(void* stream) {
         if (st != 0) cudaMemset(work, 0, kStatusBytes);
         seen |= st;
     }
-    if (seen != 0) return fail(CSR_ERR_TIMEOUT, "a device-side wait expired (status word 0x%x)", seen);
+    if (seen & kStatusTimeout) return fail(CSR_ERR_TIMEOUT, "a device-side wait expired (status word 0x%x)", seen);
+    if (seen & kStatusBounds)
+        return fail(CSR_ERR_BOUNDS, "an index used for a gather was out of range and was clamped (status word 0x%x)", seen);
+    if (seen != 0) return fail(CSR_ERR_CUDA, "unknown device status 0x%x", seen);
     return CSR_OK;
 }
 

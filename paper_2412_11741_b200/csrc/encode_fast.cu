@@ -119,6 +119,20 @@ __device__ __forceinline__ uint32_t swz_off(int r, int chunk) {
     return khalf * (TILE_M * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
 }
 
+// First atom of the group a (key, tile) pair names.  Whatever the keys say (NaN correlations can
+// make a zero-filled column past the dictionary win) the gather that follows stays inside the
+// padded bf16 copy; a build with CSR_DEBUG_CHECKS also records that the clamp was needed.
+template <int G>
+__device__ __forceinline__ int candidate_start(uint32_t best_key, uint32_t best_t, int N, [[maybe_unused]] uint32_t* status) {
+    constexpr int NG = TILE_N / G;
+    const int n0 = static_cast<int>(best_t) * TILE_N + (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G;
+    const int last = ((N + 7) / 8) * 8 - G;
+#ifdef CSR_DEBUG_CHECKS
+    if (n0 > last || n0 < 0) atomicOr(status, kStatusBounds);
+#endif
+    return min(n0, last);
+}
+
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -780,9 +794,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                     best_key = static_cast<uint32_t>(mine >> 32);
                     best_t = 0xFFFFFFFFu - static_cast<uint32_t>(mine);
                     if (acc == 0) {
-                        pick_n0[r] = min(static_cast<int>(best_t) * TILE_N +
-                                             (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G,
-                                         ((N + 7) / 8) * 8 - G);
+                        pick_n0[r] = candidate_start<G>(best_key, best_t, N, status);
                         mbar_arrive(&sm.pick_bar);
                         row_mask &= 0x0000FFFFu;
                     } else {
@@ -836,11 +848,7 @@ encode_fast_kernel(const __grid_constant__ CUtensorMap tmap_d, const uint16_t* _
                 }
                 // ---- pick, signed coefficient, residual update ----
                 const int gi = g & (CODE_BLOCK - 1);
-                // (NaN correlations can make a zero-filled column past the dictionary win: keep the
-                // gather inside the padded bf16 copy whatever the keys say)
-                int n0 = min(static_cast<int>(best_t) * TILE_N +
-                                 (NG - 1 - static_cast<int>(best_key & static_cast<uint32_t>(NG - 1))) * G,
-                             ((N + 7) / 8) * 8 - G);
+                int n0 = candidate_start<G>(best_key, best_t, N, status);
                 if (CL == 2 && acc == 1) n0 = n0_other;
                 if constexpr (CL)
                     pick_and_update<D_, G, true>(Atile, q, lane, Db, n0, g + 1 < s, code_idx, code_coef, gi, row_mask);

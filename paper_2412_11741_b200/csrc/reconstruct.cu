@@ -143,7 +143,7 @@ __device__ __forceinline__ void stage_codes(uint16_t* s_idx, unsigned char* s_co
 template <int CH, int LPR, typename P>
 __device__ __forceinline__ void rows_generic(const uint4* __restrict__ Dl, const uint16_t* ci, const unsigned char* cc,
                                              int cbytes, int s, int N, const int (&r)[PP], const bool (&valid)[PP],
-                                             float (&acc)[PP][CH]) {
+                                             float (&acc)[PP][CH], [[maybe_unused]] uint32_t* status) {
     for (int g0 = 0; g0 < s; g0 += INFLIGHT) {
         uint4 v[PP][INFLIGHT];
         float c[PP][INFLIGHT];
@@ -156,6 +156,9 @@ __device__ __forceinline__ void rows_generic(const uint4* __restrict__ Dl, const
                 c[w][u] = 0.f;
                 if (g < s && valid[w]) {
                     const int i = min(static_cast<int>(ci[r[w] * s + g]), N - 1);
+#ifdef CSR_DEBUG_CHECKS
+                    if (static_cast<int>(ci[r[w] * s + g]) >= N) atomicOr(status, kStatusBounds);
+#endif
                     c[w][u] = cbytes == 2 ? __half2float(reinterpret_cast<const __half*>(cc)[r[w] * s + g])
                                           : reinterpret_cast<const float*>(cc)[r[w] * s + g];
                     v[w][u] = __ldg(Dl + static_cast<size_t>(i) * LPR);
@@ -174,7 +177,7 @@ __device__ __forceinline__ void rows_generic(const uint4* __restrict__ Dl, const
 // is predicated.
 template <int CH, int LPR, typename P, bool COEF16>
 __device__ __forceinline__ void rows_by_four(const uint4* __restrict__ Dl, const uint16_t* ci, const unsigned char* cc, int s,
-                                             int N, const int (&r)[PP], float (&acc)[PP][CH]) {
+                                             int N, const int (&r)[PP], float (&acc)[PP][CH], [[maybe_unused]] uint32_t* status) {
     static_assert(INFLIGHT == 4, "four steps per trip");
     constexpr bool RAW16 = COEF16 && CH == 8;             // fp16 coefficients meet fp16 atoms: no conversion
     using CoefT = typename std::conditional<RAW16, uint16_t, float>::type;
@@ -208,6 +211,10 @@ __device__ __forceinline__ void rows_by_four(const uint4* __restrict__ Dl, const
             }
             const int i0 = min(static_cast<int>(iw.x & 0xFFFFu), nmax), i1 = min(static_cast<int>(iw.x >> 16), nmax);
             const int i2 = min(static_cast<int>(iw.y & 0xFFFFu), nmax), i3 = min(static_cast<int>(iw.y >> 16), nmax);
+#ifdef CSR_DEBUG_CHECKS
+            if (static_cast<int>(max(max(iw.x & 0xFFFFu, iw.x >> 16), max(iw.y & 0xFFFFu, iw.y >> 16))) > nmax)
+                atomicOr(status, kStatusBounds);
+#endif
             v[w][0] = __ldg(Dl + static_cast<uint32_t>(i0 * LPR));
             v[w][1] = __ldg(Dl + static_cast<uint32_t>(i1 * LPR));
             v[w][2] = __ldg(Dl + static_cast<uint32_t>(i2 * LPR));
@@ -224,7 +231,7 @@ template <int D_, bool F16>
 __global__ void __launch_bounds__(NT, F16 ? 3 : 4)
 reconstruct_kernel(const void* __restrict__ Dict, const uint16_t* __restrict__ idx, const void* __restrict__ coef,
                    int coef_dtype, int64_t ldc, int64_t M, int N, int s, void* __restrict__ X_hat, int out_dtype,
-                   int64_t ldxh, int dense_codes) {
+                   int64_t ldxh, int dense_codes, uint32_t* status) {
     using P = Piece<F16>;
     constexpr int CH = P::CH;                             // channels per lane
     constexpr int LPR = D_ / CH;                          // lanes per row: 32, 16 or 8
@@ -275,11 +282,11 @@ reconstruct_kernel(const void* __restrict__ Dict, const uint16_t* __restrict__ i
             }
             if (whole && by_four) {
                 if (cbytes == 2)
-                    rows_by_four<CH, LPR, P, true>(Dl, ci, cc, s, N, r, acc);
+                    rows_by_four<CH, LPR, P, true>(Dl, ci, cc, s, N, r, acc, status);
                 else
-                    rows_by_four<CH, LPR, P, false>(Dl, ci, cc, s, N, r, acc);
+                    rows_by_four<CH, LPR, P, false>(Dl, ci, cc, s, N, r, acc, status);
             } else {
-                rows_generic<CH, LPR, P>(Dl, ci, cc, cbytes, s, N, r, valid, acc);
+                rows_generic<CH, LPR, P>(Dl, ci, cc, cbytes, s, N, r, valid, acc, status);
             }
 #pragma unroll
             for (int w = 0; w < PP; ++w)
@@ -317,7 +324,7 @@ int launch_t(const ReconstructArgs& a, const void* dict) {
     const uintptr_t pi = reinterpret_cast<uintptr_t>(a.idx), pc = reinterpret_cast<uintptr_t>(a.coef);
     const int dense = a.ld_code == a.s && pi % 16 == 0 && pc % 16 == 0;
     reconstruct_kernel<D_, F16><<<grid, NT, smem, a.stream>>>(dict, a.idx, a.coef, a.coef_dtype, a.ld_code, a.M, a.N, a.s,
-                                                              a.X_hat, a.out_dtype, a.ld_xhat, dense);
+                                                              a.X_hat, a.out_dtype, a.ld_xhat, dense, a.status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "reconstruct launch: %s", cudaGetErrorString(e));
     return CSR_OK;
