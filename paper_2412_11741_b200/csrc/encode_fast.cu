@@ -189,16 +189,26 @@ __device__ __forceinline__ void chunk_key_max(const uint32_t (&v)[32], uint32_t 
     }
 }
 
+// even += lo(r) * lo(a), odd += hi(r) * hi(a) for one word of two bf16 values each: the product of
+// two bf16 values is exact in fp32 and the sum is rounded once (the value fmaf gives on the widened
+// operands), and the mixed-precision instruction takes the 16-bit halves as they are.
+__device__ __forceinline__ void fma2_bf16(float& even, float& odd, uint32_t r, uint32_t a) {
+    asm("{\n"
+        ".reg .b16 rl, rh, al, ah;\n"
+        "mov.b32 {rl, rh}, %2;\n"
+        "mov.b32 {al, ah}, %3;\n"
+        "fma.rn.f32.bf16 %0, rl, al, %0;\n"
+        "fma.rn.f32.bf16 %1, rh, ah, %1;\n"
+        "}\n"
+        : "+f"(even), "+f"(odd)
+        : "r"(r), "r"(a));
+}
 // fp32 dot product of eight bf16 pairs (one 16-byte chunk of a residual row and of an atom)
 __device__ __forceinline__ void dot8(const uint4& rv, const uint4& av, float& even, float& odd) {
-    even = fmaf(bf_lo(rv.x), bf_lo(av.x), even);
-    odd = fmaf(bf_hi(rv.x), bf_hi(av.x), odd);
-    even = fmaf(bf_lo(rv.y), bf_lo(av.y), even);
-    odd = fmaf(bf_hi(rv.y), bf_hi(av.y), odd);
-    even = fmaf(bf_lo(rv.z), bf_lo(av.z), even);
-    odd = fmaf(bf_hi(rv.z), bf_hi(av.z), odd);
-    even = fmaf(bf_lo(rv.w), bf_lo(av.w), even);
-    odd = fmaf(bf_hi(rv.w), bf_hi(av.w), odd);
+    fma2_bf16(even, odd, rv.x, av.x);
+    fma2_bf16(even, odd, rv.y, av.y);
+    fma2_bf16(even, odd, rv.z, av.z);
+    fma2_bf16(even, odd, rv.w, av.w);
 }
 // r -= coef * a on one 16-byte chunk, rounded back to bf16
 __device__ __forceinline__ uint4 axpy8(const uint4& rv, const uint4& av, float coef) {
