@@ -208,6 +208,27 @@ def test_training_step_at_2048_atoms(csr, mode_name):
     assert np.abs(want - D0).max() > 2e-3 and np.abs(got - want).max() <= 1e-6
 
 
+@pytest.mark.parametrize("N,d", [(4200, 128), (2500, 64)])
+def test_diversity_step_alone_ragged_and_in_several_passes(csr, N, d):
+    """The diversity term by itself (an empty batch) on dictionaries whose size is no multiple of
+    the kernels' 128-atom blocks; at N = 4200, d = 128 the scratch copy of D D^T - I is filled and
+    consumed in two passes of rows.  Against the oracle's loss and gradient, to the tolerance of
+    the full step."""
+    rng = np.random.default_rng(N)
+    D0 = wl.normalise_rows(rng.standard_normal((N, d)).astype(np.float32) + np.float32(0.3))    # coherent atoms: a large gradient
+    l_div, g_div = orc.div_loss_and_grad(D0)
+    lr, beta = 2000.0, 0.5
+    Dd = torch.from_numpy(D0.copy()).to(DEV)
+    X0 = torch.empty((0, d), dtype=torch.float32, device=DEV)
+    losses = csr.csr_dict_train_step(Dd, X0, 4, lr, beta).cpu().numpy()
+    assert csr.csr_device_status() == csr.CSR_OK
+    W = D0.astype(np.float64) - lr * beta * g_div
+    want = (W / np.linalg.norm(W, axis=1, keepdims=True)).astype(np.float32)
+    got = Dd.cpu().numpy()
+    assert losses[0] == 0.0 and losses[1] == pytest.approx(l_div, rel=2e-5)
+    assert np.abs(want - D0).max() > 2e-3 and np.abs(got - want).max() <= 1e-6, (float(np.abs(want - D0).max()), float(np.abs(got - want).max()))
+
+
 # ---------------------------------------------------------------------------------------
 # robustness
 # ---------------------------------------------------------------------------------------
