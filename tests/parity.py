@@ -8,6 +8,12 @@ Rules (derived from the stated tolerances):
       |correlations| differ by less than 1e-6 relative (or its residual is numerically
       zero) a different pick is allowed; comparison of that vector stops there and its
       reconstruction error must then be within [0.75, 1.25] of the oracle's;
+    - the same where the oracle's winning correlation is itself below the rounding error of
+      its own evaluation, |c_g| <= 8 d 2^-53 ||R_g|| (a d-term fp64 dot product of a residual
+      of that size): with a handful of atoms and many iterations the residual ends up
+      orthogonal to every atom, the correlations are 1e-16 ||x|| and below, and the oracle
+      itself changes its pick when its channels are summed in another order
+      (tests/test_parity_rules.py shows it);
     - coefficients: |c - c_oracle| <= 1e-4 |c_oracle| + 1e-6 ||x||.
   fast (bf16-operand) mode
     - mean reconstruction error over the sample within 1 % of the oracle's mean;
@@ -25,9 +31,13 @@ Rules (derived from the stated tolerances):
       the largest value a bf16 emulation of the pursuit reaches on samples of every
       configuration (tests/test_parity_rules.py measures it);
     - the error ratio of a divergent vector (the two greedy trajectories legitimately
-      differ after a near-tie) stays within fast_ratio_cap(s) and, on samples of at least
-      512 rows, the 99th percentile within fast_ratio_p99_cap(s); the emulation's own
-      ratios set these numbers (same test).
+      differ after a near-tie) stays within 1 + 0.12 / e (at most 1.5) and, on samples of at
+      least 512 rows, the 99th percentile within 1 + 0.035 / e, e being the oracle's mean
+      relative error on the sample: a different atom at a near-tie changes a vector's final
+      error by an amount that does not shrink with the error itself, so the RATIO spreads as
+      the error falls.  The bf16 emulation's own ratios set the two constants: its
+      (p99 - 1) e is 0.018-0.022 and its (max - 1) e at most 0.092 on every configuration and
+      on d = 64 dictionaries of 5000 atoms at s = 12-16 (same test).
 """
 from __future__ import annotations
 
@@ -55,7 +65,9 @@ def compare_exact(D, X, s, idx_gpu, coef_gpu, res=None) -> ExactReport:
     M = X.shape[0]
     xnorm = np.linalg.norm(X.astype(np.float64), axis=1)
     prev_norm = np.concatenate([xnorm[:, None], res.resnorm[:, :-1]], axis=1)
-    exempt_step = (res.gap < 1e-6) | (prev_norm < 1e-6 * xnorm[:, None])
+    d = X.shape[1]
+    noise_step = np.abs(res.coef) <= 8.0 * d * 2.0 ** -53 * prev_norm        # the pick is decided by fp64 rounding
+    exempt_step = (res.gap < 1e-6) | (prev_norm < 1e-6 * xnorm[:, None]) | noise_step
     differ = idx_gpu != res.idx
     first = np.where(differ.any(1), differ.argmax(1), s)          # first differing step, s if none
     rows = np.arange(M)
@@ -90,8 +102,13 @@ def compare_exact(D, X, s, idx_gpu, coef_gpu, res=None) -> ExactReport:
         if np.any((ratio < 0.75) | (ratio > 1.25)):
             detail.append(f"excused rows with error ratio outside [0.75,1.25]: {ratio}")
             ok = False
-    if excused.sum() > max(4, 2e-3 * M * s):
-        detail.append(f"too many tie-excused rows: {int(excused.sum())} of {M}")
+    # near-ties must be rare (many of them mean a bug, not ties); steps below the oracle's own
+    # noise floor are not ties and are not counted
+    by_noise = np.zeros(M, bool)
+    by_noise[has_diff] = noise_step[rows[has_diff], first[has_diff]]
+    ties = excused & ~by_noise
+    if ties.sum() > max(4, 2e-3 * M * s):
+        detail.append(f"too many tie-excused rows: {int(ties.sum())} of {M}")
         ok = False
     return ExactReport(M, int(excused.sum()), int(unexplained.sum()), float(rel.max()) if rel.size else 0.0, ok,
                        "; ".join(detail))
@@ -117,15 +134,15 @@ class FastReport:
 FAST_GAP_C = 2.5
 
 
-def fast_ratio_cap(s: int) -> float:
-    """Largest error ratio a divergent vector may end with (emulation: 1.17 at s <= 8, 1.25 at
-    s = 16, 1.37 at s = 32 on 2048 to 4096 rows)."""
-    return 1.25 if s <= 8 else 1.3 if s <= 16 else 1.5
+FAST_RATIO_MAX_C = 0.12
+FAST_RATIO_P99_C = 0.035
 
 
-def fast_ratio_p99_cap(s: int) -> float:
-    """99th percentile of the error ratio over a sample (emulation: 1.05 up to s = 16, 1.12 at s = 32)."""
-    return 1.08 if s <= 16 else 1.18
+def fast_ratio_caps(mean_err: float):
+    """(largest error ratio a divergent vector may end with, 99th percentile of the ratio over a
+    sample) for a sample whose oracle mean relative error is mean_err."""
+    e = max(float(mean_err), 1e-3)
+    return min(1.5, 1.0 + FAST_RATIO_MAX_C / e), min(1.5, 1.0 + FAST_RATIO_P99_C / e)
 
 
 def first_divergence_margin(res, xnorm, rows, steps):
@@ -173,13 +190,13 @@ def compare_fast(D, X, s, idx_gpu, coef_gpu, res=None, gap_c=FAST_GAP_C) -> Fast
         detail.append(f"row {int(rows_div[j])} diverges at step {int(first[rows_div[j]])} where the oracle's best two atoms are "
                       f"{max_margin:.2f} accumulated bf16 roundings apart (> {gap_c}); relative gap {float(gaps[j]):.4f}")
         ok = False
-    cap = fast_ratio_cap(s)
+    cap, p99_cap = fast_ratio_caps(float(e_or[live].mean()) if live.any() else 1.0)
     if div.any() and (ratio[div].max() > cap or ratio[div].min() < 1.0 / cap):
-        detail.append(f"a divergent vector has error ratio {ratio[div].max():.3f} / {ratio[div].min():.3f} (outside [1/{cap}, {cap}])")
+        detail.append(f"a divergent vector has error ratio {ratio[div].max():.3f} / {ratio[div].min():.3f} (outside [1/{cap:.3f}, {cap:.3f}])")
         ok = False
     p99 = float(np.percentile(ratio, 99))
-    if M >= 512 and p99 > fast_ratio_p99_cap(s):
-        detail.append(f"99th percentile of the error ratio {p99:.3f} (> {fast_ratio_p99_cap(s)})")
+    if M >= 512 and p99 > p99_cap:
+        detail.append(f"99th percentile of the error ratio {p99:.3f} (> {p99_cap:.3f})")
         ok = False
     return FastReport(M, int(same.sum()), float(e_gpu.mean()), float(e_or.mean()), mean_ratio, same_dev,
                       float(np.percentile(ratio, 50)), p99, float(ratio.max()), max_gap,

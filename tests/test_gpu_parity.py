@@ -603,7 +603,9 @@ def test_host_entry_point(csr):
     csr.csr_dict_destroy(h)
 
 
-@pytest.mark.parametrize("seed", range(24))
+# (114, 141, 534: two atoms and many iterations, the picks end up below the oracle's own rounding noise;
+# 214, 421: an overcomplete d = 64 dictionary taken to a small error, where the error ratios spread)
+@pytest.mark.parametrize("seed", list(range(24)) + [114, 141, 214, 421, 534])
 def test_random_shapes_both_modes(csr, seed):
     """Seeded random (M, N, d, s, input type) combinations, ragged in every dimension, through
     both encoders and the de-sparse kernel against the oracle."""
