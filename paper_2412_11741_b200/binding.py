@@ -229,6 +229,8 @@ def _encode_params(D, X, s, out_idx, out_coef, mode, stream, workspace) -> csr_e
     if out_idx.shape[0] > 1 and out_idx.stride(0) != s:
         assert out_coef.stride(0) == out_idx.stride(0), "out_idx and out_coef must share their row stride"
         p.ld_code = out_idx.stride(0)
+    elif out_idx.data_ptr() % 16 or out_coef.data_ptr() % 16:
+        p.ld_code = s                                     # a view into wider arrays: element alignment is enough
     if workspace is not None:
         p.workspace = workspace.data_ptr()
         p.workspace_bytes = workspace.numel() * workspace.element_size()
@@ -327,6 +329,8 @@ def _reconstruct_params(D, idx, coef, out_dtype, X_hat):
     if M > 1 and idx.stride(0) != s:
         assert coef.stride(0) == idx.stride(0), "idx and coef must share their row stride"
         p.ld_code = idx.stride(0)
+    elif idx.data_ptr() % 16 or coef.data_ptr() % 16:
+        p.ld_code = s                                     # a view into wider arrays: element alignment is enough
     if M > 1 and X_hat.stride(0) != d:
         p.ld_xhat = X_hat.stride(0)
     return p, X_hat
