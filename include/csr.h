@@ -57,7 +57,7 @@
 extern "C" {
 #endif
 
-#define CSR_VERSION 110
+#define CSR_VERSION 120
 
 #define CSR_OK 0
 #define CSR_ERR_INVALID_ARG (-1)
@@ -75,17 +75,25 @@ extern "C" {
 
 /*
  * Arithmetic mode of the encoder.
- *   CSR_MODE_FP32_EXACT  correlations with fp32 operands and fp32 accumulation on the
- *                        plain ALUs; whenever the two largest |correlations| of a row
- *                        are closer than fp32 rounding can resolve, that row's step is
- *                        re-scored in fp64.  The coefficient and the residual update
- *                        are fp64.  Selects the same atoms as an fp64 evaluation of the
- *                        pursuit except at exact-to-rounding ties.
- *                        With few rows (the vectors one decoding step adds: fewer row
- *                        tiles of 64 than half the SMs) the dictionary is split across
- *                        the SMs instead of the rows, two launches per iteration, with
- *                        identical codes; this path uses the library-owned scratch
- *                        (not taken when a caller workspace is given).
+ *   CSR_MODE_FP32_EXACT  selects the same atoms as an fp64 evaluation of the pursuit except
+ *                        at exact-to-rounding ties; the coefficient and the residual
+ *                        update are fp64.  Every correlation of a sweep is computed to
+ *                        within a known band, and whenever the largest |correlations| of a
+ *                        row are closer than that band the candidates are re-scored in
+ *                        fp64.  Three encoders do this, with identical codes:
+ *                        (a) sweep on the tcgen05 tensor cores, residual and atoms each
+ *                        split into a bf16 high and low part, three bf16 products per
+ *                        correlation accumulated in fp32 (band 2^-12 * ||R||): the default
+ *                        where the library-owned scratch is in use (no caller workspace;
+ *                        about 4 * N * d + 2048 * d * min(ceil(M / 256), SMs) bytes of it);
+ *                        (b) fp32 operands and fp32 accumulation on the plain ALUs (band
+ *                        1.6e-5 * ||R||), one CTA per 64 rows, no scratch: taken when a
+ *                        caller workspace is given;
+ *                        (c) with few rows (the vectors one decoding step adds: fewer row
+ *                        tiles of 64 than half the SMs) the plain-ALU sweep with the
+ *                        dictionary split across the SMs instead of the rows, two launches
+ *                        per iteration; library-owned scratch, not taken when a caller
+ *                        workspace is given.
  *   CSR_MODE_BF16_FAST   correlations on the tcgen05 tensor cores with bf16 operands
  *                        (residual and atoms rounded to bf16) and fp32 accumulation.
  *                        Near-tied picks may differ from an fp64 evaluation; the mean
@@ -408,6 +416,8 @@ int csr_dict_check_norms(const void* D, int N, int d, float tol, void* stream, f
  *                    1 = always one CTA per pair of row tiles over the whole dictionary,
  *                    2 = no clusters;
  *   "exact_split"    0 (default: the exact mode splits the dictionary for few rows), 1 = never;
+ *   "exact_engine"   0 (default: the exact mode's tensor-core encoder unless the rows are few),
+ *                    1 = plain-ALU encoders only, 2 = the tensor-core encoder also with few rows;
  *   "wait_limit_ns"  bound of every device-side wait of the fast encoder in nanoseconds
  *                    (default 2e9).  0 lets no wait outlast a single look at its barrier, so
  *                    the first hand-off that is not already complete expires: the call
@@ -437,6 +447,14 @@ const char* csr_last_error_string(void);
 int csr_version(void);
 /* 1 if this library was built with the device-side index checks (build.py --debug), else 0. */
 int csr_debug_checks(void);
+/*
+ * Quantities only a checked build records (CSR_ERR_UNSUPPORTED otherwise); reading one
+ * synchronises the device and resets it.
+ *   "exact_tensor_error"  the largest | tensor-core correlation - fp64 correlation | / ||R||
+ *                         over the picks the exact mode's tensor-core encoder took without
+ *                         re-scoring since the last read (must stay below half the band).
+ */
+int csr_debug_read(const char* name, double* value);
 
 #ifdef __cplusplus
 }

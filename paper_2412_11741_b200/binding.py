@@ -37,7 +37,7 @@ CSR_MODE_BF16_FAST = 1
 EXPORTS = (
     "csr_encode", "csr_encode_ex", "csr_encode_workspace_bytes", "csr_reconstruct", "csr_reconstruct_ex",
     "csr_encode_host", "csr_reconstruct_host", "csr_encode_grouped", "csr_reconstruct_grouped", "csr_decode_attention", "csr_dict_append", "csr_dict_create", "csr_dict_destroy", "csr_dict_train_step", "csr_key_scores", "csr_pack_coefficients", "csr_value_mix",
-    "csr_encode_static", "csr_dict_check_norms", "csr_set_option", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version", "csr_debug_checks",
+    "csr_encode_static", "csr_dict_check_norms", "csr_set_option", "csr_device_status", "csr_release_workspace", "csr_last_error_string", "csr_version", "csr_debug_checks", "csr_debug_read",
 )
 
 
@@ -149,6 +149,8 @@ def lib() -> ctypes.CDLL:
         L.csr_version.restype = i32
         L.csr_debug_checks.argtypes = []
         L.csr_debug_checks.restype = i32
+        L.csr_debug_read.argtypes = [ctypes.c_char_p, ctypes.POINTER(ctypes.c_double)]
+        L.csr_debug_read.restype = i32
         _lib = L
     return _lib
 
@@ -163,6 +165,13 @@ def csr_version() -> int:
 
 def csr_debug_checks() -> bool:
     return bool(lib().csr_debug_checks())
+
+
+def csr_debug_read(name: str) -> float:
+    """A quantity only the checked build records (CSRError otherwise); reading resets it."""
+    v = ctypes.c_double(0.0)
+    _check(lib().csr_debug_read(name.encode(), ctypes.byref(v)))
+    return v.value
 
 
 def _check(rc: int) -> None:

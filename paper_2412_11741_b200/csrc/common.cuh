@@ -18,6 +18,8 @@ constexpr uint32_t kStatusTimeout = 1u;
 // Raised only by a library built with CSR_DEBUG_CHECKS (python -m paper_2412_11741_b200.build
 // --debug): an index about to be used for a gather was out of range and has been clamped.
 constexpr uint32_t kStatusBounds = 2u;
+// A kernel found its dynamic shared memory not 1024-byte aligned and did nothing.
+constexpr uint32_t kStatusLayout = 4u;
 
 // Process-wide switches set through csr_set_option (plain loads on the call path).
 struct Options {
@@ -25,6 +27,8 @@ struct Options {
     int fast_split;                     // 0 = chosen by the library; 1 = one CTA per pair of row tiles over the whole
                                         // dictionary; 2 = few rows split the dictionary without clusters
     int exact_split;                    // 0 = chosen by the library; 1 = the row-tile encoder also with few rows
+    int exact_engine;                   // 0 = chosen by the library; 1 = plain-ALU encoders only; 2 = the tensor-core
+                                        // encoder also with few rows
     unsigned long long wait_limit_ns;   // bound of every device-side wait
 };
 Options options();
@@ -52,6 +56,14 @@ int launch_encode_exact(const EncodeArgs& a);
 bool encode_exact_split_applies(int64_t M, int N);
 size_t encode_exact_split_scratch_bytes(int64_t M, int d, int N);
 int launch_encode_exact_split(const EncodeArgs& a, void* scratch);
+
+// The same picks with the sweep on the tensor cores (three bf16 products per correlation bound
+// it to a band; rows inside the band are re-scored in fp64).  `scratch`:
+// encode_exact_tc_scratch_bytes() bytes, 1024-byte aligned; `status` receives kStatusTimeout;
+// `diag` is a device word that a build with CSR_DEBUG_CHECKS raises to the largest error of a
+// tensor-core correlation seen, relative to ||R|| (float bits).
+size_t encode_exact_tc_scratch_bytes(int64_t M, int d, int N);
+int launch_encode_exact_tc(const EncodeArgs& a, void* scratch, uint32_t* status, uint32_t* diag);
 
 // tcgen05 bf16 matching pursuit.  `workspace` holds the bf16 copy of D (N*d*2 bytes,
 // 1024-byte aligned); `status` is a device word that receives kStatusTimeout.

@@ -33,7 +33,7 @@ int fail(int code, const char* fmt, ...) {
 }
 
 namespace {
-std::atomic<int> g_opt_fast_group{0}, g_opt_fast_split{0}, g_opt_exact_split{0};
+std::atomic<int> g_opt_fast_group{0}, g_opt_fast_split{0}, g_opt_exact_split{0}, g_opt_exact_engine{0};
 std::atomic<unsigned long long> g_opt_wait_limit_ns{2000000000ull};      // 2 s per wait
 }  // namespace
 
@@ -42,6 +42,7 @@ Options options() {
     o.fast_group = g_opt_fast_group.load(std::memory_order_relaxed);
     o.fast_split = g_opt_fast_split.load(std::memory_order_relaxed);
     o.exact_split = g_opt_exact_split.load(std::memory_order_relaxed);
+    o.exact_engine = g_opt_exact_engine.load(std::memory_order_relaxed);
     o.wait_limit_ns = g_opt_wait_limit_ns.load(std::memory_order_relaxed);
     return o;
 }
@@ -62,6 +63,7 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kStatusBytes = 256;
+constexpr int kDiagWord = 2;              // word of the status block a checked build raises (see csr_debug_read)
 constexpr uint32_t kDictMagic = 0x43535244u;   // "CSRD"
 
 // Library-owned, grow-only device buffers of one device.
@@ -328,9 +330,23 @@ int encode_device(const csr_encode_params_t* p, bool shared_scratch = true, cons
     a.stream = static_cast<cudaStream_t>(p->stream);
     const Options opt = options();
     if (p->mode == CSR_MODE_FP32_EXACT) {
-        // few rows: split the dictionary across the SMs (library-owned scratch; a caller
-        // workspace is sized for the fast mode only, so with one the row-tile encoder runs)
-        if (!p->workspace && encode_exact_split_applies(p->M, p->N) && opt.exact_split == 0) {
+        // Both the few-rows encoder and the tensor-core encoder need scratch, which comes from
+        // the library-owned buffer only (a caller workspace is sized for the fast mode, and two
+        // encodes in flight must not share it): otherwise the row-tile encoder runs.
+        const bool own = shared_scratch && !p->workspace;
+        const bool few = encode_exact_split_applies(p->M, p->N) && opt.exact_split == 0;
+        if (own && opt.exact_engine != 1 && (!few || opt.exact_engine == 2)) {
+            void* base = nullptr;
+            if (int rc = ensure_work(encode_exact_tc_scratch_bytes(p->M, p->d, p->N), &base, a.stream)) return rc;
+            uint32_t* words = static_cast<uint32_t*>(base);
+            uint32_t* status = p->dev_status ? p->dev_status : words;
+            if (p->dev_status) {
+                cudaError_t e = cudaMemsetAsync(status, 0, sizeof(uint32_t), a.stream);
+                if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+            }
+            return launch_encode_exact_tc(a, align_up(static_cast<char*>(base) + kStatusBytes, 1024), status, words + kDiagWord);
+        }
+        if (own && few) {
             void* base = nullptr;
             if (int rc = ensure_work(encode_exact_split_scratch_bytes(p->M, p->d, p->N), &base, a.stream)) return rc;
             return launch_encode_exact_split(a, align_up(static_cast<char*>(base) + kStatusBytes, 1024));
@@ -673,6 +689,10 @@ int csr_dict_train_step(const csr_train_params_t* p) {
         const size_t sp = encode_exact_split_scratch_bytes(p->M, p->d, p->N);
         if (sp > enc) enc = sp;
     }
+    if (p->M > 0 && p->mode == CSR_MODE_FP32_EXACT) {
+        const size_t sp = encode_exact_tc_scratch_bytes(p->M, p->d, p->N);
+        if (sp > enc) enc = sp;
+    }
     enc = (enc + 1023) / 1024 * 1024;
     const size_t idx_b = ((size_t)p->M * p->s * 2 + 255) / 256 * 256;
     const size_t coef_b = ((size_t)p->M * p->s * 4 + 255) / 256 * 256;
@@ -857,6 +877,7 @@ int csr_device_status(void* stream) {
         seen |= st;
     }
     if (seen & kStatusTimeout) return fail(CSR_ERR_TIMEOUT, "a device-side wait expired (status word 0x%x)", seen);
+    if (seen & kStatusLayout) return fail(CSR_ERR_CUDA, "a kernel found its shared memory misaligned and did not run");
     if (seen & kStatusBounds)
         return fail(CSR_ERR_BOUNDS, "an index used for a gather was out of range and was clamped (status word 0x%x)", seen);
     if (seen != 0) return fail(CSR_ERR_CUDA, "unknown device status 0x%x", seen);
@@ -906,6 +927,9 @@ int csr_set_option(const char* name, int64_t value) {
     } else if (!strcmp(name, "exact_split")) {
         if (value < 0 || value > 1) return fail(CSR_ERR_INVALID_ARG, "exact_split must be 0 or 1");
         g_opt_exact_split.store((int)value);
+    } else if (!strcmp(name, "exact_engine")) {
+        if (value < 0 || value > 2) return fail(CSR_ERR_INVALID_ARG, "exact_engine must be 0, 1 or 2");
+        g_opt_exact_engine.store((int)value);
     } else if (!strcmp(name, "wait_limit_ns")) {
         if (value < 0 || value > 60000000000ll) return fail(CSR_ERR_INVALID_ARG, "wait_limit_ns must lie in [0, 6e10]");
         g_opt_wait_limit_ns.store((unsigned long long)value);
@@ -913,6 +937,33 @@ int csr_set_option(const char* name, int64_t value) {
         return fail(CSR_ERR_INVALID_ARG, "unknown option '%s'", name);
     }
     return CSR_OK;
+}
+
+int csr_debug_read(const char* name, double* value) {
+    if (!name || !value) return fail(CSR_ERR_INVALID_ARG, "name or value is NULL");
+    if (strcmp(name, "exact_tensor_error") != 0) return fail(CSR_ERR_INVALID_ARG, "unknown quantity '%s'", name);
+#ifndef CSR_DEBUG_CHECKS
+    return fail(CSR_ERR_UNSUPPORTED, "only a library built with CSR_DEBUG_CHECKS records '%s'", name);
+#else
+    int dev;
+    if (int rc = current_device(&dev)) return rc;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "device sync: %s", cudaGetErrorString(e));
+    void* work = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        work = g_dev[dev].work;
+    }
+    float v = 0.f;
+    if (work) {
+        uint32_t* word = static_cast<uint32_t*>(work) + kDiagWord;
+        e = cudaMemcpy(&v, word, sizeof(float), cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess) e = cudaMemset(word, 0, sizeof(uint32_t));
+        if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "diagnostic read: %s", cudaGetErrorString(e));
+    }
+    *value = static_cast<double>(v);
+    return CSR_OK;
+#endif
 }
 
 int csr_dict_check_norms(const void* D, int N, int d, float tol, void* stream, float* max_dev) {

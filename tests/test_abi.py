@@ -34,7 +34,7 @@ def test_exports_match_header(lib):
 
 def test_version_and_struct_sizes(lib):
     from paper_2412_11741_b200 import binding
-    assert binding.csr_version() == 110
+    assert binding.csr_version() == 120
     assert ctypes.sizeof(binding.csr_encode_params_t) == 128
     assert ctypes.sizeof(binding.csr_reconstruct_params_t) == 104
 

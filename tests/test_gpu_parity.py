@@ -34,8 +34,17 @@ def csr():
 def opts(csr):
     """Sets library options (csr_set_option) for one test and restores the defaults afterwards."""
     yield csr.csr_set_option
-    for name, value in (("fast_group", 0), ("fast_split", 0), ("exact_split", 0), ("wait_limit_ns", 2_000_000_000)):
+    for name, value in (("fast_group", 0), ("fast_split", 0), ("exact_split", 0), ("exact_engine", 0), ("wait_limit_ns", 2_000_000_000)):
         csr.csr_set_option(name, value)
+
+
+@pytest.fixture(params=["library", "alu", "tensor"])
+def engine(request, csr):
+    """Runs an exact-mode test with the library's choice of encoder, with the plain-ALU encoders
+    only, and with the tensor-core encoder whatever the number of rows."""
+    csr.csr_set_option("exact_engine", {"library": 0, "alu": 1, "tensor": 2}[request.param])
+    yield request.param
+    csr.csr_set_option("exact_engine", 0)
 
 
 def _dev_x(w, X=None):
@@ -55,7 +64,7 @@ def _encode(csr, w, X, mode, coef_dtype=torch.float32):
 # exact mode
 # ---------------------------------------------------------------------------------------
 
-def test_exact_tiny_config_all_rows(csr):
+def test_exact_tiny_config_all_rows(csr, engine):
     w = wl.tiny()
     idx, coef = _encode(csr, w, w.X, csr.CSR_MODE_FP32_EXACT)
     rep = parity.compare_exact(w.D, w.X, w.s, idx, coef)
@@ -77,7 +86,7 @@ def test_exact_tiny_config_all_rows(csr):
     (lambda: wl.dict_sweep(2048, M=4096), 2048),
     (lambda: wl.dict_sweep(4096, d=64, M=4096), 2048),
 ])
-def test_exact_configs_subsample(csr, make, rows):
+def test_exact_configs_subsample(csr, make, rows, engine):
     w = make()
     sel = wl.stratified_rows(w.M, rows, seed=7)
     X = w.X[sel]
@@ -87,7 +96,7 @@ def test_exact_configs_subsample(csr, make, rows):
 
 
 @pytest.mark.parametrize("M", [0, 1, 2, 63, 64, 65, 127, 129, 200])
-def test_exact_ragged_rows(csr, M):
+def test_exact_ragged_rows(csr, M, engine):
     rng = np.random.default_rng(M)
     D = wl.normalise_rows(rng.standard_normal((272, 128)).astype(np.float32))   # N not a tile multiple
     X = rng.standard_normal((M, 128)).astype(np.float32)
@@ -104,7 +113,7 @@ def test_exact_ragged_rows(csr, M):
 
 
 @pytest.mark.parametrize("N,s", [(1, 3), (16, 1), (130, 7), (1024, 64)])
-def test_exact_small_dictionaries(csr, N, s):
+def test_exact_small_dictionaries(csr, N, s, engine):
     rng = np.random.default_rng(N * 100 + s)
     D = wl.normalise_rows(rng.standard_normal((N, 64)).astype(np.float32))
     X = rng.standard_normal((150, 64)).astype(np.float32)
@@ -113,7 +122,7 @@ def test_exact_small_dictionaries(csr, N, s):
     assert rep.ok, rep.detail
 
 
-def test_exact_degenerate_inputs(csr):
+def test_exact_degenerate_inputs(csr, engine):
     """Zero vectors, exact ties, an input that is itself an atom, a duplicated atom."""
     rng = np.random.default_rng(5)
     D = wl.normalise_rows(rng.standard_normal((256, 128)).astype(np.float32))
@@ -133,7 +142,7 @@ def test_exact_degenerate_inputs(csr):
     assert rep.ok, rep.detail
 
 
-def test_exact_identity_dictionary_recovers_exactly(csr):
+def test_exact_identity_dictionary_recovers_exactly(csr, engine):
     rng = np.random.default_rng(8)
     D = np.eye(64, dtype=np.float32)
     X = rng.standard_normal((130, 64)).astype(np.float32)
@@ -354,7 +363,7 @@ def test_pack_coefficients_is_round_to_nearest_even(csr, n):
     assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
 
 
-def test_fp16_inputs_and_outputs(csr):
+def test_fp16_inputs_and_outputs(csr, engine):
     """fp16 is the paper's model precision: X may be fp16 (read exactly by the exact mode,
     rounded to bf16 by the fast mode) and X_hat may be written as fp16."""
     rng = np.random.default_rng(16)
@@ -505,7 +514,7 @@ def test_fast_every_group_size(csr, G, d, opts):
         assert rep.ok, (G, d, N, rep.detail)
 
 
-def test_largest_dictionary_and_most_iterations(csr):
+def test_largest_dictionary_and_most_iterations(csr, engine):
     """The limits of the interface: N = 65536 (indices fill the uint16 range) and s = 64, in
     both modes, against the oracle."""
     rng = np.random.default_rng(65536)
@@ -631,6 +640,14 @@ def test_random_shapes_both_modes(csr, seed):
     idx, coef = csr.csr_encode_ex(Dd, Xd, s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
     rep = parity.compare_exact(D, X, s, _np_idx(idx), coef.cpu().numpy(), res)
     assert rep.ok, (d, N, M, s, kind, rep.detail)
+    csr.csr_set_option("exact_engine", 2)                 # the tensor-core encoder, whatever the number of rows
+    try:
+        idx_t, coef_t = csr.csr_encode_ex(Dd, Xd, s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
+    finally:
+        csr.csr_set_option("exact_engine", 0)
+    assert csr.csr_device_status() == csr.CSR_OK
+    rep = parity.compare_exact(D, X, s, _np_idx(idx_t), coef_t.cpu().numpy(), res)
+    assert rep.ok, ("tensor", d, N, M, s, kind, rep.detail)
     xh = csr.csr_reconstruct_ex(Dd, idx, coef, out_dtype=torch.float32).cpu().numpy()
     ref = orc.reconstruct(D, _np_idx(idx).astype(np.int32), coef.cpu().numpy().astype(np.float64))
     scale = np.abs(coef.cpu().numpy()).sum(1, keepdims=True) + 1e-30
@@ -666,9 +683,14 @@ def test_nan_and_inf_rows_do_no_harm(csr, M, N):
     good = np.ones(M, bool)
     good[[5, 9, 17]] = False
     Dd = torch.from_numpy(D).to(DEV)
-    for mode, dt in ((csr.CSR_MODE_BF16_FAST, torch.bfloat16), (csr.CSR_MODE_FP32_EXACT, torch.float32)):
-        i0, c0 = csr.csr_encode_ex(Dd, torch.from_numpy(X).to(DEV).to(dt), 6, mode=mode, coef_dtype=torch.float32)
-        i1, c1 = csr.csr_encode_ex(Dd, torch.from_numpy(bad).to(DEV).to(dt), 6, mode=mode, coef_dtype=torch.float32)
+    for mode, dt, eng in ((csr.CSR_MODE_BF16_FAST, torch.bfloat16, 0), (csr.CSR_MODE_FP32_EXACT, torch.float32, 1),
+                          (csr.CSR_MODE_FP32_EXACT, torch.float32, 2)):
+        csr.csr_set_option("exact_engine", eng)
+        try:
+            i0, c0 = csr.csr_encode_ex(Dd, torch.from_numpy(X).to(DEV).to(dt), 6, mode=mode, coef_dtype=torch.float32)
+            i1, c1 = csr.csr_encode_ex(Dd, torch.from_numpy(bad).to(DEV).to(dt), 6, mode=mode, coef_dtype=torch.float32)
+        finally:
+            csr.csr_set_option("exact_engine", 0)
         assert csr.csr_device_status() == csr.CSR_OK
         g = torch.from_numpy(good).to(DEV)
         assert torch.equal(i0.view(torch.int16)[g], i1.view(torch.int16)[g]) and torch.equal(c0[g], c1[g])
