@@ -19,13 +19,14 @@
 //   - each row tile has one 256-column fp32 accumulator in TMEM.  All eight epilogue warps drain
 //     every accumulator: warp w reads the 32 TMEM lanes of w % 4 and the 128 columns of w / 4, i.e.
 //     all of them sit in registers after one round of loads and the accumulator goes straight back
-//     to the tensor core.  Each thread keeps the three largest keys of its half row, a key being
+//     to the tensor core.  Each thread keeps the four largest keys of its half row, a key being
 //     |value| with its seven lowest mantissa bits replaced by the column's tag, and where the
-//     largest two came from;
+//     largest three came from.  Groups of four values are first reduced to their largest
+//     magnitude and only groups within the band of the running maximum are inserted;
 //   - at the end of a sweep the halves are merged through shared memory, and each warp settles
 //     its 32 rows, eight lanes per row: rows whose best and second-best keys are further apart
 //     than the band take the best; rows where only the second is inside the band compare the two
-//     in fp64; rows where the third is inside too (about one in 10^4) are re-scored by the warp
+//     or three in fp64; rows where the fourth is inside too (about one in 10^6) are re-scored by the warp
 //     over the whole dictionary (fp32 filter, then fp64).  Coefficient (Eq. 2, signed) and
 //     residual update (Eq. 4) are fp64, as in the plain-ALU encoder.
 // Warp roles: 0-7 epilogue, 8 TMA producer, 9 TMEM owner and MMA issuer.  All waits are bounded.
@@ -234,12 +235,18 @@ __device__ __forceinline__ void load_atom(const float* __restrict__ src, float (
         a[4 * q + 3] = v.w;
     }
 }
+// (four running sums: a single chain of fp64 FMAs would wait out the pipe's latency CH times)
 template <int CH>
 __device__ __forceinline__ double slice_dot(const double (&R)[CH], const float (&a)[CH]) {
-    double c = 0.0;
+    double c0 = 0.0, c1 = 0.0, c2 = 0.0, c3 = 0.0;
 #pragma unroll
-    for (int k = 0; k < CH; ++k) c = fma(R[k], static_cast<double>(a[k]), c);
-    return c;
+    for (int k = 0; k < CH; k += 4) {
+        c0 = fma(R[k], static_cast<double>(a[k]), c0);
+        c1 = fma(R[k + 1], static_cast<double>(a[k + 1]), c1);
+        c2 = fma(R[k + 2], static_cast<double>(a[k + 2]), c2);
+        c3 = fma(R[k + 3], static_cast<double>(a[k + 3]), c3);
+    }
+    return (c0 + c1) + (c2 + c3);
 }
 
 // Writes this lane's CH residual values: fp64 to the scratch row, bf16 high and low parts into
@@ -247,13 +254,17 @@ __device__ __forceinline__ double slice_dot(const double (&R)[CH], const float (
 template <int CH>
 __device__ __forceinline__ double store_residual(const double (&R)[CH], double* __restrict__ dst, uint8_t* Ahi, uint8_t* Alo,
                                                  int r, int l8) {
-    double nn = 0.0;
+    double n0 = 0.0, n1 = 0.0, n2 = 0.0, n3 = 0.0;
 #pragma unroll
-    for (int q = 0; q < CH / 2; ++q) {
-        reinterpret_cast<double2*>(dst)[q] = make_double2(R[2 * q], R[2 * q + 1]);
-        nn = fma(R[2 * q], R[2 * q], nn);
-        nn = fma(R[2 * q + 1], R[2 * q + 1], nn);
+    for (int q = 0; q < CH / 4; ++q) {
+        reinterpret_cast<double2*>(dst)[2 * q] = make_double2(R[4 * q], R[4 * q + 1]);
+        reinterpret_cast<double2*>(dst)[2 * q + 1] = make_double2(R[4 * q + 2], R[4 * q + 3]);
+        n0 = fma(R[4 * q], R[4 * q], n0);
+        n1 = fma(R[4 * q + 1], R[4 * q + 1], n1);
+        n2 = fma(R[4 * q + 2], R[4 * q + 2], n2);
+        n3 = fma(R[4 * q + 3], R[4 * q + 3], n3);
     }
+    const double nn = (n0 + n1) + (n2 + n3);
 #pragma unroll
     for (int j = 0; j < CH / 8; ++j) {
         uint32_t hw[4], lw[4];
@@ -305,7 +316,7 @@ __device__ __forceinline__ void load_x8(const void* X, int x_dtype, int64_t off,
 // correlations decide, the lowest atom among equal values.  More than 32 candidates (copies of
 // one atom): every atom is scored in fp64.
 template <int D_>
-__device__ int rescore_row(const float* __restrict__ D, int N, const double* __restrict__ Rrow, float thresh, int lane) {
+__device__ __noinline__ int rescore_row(const float* __restrict__ D, int N, const double* __restrict__ Rrow, float thresh, int lane) {
     constexpr int PER = D_ / 32;
     double R[PER];
     float rf[PER];
@@ -419,7 +430,7 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                     for (int t = 0; t < T && ok; ++t) {
                         for (int hp = 0; hp < 2 * KH; ++hp, ++p) {
                             const int stage = p % STAGES;
-                            if (!wait_bounded(&sm.empty_b[stage], ((p / STAGES) & 1) ^ 1, wc)) {
+                            if (!wait_bounded_suspended(&sm.empty_b[stage], ((p / STAGES) & 1) ^ 1, wc, 2000)) {
                                 ok = false;
                                 break;
                             }
@@ -447,7 +458,7 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
             bool ok = true;
             for (int64_t pair = blockIdx.x; pair < n_pairs && ok; pair += gridDim.x) {
                 for (int g = 0; g < s && ok; ++g, ++steps) {
-                    if (!wait_bounded(&sm.res_ready, steps & 1, wc)) {
+                    if (!wait_bounded_suspended(&sm.res_ready, steps & 1, wc, 4000)) {
                         ok = false;
                         break;
                     }
@@ -456,14 +467,14 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                             const int stage = p % STAGES;
                             const int h = hp >> 1;
                             const bool low = hp & 1;      // this stage holds low parts of the atoms
-                            if (!wait_bounded(&sm.full_b[stage], (p / STAGES) & 1, wc)) {
+                            if (!wait_bounded_suspended(&sm.full_b[stage], (p / STAGES) & 1, wc, 1000)) {
                                 ok = false;
                                 break;
                             }
                             tc_fence_after();
                             const uint64_t b0 = make_smem_desc(smem_u32(&sm.B[stage][0]));
                             for (int tile = 0; tile < 2; ++tile) {
-                                if (hp == 0 && !wait_bounded(&sm.acc_empty[tile], (accn & 1) ^ 1, wc)) {
+                                if (hp == 0 && !wait_bounded_suspended(&sm.acc_empty[tile], (accn & 1) ^ 1, wc, 1000)) {
                                     ok = false;
                                     break;
                                 }
@@ -550,7 +561,7 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                 for (int t = 0; t < T && ok; ++t, ++accn) {
 #pragma unroll 1
                     for (int a = 0; a < 2; ++a) {           // (rolled: one copy of the drain's code)
-                        bool got = wait_bounded(&sm.acc_full[a], accn & 1, wc);
+                        bool got = wait_bounded_suspended(&sm.acc_full[a], accn & 1, wc, 2000);
                         got = __all_sync(FULL, got);
                         if (!got) {
                             ok = false;
@@ -602,101 +613,109 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                 }
                 const float my_thresh = v0 - 1.5f * band;
 
-                // ---- settle the 32 rows of this warp: eight lanes per row, two rows per lane group
-                // (passes pp and pp + 4) worked on side by side ----
+                // ---- settle the 32 rows of this warp, eight lanes per row, four rows per pass; the
+                // next pass's residual rows and atoms are requested before this pass is worked on
+                // (one copy of the code: it has to stay in the instruction cache next to the sweep) ----
+                auto fetch = [&](int p, int& n, int& flags, double (&R)[CH], float (&a)[CH]) {
+                    const int src = 4 * p + grp;
+                    n = __shfl_sync(FULL, my_n1, src);
+                    flags = __shfl_sync(FULL, my_flags, src);
+                    const double* Rrow = Rd_cta + static_cast<int64_t>(own_tile * TILE_M + q * 32 + src) * D_ + l8 * CH;
+#pragma unroll
+                    for (int k = 0; k < CH / 2; ++k) {
+                        const double2 v = reinterpret_cast<const double2*>(Rrow)[k];
+                        R[2 * k] = v.x;
+                        R[2 * k + 1] = v.y;
+                    }
+                    load_atom<CH>(D + static_cast<int64_t>(n) * D_ + l8 * CH, a);
+                };
+                int n, flags;
+                double R[CH];
+                float a[CH];
+                fetch(0, n, flags, R, a);
 #pragma unroll 1
-                for (int pp = 0; pp < 4; ++pp) {
-                    int n[2], flags[2];
-                    double R[2][CH];
-                    float a[2][CH];
-                    double* Rrow[2];
+                for (int p = 0; p < 8; ++p) {
+                    int n_nx = 0, flags_nx = 0;
+                    double R_nx[CH];
+                    float a_nx[CH];
+                    if (p + 1 < 8) {
+                        fetch(p + 1, n_nx, flags_nx, R_nx, a_nx);
+                    } else {
 #pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int src = 4 * (pp + 4 * u) + grp;
-                        n[u] = __shfl_sync(FULL, my_n1, src);
-                        flags[u] = __shfl_sync(FULL, my_flags, src);
-                        Rrow[u] = Rd_cta + static_cast<int64_t>(own_tile * TILE_M + q * 32 + src) * D_ + l8 * CH;
-#pragma unroll
-                        for (int k = 0; k < CH / 2; ++k) {
-                            const double2 v = reinterpret_cast<const double2*>(Rrow[u])[k];
-                            R[u][2 * k] = v.x;
-                            R[u][2 * k + 1] = v.y;
+                        for (int k = 0; k < CH; ++k) {
+                            R_nx[k] = 0.0;
+                            a_nx[k] = 0.f;
                         }
-                        load_atom<CH>(D + static_cast<int64_t>(n[u]) * D_ + l8 * CH, a[u]);
                     }
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        if (!__any_sync(FULL, flags[u] != 0)) continue;
+                    const int src = 4 * p + grp;
+                    const int r = q * 32 + src;
+                    const int64_t m = pair * ROWS + own_tile * TILE_M + r;
+                    double* Rrow = Rd_cta + static_cast<int64_t>(own_tile * TILE_M + r) * D_ + l8 * CH;
+                    if (__any_sync(FULL, flags != 0)) {
                         // some row of this pass is not decided by its largest key alone
-                        const int src = 4 * (pp + 4 * u) + grp;
-                        const int n_first = n[u];
-                        if (__any_sync(FULL, flags[u] & 4)) {
+                        const int n_first = n;
+                        if (__any_sync(FULL, flags & 4)) {
                             for (int j = 0; j < 4; ++j) {   // four keys inside the band: the whole dictionary, by the warp
-                                const int fj = __shfl_sync(FULL, flags[u], 8 * j);
-                                const float th = __shfl_sync(FULL, my_thresh, 4 * (pp + 4 * u) + j);
+                                const int fj = __shfl_sync(FULL, flags, 8 * j);
+                                const float th = __shfl_sync(FULL, my_thresh, 4 * p + j);
                                 if (fj & 4) {
-                                    const int nr = rescore_row<D_>(D, N, Rd_cta + static_cast<int64_t>(own_tile * TILE_M + q * 32 + 4 * (pp + 4 * u) + j) * D_, th, lane);
-                                    if (grp == j) n[u] = nr;
+                                    const int nr = rescore_row<D_>(D, N, Rd_cta + static_cast<int64_t>(own_tile * TILE_M + q * 32 + 4 * p + j) * D_, th, lane);
+                                    if (grp == j) n = nr;
                                 }
                             }
                         }
-                        const bool cmp = (flags[u] & 4) == 0 && flags[u] != 0;   // this lane's row compares two or three
+                        const bool cmp = (flags & 4) == 0 && flags != 0;   // this lane's row compares two or three
                         if (__any_sync(FULL, cmp)) {
-                            double cbest = fabs(group8_sum(slice_dot<CH>(R[u], a[u])));
-                            int nbest = n[u];
-                            float ax[CH];
-                            const int nc2 = __shfl_sync(FULL, my_n2, src);
-                            load_atom<CH>(D + static_cast<int64_t>(nc2) * D_ + l8 * CH, ax);
-                            const double c2 = fabs(group8_sum(slice_dot<CH>(R[u], ax)));
-                            if (c2 > cbest || (c2 == cbest && nc2 < nbest)) {
-                                cbest = c2;
-                                nbest = nc2;
-                            }
-                            if (__any_sync(FULL, cmp && (flags[u] & 2))) {
-                                const int nc3 = __shfl_sync(FULL, my_n3, src);
-                                load_atom<CH>(D + static_cast<int64_t>(nc3) * D_ + l8 * CH, ax);
-                                const double c3 = fabs(group8_sum(slice_dot<CH>(R[u], ax)));
-                                if ((flags[u] & 2) && (c3 > cbest || (c3 == cbest && nc3 < nbest))) {
-                                    cbest = c3;
-                                    nbest = nc3;
+                            double cbest = fabs(group8_sum(slice_dot<CH>(R, a)));
+                            int nbest = n;
+#pragma unroll 1
+                            for (int cand = 0; cand < 2; ++cand) {
+                                if (cand == 1 && !__any_sync(FULL, cmp && (flags & 2))) break;
+                                const int nc = __shfl_sync(FULL, cand ? my_n3 : my_n2, src);
+                                float ax[CH];
+                                load_atom<CH>(D + static_cast<int64_t>(nc) * D_ + l8 * CH, ax);
+                                const double cc = fabs(group8_sum(slice_dot<CH>(R, ax)));
+                                if ((cand == 0 || (flags & 2)) && (cc > cbest || (cc == cbest && nc < nbest))) {
+                                    cbest = cc;
+                                    nbest = nc;
                                 }
                             }
-                            if (cmp) n[u] = nbest;
+                            if (cmp) n = nbest;
                         }
-                        if (__any_sync(FULL, n[u] != n_first)) load_atom<CH>(D + static_cast<int64_t>(n[u]) * D_ + l8 * CH, a[u]);
+                        if (__any_sync(FULL, n != n_first)) load_atom<CH>(D + static_cast<int64_t>(n) * D_ + l8 * CH, a);
                     }
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int p = pp + 4 * u;
-                        const int src = 4 * p + grp;
-                        const int r = q * 32 + src;
-                        const int64_t m = pair * ROWS + own_tile * TILE_M + r;
-                        const double c = group8_sum(slice_dot<CH>(R[u], a[u]));
+                    const double c = group8_sum(slice_dot<CH>(R, a));
 #ifdef CSR_DEBUG_CHECKS
-                        {   // largest |tensor-core value - fp64 value| / ||R|| seen, as float bits
-                            const float vbo = __shfl_sync(FULL, v0, src), bo = __shfl_sync(FULL, band, src);
-                            if (l8 == 0 && m < M && flags[u] == 0 && bo > 0.f) {
-                                const float rel = fabsf(vbo - static_cast<float>(fabs(c))) / (bo / kBandRel);
-                                atomicMax(diag, __float_as_uint(rel));
-                            }
+                    {   // largest |tensor-core value - fp64 value| / ||R|| seen, as float bits
+                        const float vbo = __shfl_sync(FULL, v0, src), bo = __shfl_sync(FULL, band, src);
+                        if (l8 == 0 && m < M && flags == 0 && bo > 0.f) {
+                            const float rel = fabsf(vbo - static_cast<float>(fabs(c))) / (bo / kBandRel);
+                            atomicMax(diag, __float_as_uint(rel));
                         }
+                    }
 #endif
-                        if (l8 == 0 && m < M) {
-                            out_idx[m * ldc + g] = static_cast<uint16_t>(n[u]);
-                            const float cf = static_cast<float>(c);
-                            if (coef_dtype == CSR_DTYPE_F16)
-                                reinterpret_cast<__half*>(out_coef)[m * ldc + g] = __float2half_rn(cf);
-                            else
-                                reinterpret_cast<float*>(out_coef)[m * ldc + g] = cf;
-                        }
-                        if (g + 1 < s) {
+                    if (l8 == 0 && m < M) {
+                        out_idx[m * ldc + g] = static_cast<uint16_t>(n);
+                        const float cf = static_cast<float>(c);
+                        if (coef_dtype == CSR_DTYPE_F16)
+                            reinterpret_cast<__half*>(out_coef)[m * ldc + g] = __float2half_rn(cf);
+                        else
+                            reinterpret_cast<float*>(out_coef)[m * ldc + g] = cf;
+                    }
+                    if (g + 1 < s) {
 #pragma unroll
-                            for (int k = 0; k < CH; ++k) R[u][k] = fma(-c, static_cast<double>(a[u][k]), R[u][k]);
-                            double nn = store_residual<CH>(R[u], Rrow[u], Ahi, Alo, r, l8);
-                            nn = group8_sum(nn);
-                            const float nn_o = static_cast<float>(__shfl_sync(FULL, nn, (lane & 3) * 8));
-                            if ((lane >> 2) == p) band = kBandRel * sqrtf(nn_o) * 1.001f;
-                        }
+                        for (int k = 0; k < CH; ++k) R[k] = fma(-c, static_cast<double>(a[k]), R[k]);
+                        double nn = store_residual<CH>(R, Rrow, Ahi, Alo, r, l8);
+                        nn = group8_sum(nn);
+                        const float nn_o = static_cast<float>(__shfl_sync(FULL, nn, (lane & 3) * 8));
+                        if ((lane >> 2) == p) band = kBandRel * sqrtf(nn_o) * 1.001f;
+                    }
+                    n = n_nx;
+                    flags = flags_nx;
+#pragma unroll
+                    for (int k = 0; k < CH; ++k) {
+                        R[k] = R_nx[k];
+                        a[k] = a_nx[k];
                     }
                 }
                 if (g + 1 < s) {

@@ -40,6 +40,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// The same with a hint of how long the hardware may keep the thread suspended (nanoseconds)
+// before the instruction returns false: a thread that polls with a long hint leaves the issue
+// slots of its scheduler to the other warps.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t suspend_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(suspend_ns)
+        : "memory");
+    return ok != 0;
+}
 // One look at the barrier without suspending the thread.
 __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
@@ -195,6 +211,27 @@ __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, con
         for (uint32_t it = 1; it < (1u << 28); ++it) {
             if (mbar_try_wait(bar, parity)) return true;
             if ((it & 63u) == 0) {
+                if (*w.abort) return false;
+                if (globaltimer_ns() - t0 > w.limit_ns) break;
+            }
+        }
+    } else if (mbar_test_wait(bar, parity)) {
+        return true;
+    }
+    *w.abort = 1;
+    atomicOr(w.status, kStatusTimeout);
+    return false;
+}
+
+// The same wait for hand-offs that take long (a whole pick, a whole sweep): every poll lets the
+// hardware suspend the thread for up to `suspend_ns`.
+__device__ __forceinline__ bool wait_bounded_suspended(uint64_t* bar, uint32_t parity, const WaitCtx& w, uint32_t suspend_ns) {
+    if (w.limit_ns != 0) {
+        if (mbar_try_wait(bar, parity)) return true;
+        const unsigned long long t0 = globaltimer_ns();
+        for (uint32_t it = 1; it < (1u << 28); ++it) {
+            if (mbar_try_wait_hint(bar, parity, suspend_ns)) return true;
+            if ((it & 7u) == 0) {
                 if (*w.abort) return false;
                 if (globaltimer_ns() - t0 > w.limit_ns) break;
             }
