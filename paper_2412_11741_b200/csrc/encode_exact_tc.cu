@@ -52,6 +52,9 @@ constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t kInstrDesc = instr_desc_bf16(TILE_M, TILE_N);
 constexpr uint32_t kKeyMask = 0x7FFFFF80u;                // |value| without its seven lowest mantissa bits
 constexpr uint32_t FULL = 0xffffffffu;
+#ifndef CSR_TC_GROUP128
+#define CSR_TC_GROUP128 2                                 // measured: 12-17 % faster than 1 at d = 128
+#endif
 // Half-width of the undecided zone relative to ||R||: twice the error of a tensor-core
 // correlation (the split's 1.2e-5 plus the fp32 accumulation of 3 d products in groups of 16)
 // plus the 2^-16 relative truncation of the keys.
@@ -223,16 +226,17 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
+// The eight lanes that share a row own its channels in pairs: lane l8 has channels 2 (8 k + l8)
+// and the next one, k = 0 .. CH / 2 - 1, so that one load or store instruction of the eight lanes
+// covers one contiguous run (whole 32-byte sectors of the fp64 row).
 // CH channels of one atom (fp32 master copy), as this lane's slice.
 template <int CH>
-__device__ __forceinline__ void load_atom(const float* __restrict__ src, float (&a)[CH]) {
+__device__ __forceinline__ void load_atom(const float* __restrict__ atom, int l8, float (&a)[CH]) {
 #pragma unroll
-    for (int q = 0; q < CH / 4; ++q) {
-        const float4 v = __ldg(reinterpret_cast<const float4*>(src) + q);
-        a[4 * q + 0] = v.x;
-        a[4 * q + 1] = v.y;
-        a[4 * q + 2] = v.z;
-        a[4 * q + 3] = v.w;
+    for (int k = 0; k < CH / 2; ++k) {
+        const float2 v = __ldg(reinterpret_cast<const float2*>(atom) + 8 * k + l8);
+        a[2 * k] = v.x;
+        a[2 * k + 1] = v.y;
     }
 }
 // (four running sums: a single chain of fp64 FMAs would wait out the pipe's latency CH times)
@@ -249,63 +253,46 @@ __device__ __forceinline__ double slice_dot(const double (&R)[CH], const float (
     return (c0 + c1) + (c2 + c3);
 }
 
-// Writes this lane's CH residual values: fp64 to the scratch row, bf16 high and low parts into
-// the operand tiles.  Returns the lane's share of ||R||^2.
+// Writes this lane's CH residual values: fp64 to the scratch row (`row`: its first element), bf16
+// high and low parts into the operand tiles.  Returns the lane's share of ||R||^2.
 template <int CH>
-__device__ __forceinline__ double store_residual(const double (&R)[CH], double* __restrict__ dst, uint8_t* Ahi, uint8_t* Alo,
+__device__ __forceinline__ double store_residual(const double (&R)[CH], double* __restrict__ row, uint8_t* Ahi, uint8_t* Alo,
                                                  int r, int l8) {
-    double n0 = 0.0, n1 = 0.0, n2 = 0.0, n3 = 0.0;
+    double n0 = 0.0, n1 = 0.0;
 #pragma unroll
-    for (int q = 0; q < CH / 4; ++q) {
-        reinterpret_cast<double2*>(dst)[2 * q] = make_double2(R[4 * q], R[4 * q + 1]);
-        reinterpret_cast<double2*>(dst)[2 * q + 1] = make_double2(R[4 * q + 2], R[4 * q + 3]);
-        n0 = fma(R[4 * q], R[4 * q], n0);
-        n1 = fma(R[4 * q + 1], R[4 * q + 1], n1);
-        n2 = fma(R[4 * q + 2], R[4 * q + 2], n2);
-        n3 = fma(R[4 * q + 3], R[4 * q + 3], n3);
+    for (int k = 0; k < CH / 2; ++k) {
+        reinterpret_cast<double2*>(row)[8 * k + l8] = make_double2(R[2 * k], R[2 * k + 1]);
+        n0 = fma(R[2 * k], R[2 * k], n0);
+        n1 = fma(R[2 * k + 1], R[2 * k + 1], n1);
+        const float f0 = static_cast<float>(R[2 * k]), f1 = static_cast<float>(R[2 * k + 1]);
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
+        const __nv_bfloat16 l0 = __float2bfloat16_rn(f0 - __bfloat162float(h0));
+        const __nv_bfloat16 l1 = __float2bfloat16_rn(f1 - __bfloat162float(h1));
+        // channels 2 (8 k + l8), +1: 16-byte chunk 2 k + l8 / 4 of the row, word l8 % 4 of it
+        const uint32_t off = swz_off(r, 2 * k + (l8 >> 2)) + (l8 & 3) * 4;
+        *reinterpret_cast<uint32_t*>(Ahi + off) =
+            static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+        *reinterpret_cast<uint32_t*>(Alo + off) =
+            static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
     }
-    const double nn = (n0 + n1) + (n2 + n3);
-#pragma unroll
-    for (int j = 0; j < CH / 8; ++j) {
-        uint32_t hw[4], lw[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float f0 = static_cast<float>(R[8 * j + 2 * q]), f1 = static_cast<float>(R[8 * j + 2 * q + 1]);
-            const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
-            const __nv_bfloat16 l0 = __float2bfloat16_rn(f0 - __bfloat162float(h0));
-            const __nv_bfloat16 l1 = __float2bfloat16_rn(f1 - __bfloat162float(h1));
-            hw[q] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
-            lw[q] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
-        }
-        const uint32_t off = swz_off(r, l8 * (CH / 8) + j);
-        *reinterpret_cast<uint4*>(Ahi + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-        *reinterpret_cast<uint4*>(Alo + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-    }
-    return nn;
+    return n0 + n1;
 }
 
-// Eight consecutive elements of X widened to fp64.
-__device__ __forceinline__ void load_x8(const void* X, int x_dtype, int64_t off, double* out) {
+// Elements `off` and `off + 1` of X widened to fp64.
+__device__ __forceinline__ void load_x2(const void* X, int x_dtype, int64_t off, double& x0, double& x1) {
     if (x_dtype == CSR_DTYPE_F32) {
-        const float4 a = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X) + off));
-        const float4 b = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X) + off) + 1);
-        out[0] = a.x, out[1] = a.y, out[2] = a.z, out[3] = a.w, out[4] = b.x, out[5] = b.y, out[6] = b.z, out[7] = b.w;
+        const float2 v = __ldg(reinterpret_cast<const float2*>(reinterpret_cast<const float*>(X) + off));
+        x0 = v.x;
+        x1 = v.y;
     } else {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(X) + off));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            float lo, hi;
-            if (x_dtype == CSR_DTYPE_BF16) {
-                lo = __uint_as_float(w[q] << 16);
-                hi = __uint_as_float(w[q] & 0xFFFF0000u);
-            } else {
-                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[q]));
-                lo = f.x;
-                hi = f.y;
-            }
-            out[2 * q] = lo;
-            out[2 * q + 1] = hi;
+        const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint16_t*>(X) + off));
+        if (x_dtype == CSR_DTYPE_BF16) {
+            x0 = __uint_as_float(w << 16);
+            x1 = __uint_as_float(w & 0xFFFF0000u);
+        } else {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+            x0 = f.x;
+            x1 = f.y;
         }
     }
 }
@@ -393,6 +380,9 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
     constexpr int KH = D_ / STAGE_CH;                       // 64-channel blocks per row
     constexpr int KSTEPS = STAGE_CH / UMMA_K;
     constexpr int STAGES = S::kStages;
+    constexpr int NSTG = 2 * KH;                            // stages per dictionary tile
+    constexpr int GROUP = STAGES >= NSTG + 2 ? NSTG : CSR_TC_GROUP128;
+    static_assert(GROUP < STAGES && NSTG % GROUP == 0, "a group of stages must fit the ring with one stage to spare");
     const WaitCtx wc{&sm.abort, status, wait_limit_ns};
 
     if (threadIdx.x == 0) {
@@ -462,41 +452,48 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                         ok = false;
                         break;
                     }
-                    for (int t = 0; t < T && ok; ++t, ++accn) {
-                        for (int hp = 0; hp < 2 * KH && ok; ++hp, ++p) {
-                            const int stage = p % STAGES;
-                            const int h = hp >> 1;
-                            const bool low = hp & 1;      // this stage holds low parts of the atoms
-                            if (!wait_bounded_suspended(&sm.full_b[stage], (p / STAGES) & 1, wc, 1000)) {
-                                ok = false;
-                                break;
-                            }
-                            tc_fence_after();
-                            const uint64_t b0 = make_smem_desc(smem_u32(&sm.B[stage][0]));
-                            for (int tile = 0; tile < 2; ++tile) {
-                                if (hp == 0 && !wait_bounded_suspended(&sm.acc_empty[tile], (accn & 1) ^ 1, wc, 1000)) {
-                                    ok = false;
-                                    break;
-                                }
-                                if (hp == 0) tc_fence_after();
-                                const uint32_t d_tmem = tmem_base + tile * TILE_N;
-                                const uint64_t ah = make_smem_desc(smem_u32(&sm.A[tile][0][h * (TILE_M * 128)]));
-                                const uint64_t al = make_smem_desc(smem_u32(&sm.A[tile][1][h * (TILE_M * 128)]));
-#pragma unroll
-                                for (int k = 0; k < KSTEPS; ++k) {
-                                    const uint64_t off = static_cast<uint64_t>((k * 32) >> 4);
-                                    umma_bf16(d_tmem, ah + off, b0 + off, kInstrDesc, (hp | k) ? 1u : 0u);
-                                }
-                                if (!low) {
+                    // A dictionary tile is NSTG stages (high and low parts of each 64-channel block).
+                    // Each row tile takes GROUP stages in a row before the other takes the same ones,
+                    // and a stage goes back to the producer after the second row tile's use: the
+                    // larger the group, the further apart the two accumulators complete (the epilogue
+                    // drains them one after the other), at the price of a shorter prefetch distance.
+                    for (int t = 0; t < T && ok; ++t, ++accn, p += NSTG) {
+                        for (int hp0 = 0; hp0 < NSTG && ok; hp0 += GROUP) {
+                            for (int tile = 0; tile < 2 && ok; ++tile) {
+                                for (int hp = hp0; hp < hp0 + GROUP; ++hp) {
+                                    const uint32_t ps = p + hp;
+                                    const int stage = ps % STAGES;
+                                    const int h = hp >> 1;
+                                    const bool low = hp & 1;      // this stage holds low parts of the atoms
+                                    if (tile == 0 && !wait_bounded_suspended(&sm.full_b[stage], (ps / STAGES) & 1, wc, 1000)) {
+                                        ok = false;
+                                        break;
+                                    }
+                                    if (hp == 0 && !wait_bounded_suspended(&sm.acc_empty[tile], (accn & 1) ^ 1, wc, 1000)) {
+                                        ok = false;
+                                        break;
+                                    }
+                                    tc_fence_after();
+                                    const uint64_t b0 = make_smem_desc(smem_u32(&sm.B[stage][0]));
+                                    const uint32_t d_tmem = tmem_base + tile * TILE_N;
+                                    const uint64_t ah = make_smem_desc(smem_u32(&sm.A[tile][0][h * (TILE_M * 128)]));
+                                    const uint64_t al = make_smem_desc(smem_u32(&sm.A[tile][1][h * (TILE_M * 128)]));
 #pragma unroll
                                     for (int k = 0; k < KSTEPS; ++k) {
                                         const uint64_t off = static_cast<uint64_t>((k * 32) >> 4);
-                                        umma_bf16(d_tmem, al + off, b0 + off, kInstrDesc, 1u);
+                                        umma_bf16(d_tmem, ah + off, b0 + off, kInstrDesc, (hp | k) ? 1u : 0u);
                                     }
+                                    if (!low) {
+#pragma unroll
+                                        for (int k = 0; k < KSTEPS; ++k) {
+                                            const uint64_t off = static_cast<uint64_t>((k * 32) >> 4);
+                                            umma_bf16(d_tmem, al + off, b0 + off, kInstrDesc, 1u);
+                                        }
+                                    }
+                                    if (tile == 1) umma_commit(&sm.empty_b[stage]);
+                                    if (hp == NSTG - 1) umma_commit(&sm.acc_full[tile]);
                                 }
-                                if (hp == 2 * KH - 1) umma_commit(&sm.acc_full[tile]);
                             }
-                            if (ok) umma_commit(&sm.empty_b[stage]);
                         }
                     }
                 }
@@ -532,12 +529,12 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                 double R[CH];
                 if (m < M) {
 #pragma unroll
-                    for (int j = 0; j < CH / 8; ++j) load_x8(X, x_dtype, m * ldx + l8 * CH + 8 * j, &R[8 * j]);
+                    for (int k = 0; k < CH / 2; ++k) load_x2(X, x_dtype, m * ldx + 2 * (8 * k + l8), R[2 * k], R[2 * k + 1]);
                 } else {
 #pragma unroll
                     for (int k = 0; k < CH; ++k) R[k] = 0.0;
                 }
-                double nn = store_residual<CH>(R, Rd_cta + static_cast<int64_t>(own_tile * TILE_M + r) * D_ + l8 * CH, Ahi, Alo, r, l8);
+                double nn = store_residual<CH>(R, Rd_cta + static_cast<int64_t>(own_tile * TILE_M + r) * D_, Ahi, Alo, r, l8);
                 nn = group8_sum(nn);
                 const float nn_o = static_cast<float>(__shfl_sync(FULL, nn, (lane & 3) * 8));
                 if ((lane >> 2) == p) band = kBandRel * sqrtf(nn_o) * 1.001f;
@@ -620,14 +617,14 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                     const int src = 4 * p + grp;
                     n = __shfl_sync(FULL, my_n1, src);
                     flags = __shfl_sync(FULL, my_flags, src);
-                    const double* Rrow = Rd_cta + static_cast<int64_t>(own_tile * TILE_M + q * 32 + src) * D_ + l8 * CH;
+                    const double* Rrow = Rd_cta + static_cast<int64_t>(own_tile * TILE_M + q * 32 + src) * D_;
 #pragma unroll
                     for (int k = 0; k < CH / 2; ++k) {
-                        const double2 v = reinterpret_cast<const double2*>(Rrow)[k];
+                        const double2 v = reinterpret_cast<const double2*>(Rrow)[8 * k + l8];
                         R[2 * k] = v.x;
                         R[2 * k + 1] = v.y;
                     }
-                    load_atom<CH>(D + static_cast<int64_t>(n) * D_ + l8 * CH, a);
+                    load_atom<CH>(D + static_cast<int64_t>(n) * D_, l8, a);
                 };
                 int n, flags;
                 double R[CH];
@@ -650,7 +647,7 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                     const int src = 4 * p + grp;
                     const int r = q * 32 + src;
                     const int64_t m = pair * ROWS + own_tile * TILE_M + r;
-                    double* Rrow = Rd_cta + static_cast<int64_t>(own_tile * TILE_M + r) * D_ + l8 * CH;
+                    double* Rrow = Rd_cta + static_cast<int64_t>(own_tile * TILE_M + r) * D_;
                     if (__any_sync(FULL, flags != 0)) {
                         // some row of this pass is not decided by its largest key alone
                         const int n_first = n;
@@ -673,7 +670,7 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                                 if (cand == 1 && !__any_sync(FULL, cmp && (flags & 2))) break;
                                 const int nc = __shfl_sync(FULL, cand ? my_n3 : my_n2, src);
                                 float ax[CH];
-                                load_atom<CH>(D + static_cast<int64_t>(nc) * D_ + l8 * CH, ax);
+                                load_atom<CH>(D + static_cast<int64_t>(nc) * D_, l8, ax);
                                 const double cc = fabs(group8_sum(slice_dot<CH>(R, ax)));
                                 if ((cand == 0 || (flags & 2)) && (cc > cbest || (cc == cbest && nc < nbest))) {
                                     cbest = cc;
@@ -682,7 +679,7 @@ encode_exact_tc_kernel(const __grid_constant__ CUtensorMap tmap_hi, const __grid
                             }
                             if (cmp) n = nbest;
                         }
-                        if (__any_sync(FULL, n != n_first)) load_atom<CH>(D + static_cast<int64_t>(n) * D_ + l8 * CH, a);
+                        if (__any_sync(FULL, n != n_first)) load_atom<CH>(D + static_cast<int64_t>(n) * D_, l8, a);
                     }
                     const double c = group8_sum(slice_dot<CH>(R, a));
 #ifdef CSR_DEBUG_CHECKS
@@ -795,7 +792,8 @@ int run(const EncodeArgs& a, const CUtensorMap& mh, const CUtensorMap& ml, doubl
     const size_t smem = sizeof(TcSmem<D_>);
     cudaError_t e = cudaFuncSetAttribute(encode_exact_tc_kernel<D_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(CSR_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    encode_exact_tc_kernel<D_><<<ctas_for(a.M), NT, smem, a.stream>>>(mh, ml, a.D, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
+    const int grid = ctas_for(a.M);
+    encode_exact_tc_kernel<D_><<<grid, NT, smem, a.stream>>>(mh, ml, a.D, a.X, a.x_dtype, a.ldx, a.M, a.N, a.s, a.out_idx,
                                                                      a.out_coef, a.coef_dtype, a.ld_code, Rd, status, diag,
                                                                      options().wait_limit_ns);
     e = cudaGetLastError();
