@@ -84,13 +84,14 @@ extern "C" {
  *                        (a) sweep on the tcgen05 tensor cores, residual and atoms each
  *                        split into a bf16 high and low part, three bf16 products per
  *                        correlation accumulated in fp32 (band 2^-12 * ||R||): the default
- *                        where the library-owned scratch is in use (no caller workspace;
+ *                        for 2048 rows or more where the library-owned scratch is in use (no
+ *                        caller workspace;
  *                        about 4 * N * d + 2048 * d * min(ceil(M / 256), SMs) bytes of it);
  *                        (b) fp32 operands and fp32 accumulation on the plain ALUs (band
  *                        1.6e-5 * ||R||), one CTA per 64 rows, no scratch: taken when a
  *                        caller workspace is given;
- *                        (c) with few rows (the vectors one decoding step adds: fewer row
- *                        tiles of 64 than half the SMs) the plain-ALU sweep with the
+ *                        (c) with few rows (the vectors one decoding step adds: fewer than
+ *                        2048) the plain-ALU sweep with the
  *                        dictionary split across the SMs instead of the rows, two launches
  *                        per iteration; library-owned scratch, not taken when a caller
  *                        workspace is given.

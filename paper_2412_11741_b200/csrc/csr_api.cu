@@ -334,7 +334,10 @@ int encode_device(const csr_encode_params_t* p, bool shared_scratch = true, cons
         // the library-owned buffer only (a caller workspace is sized for the fast mode, and two
         // encodes in flight must not share it): otherwise the row-tile encoder runs.
         const bool own = shared_scratch && !p->workspace;
-        const bool few = encode_exact_split_applies(p->M, p->N) && opt.exact_split == 0;
+        // (measured: the tensor-core encoder takes the same time for any number of rows up to one
+        // pair of row tiles per SM and overtakes the split plain-ALU encoder at about 2048 rows)
+        const bool split_ok = encode_exact_split_applies(p->M, p->N) && opt.exact_split == 0;
+        const bool few = split_ok && p->M < 2048;
         if (own && opt.exact_engine != 1 && (!few || opt.exact_engine == 2)) {
             void* base = nullptr;
             if (int rc = ensure_work(encode_exact_tc_scratch_bytes(p->M, p->d, p->N), &base, a.stream)) return rc;
@@ -346,7 +349,7 @@ int encode_device(const csr_encode_params_t* p, bool shared_scratch = true, cons
             }
             return launch_encode_exact_tc(a, align_up(static_cast<char*>(base) + kStatusBytes, 1024), status, words + kDiagWord);
         }
-        if (own && few) {
+        if (own && split_ok) {
             void* base = nullptr;
             if (int rc = ensure_work(encode_exact_split_scratch_bytes(p->M, p->d, p->N), &base, a.stream)) return rc;
             return launch_encode_exact_split(a, align_up(static_cast<char*>(base) + kStatusBytes, 1024));

@@ -36,8 +36,16 @@ def csr():
 @pytest.fixture
 def opts(csr):
     yield csr.csr_set_option
-    for name, value in (("fast_group", 0), ("fast_split", 0), ("exact_split", 0), ("wait_limit_ns", 2_000_000_000)):
+    for name, value in (("fast_group", 0), ("fast_split", 0), ("exact_split", 0), ("exact_engine", 0), ("wait_limit_ns", 2_000_000_000)):
         csr.csr_set_option(name, value)
+
+
+@pytest.fixture(params=["alu", "tensor"])
+def engine(request, csr):
+    """The exact mode's plain-ALU encoders, then its tensor-core encoder."""
+    csr.csr_set_option("exact_engine", {"alu": 1, "tensor": 2}[request.param])
+    yield request.param
+    csr.csr_set_option("exact_engine", 0)
 
 
 # ---------------------------------------------------------------------------------------
@@ -54,6 +62,8 @@ def _exact_many_tiles(csr, w, n_rows, sample, seed):
     n_tiles = (X.shape[0] + 63) // 64
     resident = 2 * torch.cuda.get_device_properties(0).multi_processor_count
     assert n_tiles >= 2 * resident + 1, "the persistent tile loop must take more than two trips"
+    # (the tensor-core encoder holds 256 rows per CTA, one CTA per SM: more than one trip there too)
+    assert (X.shape[0] + 255) // 256 > resident // 2
     idx, coef = csr.csr_encode_ex(D, Xd, w.s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
     assert csr.csr_device_status() == csr.CSR_OK
     sel = wl.stratified_rows(X.shape[0], sample, seed=seed + 1)
@@ -76,24 +86,24 @@ def _exact_many_tiles(csr, w, n_rows, sample, seed):
     return rep
 
 
-def test_exact_full_size_llama2_layer(csr):
+def test_exact_full_size_llama2_layer(csr, engine):
     """Config 2 whole (262,144 rows: 4096 row tiles over 296 resident CTAs, 14 trips)."""
     w = wl.llama2_layer()
     _exact_many_tiles(csr, w, w.M, 2048, seed=61)
 
 
-def test_exact_many_tiles_gqa_long(csr):
+def test_exact_many_tiles_gqa_long(csr, engine):
     """Config 3: 65,536 rows spread over all sequences, heads, keys and values (N = 8192, s = 16)."""
     _exact_many_tiles(csr, wl.gqa_long(), 65536, 1024, seed=62)
 
 
-def test_exact_many_tiles_sparsity_sweep_s32(csr):
+def test_exact_many_tiles_sparsity_sweep_s32(csr, engine):
     """Config 4 at s = 32: 49,152 rows."""
     _exact_many_tiles(csr, wl.sparsity_sweep(32), 49152, 512, seed=63)
 
 
 @pytest.mark.parametrize("N,d", [(16384, 128), (4096, 64)])
-def test_exact_many_tiles_dict_sweep(csr, N, d):
+def test_exact_many_tiles_dict_sweep(csr, N, d, engine):
     """Config 5: the largest dictionary, and the d = 64 chunk shape; 49,152 rows."""
     _exact_many_tiles(csr, wl.dict_sweep(N, d=d), 49152, 768, seed=64 + d)
 
