@@ -114,30 +114,49 @@ __device__ __forceinline__ float absmax3(float a, float b, float c) {
     return r;
 }
 
+// The filter's slow path, one copy for all groups: inserts the group's values (magnitudes a0..a3,
+// `tag` = tag of the first) from the largest down until what is left is below the rising
+// threshold: one trip for nearly every lane that gets here.  Returns the new state; *thr_io is
+// updated.
+struct Top4Thr {
+    Top4 q;
+    float thr;
+};
+__device__ __noinline__ Top4Thr insert_group(Top4 q, float thr, float a0, float a1, float a2, float a3, uint32_t tag, uint32_t id,
+                                             float band) {
+    float gm = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+#pragma unroll 1
+    for (int trip = 0; trip < 4 && gm >= thr; ++trip) {
+        // position of the largest magnitude left (the lowest column among equals)
+        const uint32_t pos = a0 == gm ? 0u : (a1 == gm ? 1u : (a2 == gm ? 2u : 3u));
+        top4_insert(q, (__float_as_uint(gm) & kKeyMask) | (tag - pos), id);
+        a0 = pos == 0u ? -1.f : a0;
+        a1 = pos == 1u ? -1.f : a1;
+        a2 = pos == 2u ? -1.f : a2;
+        a3 = pos == 3u ? -1.f : a3;
+        thr = __uint_as_float(q.k0 & kKeyMask) - band;
+        gm = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+    }
+    return Top4Thr{q, thr};
+}
+
 // Folds 32 columns of this thread's 128 into its top four; `tag0` is the tag of v[0] (tags fall
 // with the column so that the lowest column wins among equal magnitudes).  Four values at a
 // time are first reduced to their largest magnitude (two instructions) and only a group that
-// reaches `thr`, the running maximum less the band, is inserted value by value (a rolled loop:
-// the sweep's code has to stay small enough for the instruction cache): whatever ends up within
-// the band of the final maximum was within the band of the running one when it came by, so
-// what the filter drops can never matter.
+// reaches `thr`, the running maximum less the band, is inserted (a call: the sweep's code has
+// to stay small enough for the instruction cache): whatever ends up within the band of the
+// final maximum was within the band of the running one when it came by, so what the filter
+// drops can never matter.
 template <int J = 0>
 __device__ __forceinline__ void chunk_top4(const uint32_t (&v)[32], Top4& q, uint32_t id, uint32_t tag0, float& thr, float band) {
     if constexpr (J < 32) {
         float gm = absmax3(__uint_as_float(v[J]), __uint_as_float(v[J + 1]), __uint_as_float(v[J + 2]));
         gm = fmaxf(gm, fabsf(__uint_as_float(v[J + 3])));
         if (gm >= thr) {
-            uint32_t t0 = v[J], t1 = v[J + 1], t2 = v[J + 2], t3 = v[J + 3];
-            uint32_t tag = tag0 - J;
-#pragma unroll 1
-            for (int i = 0; i < 4; ++i) {
-                top4_insert(q, (t0 & kKeyMask) | tag, id);
-                --tag;
-                t0 = t1;
-                t1 = t2;
-                t2 = t3;
-            }
-            thr = __uint_as_float(q.k0 & kKeyMask) - band;
+            const Top4Thr r = insert_group(q, thr, fabsf(__uint_as_float(v[J])), fabsf(__uint_as_float(v[J + 1])),
+                                           fabsf(__uint_as_float(v[J + 2])), fabsf(__uint_as_float(v[J + 3])), tag0 - J, id, band);
+            q = r.q;
+            thr = r.thr;
         }
         chunk_top4<J + 4>(v, q, id, tag0, thr, band);
     }
