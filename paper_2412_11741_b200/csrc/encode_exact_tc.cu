@@ -150,15 +150,26 @@ __device__ __noinline__ Top4Thr insert_group(Top4 q, float thr, float a0, float 
 template <int J = 0>
 __device__ __forceinline__ void chunk_top4(const uint32_t (&v)[32], Top4& q, uint32_t id, uint32_t tag0, float& thr, float band) {
     if constexpr (J < 32) {
-        float gm = absmax3(__uint_as_float(v[J]), __uint_as_float(v[J + 1]), __uint_as_float(v[J + 2]));
-        gm = fmaxf(gm, fabsf(__uint_as_float(v[J + 3])));
-        if (gm >= thr) {
-            const Top4Thr r = insert_group(q, thr, fabsf(__uint_as_float(v[J])), fabsf(__uint_as_float(v[J + 1])),
-                                           fabsf(__uint_as_float(v[J + 2])), fabsf(__uint_as_float(v[J + 3])), tag0 - J, id, band);
-            q = r.q;
-            thr = r.thr;
+        // eight values per test (one branch), four per call
+        float ga = absmax3(__uint_as_float(v[J]), __uint_as_float(v[J + 1]), __uint_as_float(v[J + 2]));
+        ga = fmaxf(ga, fabsf(__uint_as_float(v[J + 3])));
+        float gb = absmax3(__uint_as_float(v[J + 4]), __uint_as_float(v[J + 5]), __uint_as_float(v[J + 6]));
+        gb = fmaxf(gb, fabsf(__uint_as_float(v[J + 7])));
+        if (fmaxf(ga, gb) >= thr) {
+            if (ga >= thr) {
+                const Top4Thr r = insert_group(q, thr, fabsf(__uint_as_float(v[J])), fabsf(__uint_as_float(v[J + 1])),
+                                               fabsf(__uint_as_float(v[J + 2])), fabsf(__uint_as_float(v[J + 3])), tag0 - J, id, band);
+                q = r.q;
+                thr = r.thr;
+            }
+            if (gb >= thr) {
+                const Top4Thr r = insert_group(q, thr, fabsf(__uint_as_float(v[J + 4])), fabsf(__uint_as_float(v[J + 5])),
+                                               fabsf(__uint_as_float(v[J + 6])), fabsf(__uint_as_float(v[J + 7])), tag0 - J - 4, id, band);
+                q = r.q;
+                thr = r.thr;
+            }
         }
-        chunk_top4<J + 4>(v, q, id, tag0, thr, band);
+        chunk_top4<J + 8>(v, q, id, tag0, thr, band);
     }
 }
 
