@@ -419,7 +419,7 @@ int csr_dict_check_norms(const void* D, int N, int d, float tol, void* stream, f
  *   "exact_split"    0 (default: the exact mode splits the dictionary for few rows), 1 = never;
  *   "exact_engine"   0 (default: the exact mode's tensor-core encoder unless the rows are few),
  *                    1 = plain-ALU encoders only, 2 = the tensor-core encoder also with few rows;
- *   "wait_limit_ns"  bound of every device-side wait of the fast encoder in nanoseconds
+ *   "wait_limit_ns"  bound of every device-side wait of the tensor-core encoders in nanoseconds
  *                    (default 2e9).  0 lets no wait outlast a single look at its barrier, so
  *                    the first hand-off that is not already complete expires: the call
  *                    returns, its outputs are unspecified and the status word reports

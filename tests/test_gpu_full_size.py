@@ -274,6 +274,35 @@ def test_bounded_wait_runs_out_and_the_library_recovers(csr, opts):
     assert rep.ok, rep.detail
 
 
+def test_bounded_wait_runs_out_in_the_exact_tensor_encoder(csr, opts):
+    """The same for the exact mode's tensor-core encoder (its eight arg-max warps also meet at
+    named barriers: they all learn of the expiry at the first one after it and leave together)."""
+    rng = np.random.default_rng(10)
+    M, N, s = 700, 600, 3
+    D = wl.normalise_rows(rng.standard_normal((N, 128)).astype(np.float32))
+    X = wl.round_to_bf16(rng.standard_normal((M, 128)).astype(np.float32))
+    Dd = torch.from_numpy(D).to(DEV)
+    Xd = torch.from_numpy(X).to(DEV).to(torch.bfloat16)
+    opts("exact_engine", 2)
+    want_i, want_c = csr.csr_encode_ex(Dd, Xd, s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
+    assert csr.csr_device_status() == csr.CSR_OK
+    word = torch.zeros(1, dtype=torch.int32, device=DEV)
+    opts("wait_limit_ns", 0)
+    csr.csr_encode_ex(Dd, Xd, s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
+    assert csr.csr_device_status() == csr.CSR_ERR_TIMEOUT
+    assert csr.csr_device_status() == csr.CSR_OK
+    csr.csr_encode_ex(Dd, Xd, s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32, dev_status=word)
+    torch.cuda.synchronize()
+    assert int(word.item()) != 0 and csr.csr_device_status() == csr.CSR_OK
+    opts("wait_limit_ns", 2_000_000_000)
+    got_i, got_c = csr.csr_encode_ex(Dd, Xd, s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32, dev_status=word)
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0
+    assert np.array_equal(_np_idx(got_i), _np_idx(want_i)) and torch.equal(got_c, want_c)
+    rep = parity.compare_exact(D, X, s, _np_idx(got_i), got_c.cpu().numpy())
+    assert rep.ok, rep.detail
+
+
 def test_two_streams_with_their_own_scratch_do_not_disturb_each_other(csr):
     """Keys and values have their own dictionaries and may be encoded side by side: with a
     workspace (or a handle) and a status word each, two calls on two streams return what each
