@@ -83,13 +83,6 @@ __device__ __forceinline__ uint32_t swz_off(int r, int chunk) {
     return kblock * (TILE_M * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
 }
 
-template <uint32_t TAG>
-__device__ __forceinline__ uint32_t masked_key(uint32_t a) {
-    uint32_t r;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(kKeyMask), "n"(TAG));
-    return r;
-}
-
 // The four largest keys seen, in descending order, and the places (2 * dictionary tile + column
 // half) the first three came from.
 struct Top4 {
@@ -116,8 +109,7 @@ __device__ __forceinline__ float absmax3(float a, float b, float c) {
 
 // The filter's slow path, one copy for all groups: inserts the group's values (magnitudes a0..a3,
 // `tag` = tag of the first) from the largest down until what is left is below the rising
-// threshold: one trip for nearly every lane that gets here.  Returns the new state; *thr_io is
-// updated.
+// threshold: one trip for nearly every lane that gets here.  Returns the new state and threshold.
 struct Top4Thr {
     Top4 q;
     float thr;
