@@ -347,7 +347,8 @@ int csr_dict_train_step(const csr_train_params_t* p);
  * pointer.  Uses library-owned device staging buffers (grow-only, per device) and two
  * library-owned streams, which first wait for everything enqueued so far on params.stream
  * (so a dictionary still being written there is complete before it is read); the fast
- * mode's bf16 copy of D is made once per call.  dev_status is ignored.
+ * mode's bf16 copy of D is made once per call; the exact mode's chunk encodes run one after
+ * the other (they share the library's scratch) under the copies.  dev_status is ignored.
  */
 int csr_encode_host(const csr_encode_params_t* p);
 

@@ -794,8 +794,26 @@ int csr_encode_host(const csr_encode_params_t* p) {
         q.workspace = nullptr;
         q.workspace_bytes = 0;
         q.dev_status = nullptr;                           // the chunks run side by side: the library's word collects them
-        rc = encode_device(&q, n_chunks == 1, prepared);
+        // The exact mode's encoders keep their scratch in the library-owned buffer: the chunks'
+        // kernels then run one after the other (each waits for the one before it, on the other
+        // stream; they fill the GPU anyway) while the copies still overlap them.
+        const bool chained = p->mode == CSR_MODE_FP32_EXACT && n_chunks > 1;
+        if (chained && j > 0) {
+            e = cudaStreamWaitEvent(st, b.ev_in[1], 0);
+            if (e != cudaSuccess) {
+                rc = fail(CSR_ERR_CUDA, "chunk ordering: %s", cudaGetErrorString(e));
+                break;
+            }
+        }
+        rc = encode_device(&q, n_chunks == 1 || chained, prepared);
         if (rc != CSR_OK) break;
+        if (chained) {
+            e = cudaEventRecord(b.ev_in[1], st);
+            if (e != cudaSuccess) {
+                rc = fail(CSR_ERR_CUDA, "chunk ordering: %s", cudaGetErrorString(e));
+                break;
+            }
+        }
         e = cudaMemcpyAsync(reinterpret_cast<char*>(p->out_idx) + (size_t)r0 * ib, b.stage_idx[slot],
                             (size_t)rows * ib, cudaMemcpyDeviceToHost, st);
         if (e == cudaSuccess)

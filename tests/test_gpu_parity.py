@@ -612,6 +612,25 @@ def test_host_entry_point(csr):
     csr.csr_dict_destroy(h)
 
 
+def test_host_entry_point_exact_mode_in_several_chunks(csr):
+    """The exact mode through the host entry point: the chunks' encodes share the library's
+    scratch, so they are chained one after the other while the copies overlap them; the codes
+    are those of the device entry point on the whole tensor, and the oracle's."""
+    w = wl.llama2_layer(tokens=1100, N=1024)        # 70400 rows: three chunks of 32768, the last ragged
+    D = torch.from_numpy(w.D).to(DEV)
+    Xh = torch.from_numpy(w.X).to(torch.bfloat16).pin_memory()
+    oi = torch.empty((w.M, w.s), dtype=torch.uint16).pin_memory()
+    oc = torch.empty((w.M, w.s), dtype=torch.float32).pin_memory()
+    csr.csr_encode_host(D, Xh, w.s, oi, oc, mode=csr.CSR_MODE_FP32_EXACT)
+    assert csr.csr_device_status() == csr.CSR_OK
+    idx, coef = csr.csr_encode_ex(D, Xh.to(DEV), w.s, mode=csr.CSR_MODE_FP32_EXACT, coef_dtype=torch.float32)
+    torch.cuda.synchronize()
+    assert np.array_equal(_np_idx(oi), _np_idx(idx)) and torch.equal(oc, coef.cpu())
+    sel = wl.stratified_rows(w.M, 1024, seed=3)
+    rep = parity.compare_exact(w.D, w.X[sel], w.s, _np_idx(oi)[sel], oc.numpy()[sel])
+    assert rep.ok, rep.detail
+
+
 # (114, 141, 534: two atoms and many iterations, the picks end up below the oracle's own rounding noise;
 # 214, 421: an overcomplete d = 64 dictionary taken to a small error, where the error ratios spread)
 @pytest.mark.parametrize("seed", list(range(24)) + [114, 141, 214, 421, 534])
